@@ -1,0 +1,123 @@
+/*
+ * gptq_b200.h -- C ABI of the B200 (sm_100a) GPTQ layer solver.
+ *
+ * The library solves the layer-wise quantization problem of Section 2 (Eq. 1):
+ * given a linear layer's weights W (d_row x d_col, here R x C) and calibration
+ * inputs X, find grid-valued weights W^ minimising ||W X - W^ X||^2, with the
+ * procedure of Algorithm 1 (Section 3).  Three calls, one per stage:
+ *
+ *   gptq_hessian_accumulate   H += 2 X X^T                 (Section 2; Alg. 1 caption)
+ *   gptq_prepare_hinv         U = Cholesky((H + lambda I)^-1)^T   (Section 3 Step 3; Alg. 1)
+ *   gptq_quantize_layer       Algorithm 1's two loops -> packed codes, scales,
+ *                             zeros, loss
+ *
+ * Conventions shared by every call
+ *   - Every pointer except `stream` is DEVICE memory owned by the caller
+ *     (unless a parameter says "host").  The library allocates no device
+ *     memory: scratch comes from the caller's workspace `ws` (256-byte
+ *     aligned, at least the size the matching *_workspace_bytes() reports).
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream) and the call returns without synchronising.
+ *   - Argument errors are reported synchronously through the return value and
+ *     nothing is enqueued.  Numerical / device-side conditions (a non-positive
+ *     pivot, a bounded wait that ran out) are written to `dev_info` and are
+ *     read by the caller after synchronising the stream; kernels never trap.
+ *   - Matrices are dense row-major.  The paper's X is d_col x m; this API takes
+ *     its transpose, token-major: X[t][c], t < n_tokens, c < C.
+ *   - C must be a multiple of 32.
+ */
+#ifndef GPTQ_B200_H_
+#define GPTQ_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  GPTQ_OK = 0,
+  GPTQ_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, C % 32 != 0, misaligned pointer */
+  GPTQ_ERR_UNSUPPORTED = 2, /* bits / group / block combination outside the supported set */
+  GPTQ_ERR_NOT_PD = 3,      /* (dev_info only) H + lambda I is not positive definite */
+  GPTQ_ERR_WORKSPACE = 4,   /* workspace missing, misaligned or too small */
+  GPTQ_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed */
+  GPTQ_ERR_TIMEOUT = 6,     /* (dev_info only) a bounded device-side wait ran out */
+  GPTQ_ERR_NONFINITE = 7    /* (dev_info only) a non-finite value was met */
+} gptq_status_t;
+
+/* bits value selecting the ternary grid {-1, 0, +1} x scale (Section 5, "Extreme
+ * Quantization"); its codes 0, 1, 2 are stored in 2-bit fields. */
+#define GPTQ_BITS_TERNARY (-1)
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* gptq_status_string(gptq_status_t status);
+
+/* ------------------------------------------------------------------ stage 1
+ * H += 2 * sum_t x_t x_t^T                     (Section 2: H_F = 2 X_F X_F^T;
+ *                                               Algorithm 1 caption: 2 X X^T)
+ *   H        [C x C] fp32, in/out.  The caller zeroes it before the first call;
+ *            calls add, so calibration batches may arrive in any chunking
+ *            (Section 5, Setup: "accumulate the layer-Hessians").  Both
+ *            triangles are valid on return.  No 1/m normalisation.
+ *   X_bf16   [n_tokens x C] bfloat16, row-major, 16-byte aligned.
+ *   n_tokens >= 0 (0 is a no-op).
+ * Products of bf16 values are exact in fp32; accumulation is fp32. */
+size_t gptq_hessian_workspace_bytes(int C, int64_t n_tokens);
+gptq_status_t gptq_hessian_accumulate(float* H, const void* X_bf16, int64_t n_tokens, int C,
+                                      void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------ stage 2
+ * lambda = damp * mean(diag H);  H~ = H + lambda I          (Section 3, Step 3)
+ * U = Cholesky(H~^-1)^T: upper triangular, positive diagonal, U^T U = H~^-1
+ *                                                          (Algorithm 1, line 3)
+ *   H        [C x C] fp32, symmetric (only its upper triangle is read); left intact.
+ *   U        [C x C] fp32, fully overwritten; the strict lower triangle is set to 0.
+ *            U must not alias H.
+ *   dev_info int[2]: [0] = GPTQ_OK or GPTQ_ERR_NOT_PD, [1] = index of the first
+ *            non-positive pivot.  On NOT_PD the contents of U are unspecified
+ *            but finite operations continue (no trap, no hang).
+ * Computed as the inverse of the upper factor of H~ = U~ U~^T, which equals
+ * Cholesky(H~^-1)^T by uniqueness of the Cholesky factor. */
+size_t gptq_prepare_hinv_workspace_bytes(int C);
+gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, float* U,
+                                void* ws, size_t ws_bytes, int* dev_info, void* stream);
+
+/* ------------------------------------------------------------------ stage 3
+ * Algorithm 1: for each block of `block` columns, quantize column by column
+ * (Q_j = quant(W_j); E_j = (W_j - Q_j) / U_jj; W[:, j:blockend] -= E_j U[j, j:blockend]),
+ * then push the block's errors onto all later columns (W[:, blockend:] -= E U[block, blockend:]).
+ *   W_fp16     [R x C] IEEE half, row-major, 16-byte aligned; not modified.
+ *   U          [C x C] fp32 from gptq_prepare_hinv.
+ *   bits       2, 3, 4, 8 or GPTQ_BITS_TERNARY.
+ *   group_size <= 0: one grid per row, fixed from the original row before the
+ *              process (Section 2; Section 5 Setup: per-row asymmetric min-max).
+ *              > 0: g consecutive weights share a grid, taken at the group's first
+ *              column from the weights as updated so far (Section 5: "always using
+ *              the most current updated weights").  Must divide C, and nest with
+ *              `block` (g % block == 0 or block % g == 0).
+ *   sym        0: asymmetric min-max grid (range widened to contain 0, integer
+ *              zero-point).  non-zero: symmetric grid, zero = (maxq+1)/2.
+ *              The ternary grid is always symmetric.
+ *   block      B of Algorithm 1: a multiple of 32 in [32, 256].  The result does
+ *              not depend on it (Section 3, Step 2) up to rounding.
+ *   qweight    [R x C*f/32] uint32, f = field width (bits; 2 for ternary): per
+ *              row a little-endian bit stream, code of column c in stream bits
+ *              [c f, c f + f), word k = stream bits [32k, 32k+32).
+ *   scales     [R x G] fp32, G = 1 (per row) or C / group_size.
+ *   zeros      [R x G] fp32 holding integer zero-points in [0, maxq].
+ *              The quantized weight is scales * (code - zeros).
+ *   loss       double[1]: sum over all weights of E^2 = (w - q)^2 / U_jj^2 (Eq. 2 summed).
+ *   dev_info   int[2], [0] = GPTQ_OK / GPTQ_ERR_NONFINITE / GPTQ_ERR_TIMEOUT.
+ * All outputs are fully overwritten. */
+size_t gptq_quantize_workspace_bytes(int R, int C, int bits, int group_size, int block);
+gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U, int R, int C,
+                                  int bits, int group_size, int sym, int block,
+                                  uint32_t* qweight, float* scales, float* zeros, double* loss,
+                                  void* ws, size_t ws_bytes, int* dev_info, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GPTQ_B200_H_ */

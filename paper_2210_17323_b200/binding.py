@@ -1,0 +1,147 @@
+"""Thin ctypes binding over libgptq_b200.so: argument marshalling only.
+
+Every step of the solver runs in the CUDA library; torch is used for device memory and
+streams.  Loading fails loudly if the library has not been built -- there is no fallback.
+Function names and argument order follow include/gptq_b200.h.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "lib", "libgptq_b200.so")
+
+BITS_TERNARY = -1
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NOT_PD, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE = range(8)
+
+EXPORTS = (
+    "gptq_status_string",
+    "gptq_hessian_workspace_bytes", "gptq_hessian_accumulate",
+    "gptq_prepare_hinv_workspace_bytes", "gptq_prepare_hinv",
+    "gptq_quantize_workspace_bytes", "gptq_quantize_layer",
+)
+
+
+class GptqError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = int(status)
+        super().__init__(f"{where}: {status_string(status)} ({int(status)})")
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2210_17323_b200.build` "
+            "(the solver has no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    c = ctypes
+    lib.gptq_status_string.restype = c.c_char_p
+    lib.gptq_status_string.argtypes = [c.c_int]
+    lib.gptq_hessian_workspace_bytes.restype = c.c_size_t
+    lib.gptq_hessian_workspace_bytes.argtypes = [c.c_int, c.c_int64]
+    lib.gptq_hessian_accumulate.restype = c.c_int
+    lib.gptq_hessian_accumulate.argtypes = [c.c_void_p, c.c_void_p, c.c_int64, c.c_int, c.c_void_p, c.c_size_t, c.c_void_p]
+    lib.gptq_prepare_hinv_workspace_bytes.restype = c.c_size_t
+    lib.gptq_prepare_hinv_workspace_bytes.argtypes = [c.c_int]
+    lib.gptq_prepare_hinv.restype = c.c_int
+    lib.gptq_prepare_hinv.argtypes = [c.c_void_p, c.c_float, c.c_int, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
+    lib.gptq_quantize_workspace_bytes.restype = c.c_size_t
+    lib.gptq_quantize_workspace_bytes.argtypes = [c.c_int] * 5
+    lib.gptq_quantize_layer.restype = c.c_int
+    lib.gptq_quantize_layer.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_int, c.c_int, c.c_int,
+                                        c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+                                        c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
+    return lib
+
+
+_lib = _load()
+
+
+def status_string(status) -> str:
+    return _lib.gptq_status_string(int(status)).decode()
+
+
+def _stream_ptr(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(t, dtype, name):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+
+
+def _ws(nbytes, device, ws):
+    if ws is not None and ws.numel() * ws.element_size() >= nbytes:
+        return ws
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def field_bits(bits: int) -> int:
+    return 2 if bits == BITS_TERNARY else bits
+
+
+def gptq_hessian_workspace_bytes(C, n_tokens):
+    return _lib.gptq_hessian_workspace_bytes(C, n_tokens)
+
+
+def gptq_prepare_hinv_workspace_bytes(C):
+    return _lib.gptq_prepare_hinv_workspace_bytes(C)
+
+
+def gptq_quantize_workspace_bytes(R, C, bits, group_size, block):
+    return _lib.gptq_quantize_workspace_bytes(R, C, bits, group_size, block)
+
+
+def gptq_hessian_accumulate(H, X, n_tokens=None, ws=None, stream=None):
+    """H += 2 X^T X for token-major bf16 X (n_tokens x C).  H: C x C fp32, zeroed by the caller first."""
+    _check(H, torch.float32, "H")
+    _check(X, torch.bfloat16, "X")
+    C = H.shape[0]
+    n = X.shape[0] if n_tokens is None else int(n_tokens)
+    ws = _ws(_lib.gptq_hessian_workspace_bytes(C, n), H.device, ws)
+    st = _lib.gptq_hessian_accumulate(H.data_ptr(), X.data_ptr(), n, C, ws.data_ptr(), ws.numel(), _stream_ptr(stream))
+    if st != OK:
+        raise GptqError(st, "gptq_hessian_accumulate")
+    return H
+
+
+def gptq_prepare_hinv(H, damp=0.01, U=None, ws=None, dev_info=None, stream=None):
+    """U = Cholesky((H + damp*mean(diag H) I)^-1)^T.  Returns (U, dev_info); dev_info is read by the caller after a sync."""
+    _check(H, torch.float32, "H")
+    C = H.shape[0]
+    U = torch.empty_like(H) if U is None else U
+    _check(U, torch.float32, "U")
+    dev_info = torch.zeros(2, dtype=torch.int32, device=H.device) if dev_info is None else dev_info
+    ws = _ws(_lib.gptq_prepare_hinv_workspace_bytes(C), H.device, ws)
+    st = _lib.gptq_prepare_hinv(H.data_ptr(), float(damp), C, U.data_ptr(), ws.data_ptr(), ws.numel(),
+                                dev_info.data_ptr(), _stream_ptr(stream))
+    if st != OK:
+        raise GptqError(st, "gptq_prepare_hinv")
+    return U, dev_info
+
+
+def gptq_quantize_layer(W, U, bits, group_size=0, sym=False, block=128, ws=None, dev_info=None, stream=None):
+    """Algorithm 1 on fp16 W (R x C) with U from gptq_prepare_hinv.
+    Returns dict(qweight uint32 [R, C*f/32] (as int32 tensor), scales [R,G], zeros [R,G], loss double[1], dev_info)."""
+    _check(W, torch.float16, "W")
+    _check(U, torch.float32, "U")
+    R, C = W.shape
+    G = C // group_size if group_size > 0 else 1
+    f = field_bits(bits)
+    dev = W.device
+    qweight = torch.empty((R, C * f // 32), dtype=torch.int32, device=dev)
+    scales = torch.empty((R, G), dtype=torch.float32, device=dev)
+    zeros = torch.empty((R, G), dtype=torch.float32, device=dev)
+    loss = torch.zeros(1, dtype=torch.float64, device=dev)
+    dev_info = torch.zeros(2, dtype=torch.int32, device=dev) if dev_info is None else dev_info
+    ws = _ws(_lib.gptq_quantize_workspace_bytes(R, C, bits, group_size, block), dev, ws)
+    st = _lib.gptq_quantize_layer(W.data_ptr(), U.data_ptr(), R, C, bits, group_size, int(bool(sym)), block,
+                                  qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), loss.data_ptr(),
+                                  ws.data_ptr(), ws.numel(), dev_info.data_ptr(), _stream_ptr(stream))
+    if st != OK:
+        raise GptqError(st, "gptq_quantize_layer")
+    return dict(qweight=qweight, scales=scales, zeros=zeros, loss=loss, dev_info=dev_info)

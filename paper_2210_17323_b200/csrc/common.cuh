@@ -1,0 +1,49 @@
+// Shared host/device helpers of the GPTQ B200 library (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/gptq_b200.h"
+
+namespace gptq {
+
+constexpr size_t kAlign = 256;
+
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+
+// Carves 256-byte aligned pieces out of the caller's workspace; with base == nullptr it only measures.
+struct WsCarver {
+  char* base;
+  size_t off = 0;
+  explicit WsCarver(void* b) : base(static_cast<char*>(b)) {}
+  template <class T>
+  T* take(size_t count) {
+    size_t o = off;
+    off = align_up(off + count * sizeof(T));
+    return base ? reinterpret_cast<T*>(base + o) : nullptr;
+  }
+};
+
+inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+#define GPTQ_CUDA_TRY(expr)                           \
+  do {                                                \
+    cudaError_t _e = (expr);                          \
+    if (_e != cudaSuccess) return GPTQ_ERR_CUDA;      \
+  } while (0)
+
+#define GPTQ_LAUNCH_CHECK() GPTQ_CUDA_TRY(cudaGetLastError())
+
+// dev_info word layout: [0] status, [1] detail (pivot index, ...).  First error wins.
+__device__ __forceinline__ void report_error(int* dev_info, int status, int detail) {
+  if (dev_info && atomicCAS(dev_info, 0, status) == 0) dev_info[1] = detail;
+}
+
+__device__ __forceinline__ int ceil_div_d(int a, int b) { return (a + b - 1) / b; }
+inline int ceil_div(int64_t a, int64_t b) { return static_cast<int>((a + b - 1) / b); }
+
+}  // namespace gptq

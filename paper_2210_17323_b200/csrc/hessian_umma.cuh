@@ -1,0 +1,9 @@
+// Tensor-core (tcgen05 / TMEM / TMA) path of the Hessian accumulation; see hessian_umma.cu.
+#pragma once
+#include "common.cuh"
+
+namespace gptq {
+bool hessian_umma_supported(int C, int64_t n_tokens);
+gptq_status_t hessian_umma(float* H, const __nv_bfloat16* X, int64_t n_tokens, int C, cudaStream_t stream);
+cudaError_t launch_mirror_upper_to_lower(float* H, int C, cudaStream_t stream);
+}  // namespace gptq

@@ -1,0 +1,354 @@
+// Stage 3: Algorithm 1's two loops -- column-by-column quantization with error feedback inside a
+// block of B columns, and lazy batched updates of the later columns (Section 3, Steps 1-3).
+//
+// Organisation on the GPU (an exact regrouping of Algorithm 1's updates; Section 3, Step 2 notes
+// that the rounding decisions of a column depend only on the updates that reached that column):
+//   * Columns are processed in OUTER blocks of B2 (about 1024) columns.  When an outer block
+//     starts, its working weights are produced in one contraction from the ORIGINAL weights and
+//     all errors so far:  Wblk = W[:, blk] - E[:, :i2] * U[:i2, blk]  ("left-looking" form of the
+//     lazy update W[:, (i+B):] -= E * U[i:(i+B), (i+B):] accumulated over all earlier blocks).
+//   * Inside an outer block the paper's loop runs with the caller's block size B: the in-block
+//     kernel quantizes B columns with immediate error feedback, then the block's errors are
+//     pushed onto the remaining columns of the outer block.
+//   * Working weights of the current outer block are fp64; E is kept in fp32; update sums are
+//     fp32-accurate.  Each weight therefore meets one rounding at fp32 level (its update sum)
+//     instead of one per preceding block.
+#include "common.cuh"
+#include "gemm_simt.cuh"
+
+namespace gptq {
+namespace {
+
+constexpr int kSB = 32;  // columns held in registers at a time by the in-block kernel
+
+struct GridSpec {
+  int maxq;        // largest code
+  int symmetric;   // symmetric (or ternary) grid
+};
+
+// Min-max grid of a set of weights with minimum mn and maximum mx (Section 5, Setup).  The range
+// is widened to contain 0 so the zero-point is an integer code; an all-zero set gets [-1, 1].
+// The scale is rounded to fp32, the precision it is returned in, and used as that value.
+__device__ __forceinline__ void find_params(double mn, double mx, GridSpec g, float& scale, float& zero) {
+  double xmin = fmin(mn, 0.0), xmax = fmax(mx, 0.0);
+  if (xmin == 0.0 && xmax == 0.0) { xmin = -1.0; xmax = 1.0; }
+  if (g.symmetric) {
+    double a = fmax(fabs(xmin), xmax);
+    scale = (float)(2.0 * a / (double)g.maxq);
+    zero = (float)((g.maxq + 1) / 2);
+  } else {
+    scale = (float)((xmax - xmin) / (double)g.maxq);
+    zero = (float)rint(-xmin / (double)scale);
+  }
+}
+
+// ---- per-row static grid from the original fp16 weights: one warp per row ----------------------
+__global__ void rowgrid_kernel(const __half* __restrict__ W, int R, int C, GridSpec g,
+                               float* __restrict__ scales, float* __restrict__ zeros) {
+  int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= R) return;
+  const uint4* p = reinterpret_cast<const uint4*>(W + (int64_t)row * C);
+  float mn = INFINITY, mx = -INFINITY;
+  for (int i = lane; i < C / 8; i += 32) {
+    uint4 v = p[i];
+    const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      float2 f = __half22float2(h[k]);
+      mn = fminf(mn, fminf(f.x, f.y));
+      mx = fmaxf(mx, fmaxf(f.x, f.y));
+    }
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  }
+  if (lane == 0) find_params((double)mn, (double)mx, g, scales[row], zeros[row]);
+}
+
+// ---- grid of a group wider than the block: one warp per row over the working weights ----------
+__global__ void groupgrid_kernel(const double* __restrict__ Wblk, int64_t ldw, int col0, int g, int R,
+                                 GridSpec gs, float* __restrict__ scales, float* __restrict__ zeros,
+                                 int G, int gi) {
+  int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= R) return;
+  const double* p = Wblk + (int64_t)row * ldw + col0;
+  double mn = INFINITY, mx = -INFINITY;
+  for (int i = lane; i < g; i += 32) { mn = fmin(mn, p[i]); mx = fmax(mx, p[i]); }
+  for (int o = 16; o > 0; o >>= 1) {
+    mn = fmin(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  }
+  if (lane == 0) find_params(mn, mx, gs, scales[(int64_t)row * G + gi], zeros[(int64_t)row * G + gi]);
+}
+
+// ---- first outer block: working weights are the original weights -------------------------------
+__global__ void wblk_from_w16_kernel(const __half* __restrict__ W, int R, int C, int nb,
+                                     double* __restrict__ Wblk, int64_t ldw) {
+  int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)R * nb) return;
+  int r = (int)(idx / nb), c = (int)(idx % nb);
+  Wblk[(int64_t)r * ldw + c] = (double)__half2float(W[(int64_t)r * C + c]);
+}
+
+// ---- the in-block loop (Algorithm 1, inner FOR) -------------------------------------------------
+struct InblockArgs {
+  const double* Wblk; int64_t ldw; int col0;  // working weights; col0 = first column of this block in Wblk
+  const float* U; int C; int i; int B;         // global first column i, width B (multiple of 32, <= 256)
+  int R; GridSpec grid;
+  int group;        // group size (<= 0: one grid per row)
+  int grid_inside;  // 1: grids of groups that start in this block are computed here (group <= B)
+  float* scales; float* zeros; int G;
+  float* E; uint8_t* codes; double* loss; int* dev_info;
+};
+
+// One thread per row.  The block's working weights sit in shared memory, column-major (thread-
+// private columns, conflict-free); 32 columns at a time are held in registers, quantized one
+// after the other with immediate feedback (W[:, j:blockend] -= E_j U[j, j:blockend]) inside the
+// registers, then their 32 errors are applied to the rest of the block in shared memory.
+template <int RPB>
+__global__ void __launch_bounds__(RPB) inblock_kernel(InblockArgs a) {
+  extern __shared__ double smem[];
+  const int B = a.B, LDS = RPB + 1;
+  double* slab = smem;                  // [B][LDS]
+  double* Us = smem + (size_t)B * LDS;  // [kSB][B]   rows j0..j0+31 of the B x B block of U
+  const int t = threadIdx.x, r0 = blockIdx.x * RPB, row = r0 + t;
+  const bool live = row < a.R;
+
+  // stage the slab: coalesced along columns, transposed into shared memory
+  for (int e = t; e < RPB * B; e += RPB) {
+    int rr = e / B, c = e % B;
+    slab[c * LDS + rr] = (r0 + rr < a.R) ? a.Wblk[(int64_t)(r0 + rr) * a.ldw + a.col0 + c] : 0.0;
+  }
+  const int G = a.G;
+  const int g = a.group;
+  float scale_f = 1.f, zero_f = 0.f;
+  if (live && !(a.grid_inside)) {
+    int gi = g > 0 ? a.i / g : 0;
+    scale_f = a.scales[(int64_t)row * G + gi];
+    zero_f = a.zeros[(int64_t)row * G + gi];
+  }
+  double scale = (double)scale_f, zero = (double)zero_f;
+  const double maxq = (double)a.grid.maxq;
+  double loss = 0.0;
+  bool bad = false;
+
+  for (int j0 = 0; j0 < B; j0 += kSB) {
+    __syncthreads();  // slab staged / previous sub-block's Us no longer read
+    for (int e = t; e < kSB * B; e += RPB) {
+      int jj = e / B, c = e % B;
+      Us[jj * B + c] = (c >= j0) ? (double)a.U[(int64_t)(a.i + j0 + jj) * a.C + a.i + c] : 0.0;
+    }
+    __syncthreads();
+    double w[kSB], err[kSB];
+    uint32_t cw[kSB / 4];
+#pragma unroll
+    for (int jj = 0; jj < kSB; ++jj) w[jj] = slab[(j0 + jj) * LDS + t];
+#pragma unroll
+    for (int k = 0; k < kSB / 4; ++k) cw[k] = 0;
+
+    // group grid starting at this sub-block (group a multiple of 32, within the block)
+    if (a.grid_inside && g >= kSB && ((a.i + j0) % g) == 0) {
+      double mn = INFINITY, mx = -INFINITY;
+      for (int c = j0; c < j0 + g; ++c) { double v = slab[c * LDS + t]; mn = fmin(mn, v); mx = fmax(mx, v); }
+      find_params(mn, mx, a.grid, scale_f, zero_f);
+      scale = (double)scale_f; zero = (double)zero_f;
+      if (live) {
+        int gi = (a.i + j0) / g;
+        a.scales[(int64_t)row * G + gi] = scale_f; a.zeros[(int64_t)row * G + gi] = zero_f;
+      }
+    }
+#pragma unroll
+    for (int jj = 0; jj < kSB; ++jj) {
+      if (a.grid_inside && g < kSB && (jj % g) == 0) {   // small groups live inside the registers
+        double mn = INFINITY, mx = -INFINITY;
+#pragma unroll
+        for (int kk = 0; kk < kSB; ++kk)
+          if (kk >= jj && kk < jj + g) { mn = fmin(mn, w[kk]); mx = fmax(mx, w[kk]); }
+        find_params(mn, mx, a.grid, scale_f, zero_f);
+        scale = (double)scale_f; zero = (double)zero_f;
+        if (live) {
+          int gi = (a.i + j0 + jj) / g;
+          a.scales[(int64_t)row * G + gi] = scale_f; a.zeros[(int64_t)row * G + gi] = zero_f;
+        }
+      }
+      const double d = Us[jj * B + j0 + jj];
+      double q = rint(w[jj] / scale) + zero;                 // quantize column
+      q = fmin(fmax(q, 0.0), maxq);
+      const double wq = scale * (q - zero);
+      const double e = (w[jj] - wq) / d;                     // quantization error
+      err[jj] = e;
+      loss += e * e;
+      bad |= !isfinite(e);
+      cw[jj >> 2] |= (uint32_t)q << (8 * (jj & 3));
+#pragma unroll
+      for (int kk = jj + 1; kk < kSB; ++kk) w[kk] -= e * Us[jj * B + j0 + kk];   // update weights in block
+    }
+    // remaining columns of the block: apply the 32 errors of this sub-block
+    for (int c = j0 + kSB; c < B; ++c) {
+      double x = slab[c * LDS + t];
+#pragma unroll
+      for (int jj = 0; jj < kSB; ++jj) x -= err[jj] * Us[jj * B + c];
+      slab[c * LDS + t] = x;
+    }
+    if (live) {
+      float4* ep = reinterpret_cast<float4*>(a.E + (int64_t)row * a.C + a.i + j0);
+#pragma unroll
+      for (int k = 0; k < kSB / 4; ++k)
+        ep[k] = make_float4((float)err[4 * k], (float)err[4 * k + 1], (float)err[4 * k + 2], (float)err[4 * k + 3]);
+      uint4* cp = reinterpret_cast<uint4*>(a.codes + (int64_t)row * a.C + a.i + j0);
+      cp[0] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+      cp[1] = make_uint4(cw[4], cw[5], cw[6], cw[7]);
+    }
+  }
+  if (!live) loss = 0.0;
+  for (int o = 16; o > 0; o >>= 1) loss += __shfl_down_sync(0xffffffffu, loss, o);
+  if ((t & 31) == 0 && loss != 0.0) atomicAdd(a.loss, loss);
+  if (live && bad) report_error(a.dev_info, GPTQ_ERR_NONFINITE, row);
+}
+
+// ---- pack codes: little-endian bit stream per row, field width f --------------------------------
+__global__ void pack_kernel(const uint8_t* __restrict__ codes, int R, int C, int f,
+                            uint32_t* __restrict__ qweight) {
+  const int nwords = C * f / 32;
+  int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)R * nwords) return;
+  int r = (int)(idx / nwords), k = (int)(idx % nwords);
+  const uint8_t* c = codes + (int64_t)r * C;
+  int lo = 32 * k / f, hi = (32 * k + 31) / f;
+  uint32_t word = 0;
+  for (int col = lo; col <= hi; ++col) {
+    int sh = col * f - 32 * k;
+    uint32_t v = c[col];
+    word |= sh >= 0 ? (v << sh) : (v >> (-sh));
+  }
+  qweight[idx] = word;
+}
+
+// ---- contraction functors -----------------------------------------------------------------------
+struct ElemE {  // A(m, k) = E[m][kofs + k]
+  static constexpr bool kInnerContig = true;
+  const float* E; int64_t C; int kofs;
+  __device__ __forceinline__ float operator()(int m, int k) const { return E[(int64_t)m * C + kofs + k]; }
+};
+struct ElemU {  // B(k, n) = U[kofs + k][nofs + n]
+  static constexpr bool kInnerContig = true;
+  const float* U; int64_t C; int kofs, nofs;
+  __device__ __forceinline__ float operator()(int k, int n) const { return U[(int64_t)(kofs + k) * C + nofs + n]; }
+};
+struct EpiInitWblk {  // Wblk[m][n] = W16[m][i2 + n] - acc
+  const __half* W; int64_t C; int i2; double* Wblk; int64_t ldw;
+  __device__ __forceinline__ void operator()(int m, int n, float acc) const {
+    Wblk[(int64_t)m * ldw + n] = (double)__half2float(W[(int64_t)m * C + i2 + n]) - (double)acc;
+  }
+};
+struct EpiSubWblk {  // Wblk[m][nofs + n] -= acc
+  double* Wblk; int64_t ldw; int nofs;
+  __device__ __forceinline__ void operator()(int m, int n, float acc) const {
+    Wblk[(int64_t)m * ldw + nofs + n] -= (double)acc;
+  }
+};
+
+inline int field_bits(int bits) { return bits == GPTQ_BITS_TERNARY ? 2 : bits; }
+inline bool bits_ok(int bits) { return bits == 2 || bits == 3 || bits == 4 || bits == 8 || bits == GPTQ_BITS_TERNARY; }
+
+// Outer (lazy) block width: a multiple of both the block and any group wider than it, about 1024.
+inline int outer_block(int C, int group, int block) {
+  int unit = (group > block) ? group : block;
+  int b2 = unit * (1024 / unit > 0 ? 1024 / unit : 1);
+  return b2 < C ? b2 : C;
+}
+
+}  // namespace
+}  // namespace gptq
+
+extern "C" size_t gptq_quantize_workspace_bytes(int R, int C, int bits, int group_size, int block) {
+  using namespace gptq;
+  if (R <= 0 || C <= 0 || block <= 0 || !bits_ok(bits)) return 0;
+  WsCarver w(nullptr);
+  w.take<double>((size_t)R * outer_block(C, group_size, block));  // working weights of the outer block
+  w.take<float>((size_t)R * C);                                   // E, all columns
+  w.take<uint8_t>((size_t)R * C);                                 // unpacked codes
+  return w.off;
+}
+
+extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U, int R, int C,
+                                             int bits, int group_size, int sym, int block,
+                                             uint32_t* qweight, float* scales, float* zeros, double* loss,
+                                             void* ws, size_t ws_bytes, int* dev_info, void* stream) {
+  using namespace gptq;
+  if (!W_fp16 || !U || !qweight || !scales || !zeros || !loss || !dev_info || R <= 0 || C <= 0 || C % 32 != 0)
+    return GPTQ_ERR_INVALID_ARG;
+  if (!aligned_to(W_fp16, 16) || !aligned_to(U, 16)) return GPTQ_ERR_INVALID_ARG;
+  if (!bits_ok(bits)) return GPTQ_ERR_UNSUPPORTED;
+  if (block <= 0) return GPTQ_ERR_INVALID_ARG;
+  if (block % 32 != 0 || block > 256) return GPTQ_ERR_UNSUPPORTED;
+  const int g = group_size > 0 ? group_size : 0;
+  if (g > 0) {
+    if (C % g != 0) return GPTQ_ERR_INVALID_ARG;
+    if (g % block != 0 && block % g != 0) return GPTQ_ERR_INVALID_ARG;   // groups and blocks must nest
+    if (g % kSB != 0 && kSB % g != 0) return GPTQ_ERR_UNSUPPORTED;
+  }
+  if (!ws || !aligned_to(ws, kAlign) || ws_bytes < gptq_quantize_workspace_bytes(R, C, bits, group_size, block))
+    return GPTQ_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const __half* W = static_cast<const __half*>(W_fp16);
+  const int B2 = outer_block(C, g, block);
+  const int G = g > 0 ? C / g : 1;
+  WsCarver w(ws);
+  double* Wblk = w.take<double>((size_t)R * B2);
+  float* E = w.take<float>((size_t)R * C);
+  uint8_t* codes = w.take<uint8_t>((size_t)R * C);
+  const int64_t ldw = B2;
+  GridSpec gs{bits == GPTQ_BITS_TERNARY ? 2 : (1 << bits) - 1, (sym != 0 || bits == GPTQ_BITS_TERNARY) ? 1 : 0};
+
+  GPTQ_CUDA_TRY(cudaMemsetAsync(dev_info, 0, 2 * sizeof(int), s));
+  GPTQ_CUDA_TRY(cudaMemsetAsync(loss, 0, sizeof(double), s));
+  if (g == 0) {
+    rowgrid_kernel<<<ceil_div(R, 8), 256, 0, s>>>(W, R, C, gs, scales, zeros);
+    GPTQ_LAUNCH_CHECK();
+  }
+  const int rpb = block > 128 ? 64 : 128;
+  auto inblock_smem = [&](int B) { return (size_t)((size_t)B * (rpb + 1) + (size_t)kSB * B) * sizeof(double); };
+  GPTQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)((256 * 65 + kSB * 256) * sizeof(double))));
+  GPTQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)((128 * 129 + kSB * 128) * sizeof(double))));
+
+  for (int i2 = 0; i2 < C; i2 += B2) {
+    const int nb2 = (C - i2 < B2) ? C - i2 : B2;
+    // working weights of the outer block: original weights minus all updates from columns < i2
+    if (i2 == 0) {
+      int64_t total = (int64_t)R * nb2;
+      wblk_from_w16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(W, R, C, nb2, Wblk, ldw);
+      GPTQ_LAUNCH_CHECK();
+    } else {
+      GPTQ_CUDA_TRY(launch_gemm_simt(R, nb2, 1, ElemE{E, C, 0}, ElemU{U, C, 0, i2}, FullRange{i2},
+                                     EpiInitWblk{W, C, i2, Wblk, ldw}, s));
+    }
+    for (int i = i2; i < i2 + nb2; i += block) {
+      const int B = (i2 + nb2 - i < block) ? i2 + nb2 - i : block;
+      if (g > B && i % g == 0) {   // a group wider than the block starts here
+        groupgrid_kernel<<<ceil_div(R, 8), 256, 0, s>>>(Wblk, ldw, i - i2, g, R, gs, scales, zeros, G, i / g);
+        GPTQ_LAUNCH_CHECK();
+      }
+      InblockArgs a{Wblk, ldw, i - i2, U, C, i, B, R, gs, g, (g > 0 && g <= B) ? 1 : 0,
+                    scales, zeros, G, E, codes, loss, dev_info};
+      if (rpb == 64) inblock_kernel<64><<<ceil_div(R, 64), 64, inblock_smem(B), s>>>(a);
+      else inblock_kernel<128><<<ceil_div(R, 128), 128, inblock_smem(B), s>>>(a);
+      GPTQ_LAUNCH_CHECK();
+      // push this block's errors onto the remaining columns of the outer block
+      const int rest = i2 + nb2 - (i + B);
+      if (rest > 0)
+        GPTQ_CUDA_TRY(launch_gemm_simt(R, rest, 1, ElemE{E, C, i}, ElemU{U, C, i, i + B}, FullRange{B},
+                                       EpiSubWblk{Wblk, ldw, i + B - i2}, s));
+    }
+  }
+  {
+    const int f = field_bits(bits);
+    int64_t total = (int64_t)R * (C * f / 32);
+    pack_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(codes, R, C, f, qweight);
+    GPTQ_LAUNCH_CHECK();
+  }
+  return GPTQ_OK;
+}

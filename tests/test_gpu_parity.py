@@ -1,0 +1,209 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 oracle, element by element."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+from oracle import gptq_oracle as O
+from paper_2210_17323_b200.synth import generator as G, workloads as WL
+from tests.parity_utils import (TOL_H_FRO, TOL_U_FRO, check_quantize_outputs, rel_fro)
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2210_17323_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def D():
+    from paper_2210_17323_b200.synth import device
+    return device
+
+
+def _np_bf16_to_torch(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def _layer(R, C, m, cfg=9, blk=0, kind="q"):
+    return WL.Layer(cfg, blk, kind, R, C, m)
+
+
+def _run_quant(B, W16, U32, bits, group, sym, block):
+    out = B.gptq_quantize_layer(torch.from_numpy(W16).cuda(), torch.from_numpy(U32).cuda(), bits, group, sym, block)
+    torch.cuda.synchronize()
+    assert out["dev_info"].tolist()[0] == 0
+    return dict(qweight=out["qweight"].cpu().numpy(), scales=out["scales"].cpu().numpy(),
+                zeros=out["zeros"].cpu().numpy(), loss=out["loss"].item())
+
+
+# ------------------------------------------------------------------ inputs
+def test_device_filler_matches_host_generator(D):
+    L = _layer(96, 160, 300)
+    X = D.fill_x(L).view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(X, L.x_bits())
+    assert np.array_equal(D.fill_x(L, 17, 200).view(torch.int16).cpu().numpy().view(np.uint16), L.x_bits(17, 200))
+    W = D.fill_w(L).cpu().numpy()
+    assert np.array_equal(W.view(np.uint16), L.w().view(np.uint16))
+
+
+# ------------------------------------------------------------------ stage 1
+@pytest.mark.parametrize("C,m", [(32, 1), (96, 77), (160, 1000), (256, 4096), (768, 8192)])
+def test_hessian_matches_oracle(B, C, m):
+    L = _layer(8, C, m)
+    bits = L.x_bits()
+    H = torch.zeros((C, C), dtype=torch.float32, device="cuda")
+    B.gptq_hessian_accumulate(H, _np_bf16_to_torch(bits))
+    Hg = H.cpu().numpy()
+    Href = O.hessian_accumulate(np.zeros((C, C)), bits)
+    assert rel_fro(Hg, Href) <= TOL_H_FRO
+    assert np.array_equal(Hg, Hg.T)
+
+
+def test_hessian_integer_inputs_bit_exact_and_chunked(B):
+    r = np.random.default_rng(3)
+    C, m = 160, 700
+    Xi = r.integers(-8, 9, size=(m, C)).astype(np.float32)
+    Xt = torch.from_numpy(Xi).cuda().to(torch.bfloat16)
+    H = torch.zeros((C, C), dtype=torch.float32, device="cuda")
+    for a, b in ((0, 33), (33, 512), (512, 700)):      # accumulate over ragged chunks
+        B.gptq_hessian_accumulate(H, Xt[a:b].contiguous())
+    exact = 2.0 * (Xi.astype(np.float64).T @ Xi.astype(np.float64))
+    assert np.array_equal(H.cpu().numpy().astype(np.float64), exact)
+    B.gptq_hessian_accumulate(H, Xt[:0].contiguous())   # empty batch: no-op
+    assert np.array_equal(H.cpu().numpy().astype(np.float64), exact)
+
+
+# ------------------------------------------------------------------ stage 2
+@pytest.mark.parametrize("C", [32, 96, 160, 768])
+def test_prepare_hinv_matches_oracle(B, C):
+    L = _layer(8, C, 4 * C + 100)
+    H64 = O.hessian_accumulate(np.zeros((C, C)), L.x_bits())
+    H32 = H64.astype(np.float32)
+    U, info = B.gptq_prepare_hinv(torch.from_numpy(H32).cuda(), 0.01)
+    torch.cuda.synchronize()
+    assert info.tolist() == [0, 0]
+    Ug = U.cpu().numpy()
+    Uref = O.cholesky_inverse_upper(O.dampen(H32.astype(np.float64), 0.01)[0])
+    assert np.array_equal(Ug, np.triu(Ug)) and (np.diag(Ug) > 0).all()
+    assert rel_fro(Ug, Uref) <= TOL_U_FRO
+    # row-wise: every row of U from the diagonal on, relative to that row's norm
+    row_err = np.linalg.norm(Ug - Uref, axis=1) / np.linalg.norm(Uref, axis=1)
+    assert row_err.max() <= 1e-4
+
+
+def test_prepare_hinv_reports_not_positive_definite(B):
+    C = 64
+    H = np.eye(C, dtype=np.float32)
+    H[10, 20] = H[20, 10] = 5.0      # indefinite
+    U, info = B.gptq_prepare_hinv(torch.from_numpy(H).cuda(), 0.01)
+    torch.cuda.synchronize()
+    st, where = info.tolist()
+    assert st == B.ERR_NOT_PD and 0 <= where < C
+    assert torch.isfinite(U).all()
+    # all-zero H (no calibration data): damping cannot help
+    U, info = B.gptq_prepare_hinv(torch.zeros((C, C), device="cuda"), 0.01)
+    torch.cuda.synchronize()
+    assert info.tolist()[0] == B.ERR_NOT_PD
+
+
+# ------------------------------------------------------------------ stage 3 (oracle's U on both sides)
+CASES = [
+    # R,   C,   bits, group, sym, block
+    (200, 768, 4, 0, False, 128),
+    (129, 160, 3, 0, False, 128),      # ragged rows, short last block
+    (7, 96, 4, 0, False, 32),
+    (1, 32, 2, 0, False, 32),
+    (300, 512, 3, 128, False, 128),
+    (300, 512, 2, 128, False, 64),     # group wider than block
+    (300, 512, 2, 128, False, 256),    # block wider than group
+    (64, 256, O.BITS_TERNARY, 128, False, 32),
+    (64, 256, 4, 16, False, 128),      # small groups inside the register sub-block
+    (64, 256, 8, 0, False, 128),
+    (64, 256, 4, 64, True, 64),        # symmetric grid
+    (260, 2304, 4, 0, False, 128),     # several outer (lazy) blocks
+    (130, 2176, 3, 128, False, 96),    # block that is not a power of two; ragged outer block
+]
+
+
+@pytest.mark.parametrize("R,C,bits,group,sym,block", CASES)
+def test_quantize_layer_matches_oracle(B, R, C, bits, group, sym, block):
+    if group and (group % block and block % group):
+        pytest.skip("not nested")
+    L = _layer(R, C, 2 * C + 64, cfg=8)
+    W16 = L.w()
+    H = O.hessian_accumulate(np.zeros((C, C)), L.x_bits())
+    U32 = O.cholesky_inverse_upper(O.dampen(H, 0.01)[0]).astype(np.float32)
+    ref = O.quantize_layer(W16, U32.astype(np.float64), bits, group, sym, block)
+    gpu = _run_quant(B, W16, U32, bits, group, sym, block)
+    check_quantize_outputs(gpu, ref, W16, bits, C, H)
+
+
+def test_quantize_block_size_invariance_on_gpu(B):
+    R, C = 128, 1024
+    L = _layer(R, C, 3000, cfg=7)
+    W16 = L.w()
+    H = O.hessian_accumulate(np.zeros((C, C)), L.x_bits())
+    U32 = O.cholesky_inverse_upper(O.dampen(H, 0.01)[0]).astype(np.float32)
+    outs = [_run_quant(B, W16, U32, 2, 128, False, blk) for blk in (32, 64, 128, 256)]
+    ref = O.quantize_layer(W16, U32.astype(np.float64), 2, 128, False, 128)
+    for o in outs:
+        check_quantize_outputs(o, ref, W16, 2, C, H)
+
+
+def test_quantize_degenerate_inputs(B):
+    C = 64
+    U32 = np.eye(C, dtype=np.float32)
+    # all-zero weights: grid [-1, 1], every code = zero-point, loss 0
+    out = _run_quant(B, np.zeros((3, C), np.float16), U32, 4, 0, False, 32)
+    ref = O.quantize_layer(np.zeros((3, C), np.float16), U32.astype(np.float64), 4, 0, False, 32)
+    check_quantize_outputs(out, ref, np.zeros((3, C), np.float16), 4, C)
+    assert out["loss"] == 0.0
+    # weights already on their own grid are reproduced exactly
+    lv = np.random.default_rng(12).integers(0, 16, size=(5, C))
+    lv[:, 0], lv[:, 1] = 0, 15
+    Wg = ((lv - 8) * 2.0 ** -7).astype(np.float16)
+    out = _run_quant(B, Wg, U32, 4, 0, False, 32)
+    assert np.array_equal(O.unpack_codes(out["qweight"].view(np.uint32), 4, C), lv) and out["loss"] == 0.0
+
+
+def test_argument_errors_are_synchronous(B):
+    H = torch.zeros((48, 48), device="cuda")
+    X = torch.zeros((4, 48), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.GptqError) as e:
+        B.gptq_hessian_accumulate(H, X)          # C % 32 != 0
+    assert e.value.status == B.ERR_INVALID_ARG
+    W = torch.zeros((4, 64), dtype=torch.float16, device="cuda")
+    U = torch.eye(64, device="cuda")
+    for kw, st in ((dict(bits=5), B.ERR_UNSUPPORTED), (dict(bits=4, block=48), B.ERR_UNSUPPORTED),
+                   (dict(bits=4, group_size=48), B.ERR_INVALID_ARG), (dict(bits=4, block=0), B.ERR_INVALID_ARG)):
+        with pytest.raises(B.GptqError) as e:
+            B.gptq_quantize_layer(W, U, **kw)
+        assert e.value.status == st
+
+
+# ------------------------------------------------------------------ end to end, config 0
+def test_config0_end_to_end(B, D):
+    wl = WL.workload(0)
+    L = wl.layers[0]
+    grid = wl.grids[0]
+    bits_host = L.x_bits()
+    W16 = L.w()
+    ref = O.solve_layer(W16, bits_host, grid.bits, grid.group_size, grid.sym, wl.block, wl.damp)
+    X = D.fill_x(L)
+    W = D.fill_w(L)
+    H = torch.zeros((L.C, L.C), dtype=torch.float32, device="cuda")
+    B.gptq_hessian_accumulate(H, X)
+    U, info = B.gptq_prepare_hinv(H, wl.damp)
+    out = B.gptq_quantize_layer(W, U, grid.bits, grid.group_size, grid.sym, wl.block)
+    torch.cuda.synchronize()
+    assert info.tolist()[0] == 0 and out["dev_info"].tolist()[0] == 0
+    assert rel_fro(H.cpu().numpy(), ref["H"]) <= TOL_H_FRO
+    assert rel_fro(U.cpu().numpy(), ref["U"]) <= TOL_U_FRO
+    gpu = dict(qweight=out["qweight"].cpu().numpy(), scales=out["scales"].cpu().numpy(),
+               zeros=out["zeros"].cpu().numpy(), loss=out["loss"].item())
+    figs = check_quantize_outputs(gpu, ref, W16, grid.bits, L.C, ref["H"])
+    print("config0 end-to-end:", figs)
