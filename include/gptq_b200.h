@@ -54,6 +54,10 @@ typedef enum {
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* gptq_status_string(gptq_status_t status);
 
+/* Diagnostic (no counterpart in the paper): number of CUDA kernels this library has
+ * launched in the calling process so far.  Host-side counter; thread-safe. */
+uint64_t gptq_launch_count(void);
+
 /* ------------------------------------------------------------------ stage 1
  * H += 2 * sum_t x_t x_t^T                     (Section 2: H_F = 2 X_F X_F^T;
  *                                               Algorithm 1 caption: 2 X X^T)

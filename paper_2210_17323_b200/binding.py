@@ -17,12 +17,7 @@ LIB_PATH = os.path.join(_HERE, "lib", "libgptq_b200.so")
 BITS_TERNARY = -1
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NOT_PD, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE = range(8)
 
-EXPORTS = (
-    "gptq_status_string",
-    "gptq_hessian_workspace_bytes", "gptq_hessian_accumulate",
-    "gptq_prepare_hinv_workspace_bytes", "gptq_prepare_hinv",
-    "gptq_quantize_workspace_bytes", "gptq_quantize_layer",
-)
+from .binding_symbols import EXPORTS  # noqa: E402,F401
 
 
 class GptqError(RuntimeError):
@@ -40,6 +35,8 @@ def _load():
     c = ctypes
     lib.gptq_status_string.restype = c.c_char_p
     lib.gptq_status_string.argtypes = [c.c_int]
+    lib.gptq_launch_count.restype = c.c_uint64
+    lib.gptq_launch_count.argtypes = []
     lib.gptq_hessian_workspace_bytes.restype = c.c_size_t
     lib.gptq_hessian_workspace_bytes.argtypes = [c.c_int, c.c_int64]
     lib.gptq_hessian_accumulate.restype = c.c_int
@@ -62,6 +59,10 @@ _lib = _load()
 
 def status_string(status) -> str:
     return _lib.gptq_status_string(int(status)).decode()
+
+
+def gptq_launch_count() -> int:
+    return int(_lib.gptq_launch_count())
 
 
 def _stream_ptr(stream):

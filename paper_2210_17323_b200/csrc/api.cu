@@ -1,5 +1,14 @@
-// Status strings of the C ABI.
+// Status strings and diagnostics of the C ABI.
+#include <atomic>
+
 #include "common.cuh"
+
+namespace gptq {
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+}  // namespace gptq
+
+extern "C" uint64_t gptq_launch_count(void) { return gptq::g_launches.load(std::memory_order_relaxed); }
 
 extern "C" const char* gptq_status_string(gptq_status_t status) {
   switch (status) {

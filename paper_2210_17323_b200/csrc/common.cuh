@@ -36,7 +36,15 @@ inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintp
     if (_e != cudaSuccess) return GPTQ_ERR_CUDA;      \
   } while (0)
 
-#define GPTQ_LAUNCH_CHECK() GPTQ_CUDA_TRY(cudaGetLastError())
+// Number of kernels this library has launched in this process (diagnostic, see gptq_launch_count()).
+void count_launch(int n = 1);
+
+// Placed after every kernel launch: counts it and surfaces launch-configuration errors.
+#define GPTQ_LAUNCH_CHECK()                 \
+  do {                                      \
+    ::gptq::count_launch();                 \
+    GPTQ_CUDA_TRY(cudaGetLastError());      \
+  } while (0)
 
 // dev_info word layout: [0] status, [1] detail (pivot index, ...).  First error wins.
 __device__ __forceinline__ void report_error(int* dev_info, int status, int detail) {

@@ -83,6 +83,7 @@ inline cudaError_t launch_gemm_simt(int M, int N, int nz, AF a, BF b, RangeF ran
   if (M <= 0 || N <= 0) return cudaSuccess;
   dim3 grid((N + kSimtBN - 1) / kSimtBN, (M + kSimtBM - 1) / kSimtBM, nz);
   gemm_simt_kernel<<<grid, kSimtThreads, 0, stream>>>(M, N, a, b, range, epi);
+  count_launch();
   return cudaGetLastError();
 }
 

@@ -61,6 +61,7 @@ __global__ void mirror_upper_to_lower_kernel(float* __restrict__ H, int C) {
 cudaError_t launch_mirror_upper_to_lower(float* H, int C, cudaStream_t stream) {
   dim3 grid(C / 32, C / 32), block(32, 32);
   mirror_upper_to_lower_kernel<<<grid, block, 0, stream>>>(H, C);
+  count_launch();
   return cudaGetLastError();
 }
 
