@@ -67,10 +67,13 @@ uint64_t gptq_launch_count(void);
  *            triangles are valid on return.  No 1/m normalisation.
  *   X_bf16   [n_tokens x C] bfloat16, row-major, 16-byte aligned.
  *   n_tokens >= 0 (0 is a no-op).
- * Products of bf16 values are exact in fp32; accumulation is fp32. */
+ *   dev_info int[2] or NULL: [0] = GPTQ_OK or GPTQ_ERR_TIMEOUT (a bounded wait inside the
+ *            kernel ran out; H is then incomplete), [1] = which wait.
+ * Products of bf16 values are exact in fp32; accumulation is fp32: at most 8192 tokens in
+ * one tensor-core accumulator, chunks summed in fp32 in memory. */
 size_t gptq_hessian_workspace_bytes(int C, int64_t n_tokens);
 gptq_status_t gptq_hessian_accumulate(float* H, const void* X_bf16, int64_t n_tokens, int C,
-                                      void* ws, size_t ws_bytes, void* stream);
+                                      void* ws, size_t ws_bytes, int* dev_info, void* stream);
 
 /* ------------------------------------------------------------------ stage 2
  * lambda = damp * mean(diag H);  H~ = H + lambda I          (Section 3, Step 3)

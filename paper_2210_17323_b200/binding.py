@@ -40,7 +40,7 @@ def _load():
     lib.gptq_hessian_workspace_bytes.restype = c.c_size_t
     lib.gptq_hessian_workspace_bytes.argtypes = [c.c_int, c.c_int64]
     lib.gptq_hessian_accumulate.restype = c.c_int
-    lib.gptq_hessian_accumulate.argtypes = [c.c_void_p, c.c_void_p, c.c_int64, c.c_int, c.c_void_p, c.c_size_t, c.c_void_p]
+    lib.gptq_hessian_accumulate.argtypes = [c.c_void_p, c.c_void_p, c.c_int64, c.c_int, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
     lib.gptq_prepare_hinv_workspace_bytes.restype = c.c_size_t
     lib.gptq_prepare_hinv_workspace_bytes.argtypes = [c.c_int]
     lib.gptq_prepare_hinv.restype = c.c_int
@@ -97,14 +97,15 @@ def gptq_quantize_workspace_bytes(R, C, bits, group_size, block):
     return _lib.gptq_quantize_workspace_bytes(R, C, bits, group_size, block)
 
 
-def gptq_hessian_accumulate(H, X, n_tokens=None, ws=None, stream=None):
+def gptq_hessian_accumulate(H, X, n_tokens=None, ws=None, dev_info=None, stream=None):
     """H += 2 X^T X for token-major bf16 X (n_tokens x C).  H: C x C fp32, zeroed by the caller first."""
     _check(H, torch.float32, "H")
     _check(X, torch.bfloat16, "X")
     C = H.shape[0]
     n = X.shape[0] if n_tokens is None else int(n_tokens)
     ws = _ws(_lib.gptq_hessian_workspace_bytes(C, n), H.device, ws)
-    st = _lib.gptq_hessian_accumulate(H.data_ptr(), X.data_ptr(), n, C, ws.data_ptr(), ws.numel(), _stream_ptr(stream))
+    st = _lib.gptq_hessian_accumulate(H.data_ptr(), X.data_ptr(), n, C, ws.data_ptr(), ws.numel(),
+                                      None if dev_info is None else dev_info.data_ptr(), _stream_ptr(stream))
     if st != OK:
         raise GptqError(st, "gptq_hessian_accumulate")
     return H

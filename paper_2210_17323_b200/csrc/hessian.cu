@@ -90,7 +90,7 @@ extern "C" size_t gptq_hessian_workspace_bytes(int C, int64_t n_tokens) {
 }
 
 extern "C" gptq_status_t gptq_hessian_accumulate(float* H, const void* X_bf16, int64_t n_tokens, int C,
-                                                 void* ws, size_t ws_bytes, void* stream) {
+                                                 void* ws, size_t ws_bytes, int* dev_info, void* stream) {
   using namespace gptq;
   (void)ws; (void)ws_bytes;
   if (!H || C <= 0 || C % 32 != 0 || n_tokens < 0) return GPTQ_ERR_INVALID_ARG;
@@ -98,6 +98,7 @@ extern "C" gptq_status_t gptq_hessian_accumulate(float* H, const void* X_bf16, i
   if (!X_bf16 || !aligned_to(X_bf16, 16) || !aligned_to(H, 16)) return GPTQ_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(X_bf16);
-  if (hessian_umma_supported(C, n_tokens)) return hessian_umma(H, X, n_tokens, C, s);
+  if (dev_info) GPTQ_CUDA_TRY(cudaMemsetAsync(dev_info, 0, 2 * sizeof(int), s));
+  if (hessian_umma_supported(C, n_tokens)) return hessian_umma(H, X, n_tokens, C, dev_info, s);
   return hessian_simt(H, X, n_tokens, C, s);
 }
