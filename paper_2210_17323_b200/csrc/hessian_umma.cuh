@@ -6,6 +6,6 @@ namespace gptq {
 bool hessian_umma_supported(int C, int64_t n_tokens);
 gptq_status_t hessian_umma(float* H, const __nv_bfloat16* X, int64_t n_tokens, int C, int* dev_info,
                            cudaStream_t stream);
-int device_sm_count();
+
 cudaError_t launch_mirror_upper_to_lower(float* H, int C, cudaStream_t stream);
 }  // namespace gptq

@@ -10,11 +10,11 @@
 //   * Inside an outer block the paper's loop runs with the caller's block size B: the in-block
 //     kernel quantizes B columns with immediate error feedback, then the block's errors are
 //     pushed onto the remaining columns of the outer block.
-//   * Working weights of the current outer block are fp64; E is kept in fp32; update sums are
-//     fp32-accurate.  Each weight therefore meets one rounding at fp32 level (its update sum)
+//   * Working weights of the current outer block are fp64; E is kept in fp32 (as a tf32 hi/lo
+//     pair); update sums come from the tensor cores with fp32 accuracy (3xTF32).  Each weight therefore meets one rounding at fp32 level (its update sum)
 //     instead of one per preceding block.
 #include "common.cuh"
-#include "gemm_simt.cuh"
+#include "gemm_umma.cuh"
 
 namespace gptq {
 namespace {
@@ -99,7 +99,7 @@ struct InblockArgs {
   int group;        // group size (<= 0: one grid per row)
   int grid_inside;  // 1: grids of groups that start in this block are computed here (group <= B)
   float* scales; float* zeros; int G;
-  float* E; uint8_t* codes; double* loss; int* dev_info;
+  float* Ehi; float* Elo; uint8_t* codes; double* loss; int* dev_info;
 };
 
 // One thread per row.  The block's working weights sit in shared memory, column-major (thread-
@@ -192,10 +192,16 @@ __global__ void __launch_bounds__(RPB) inblock_kernel(InblockArgs a) {
       slab[c * LDS + t] = x;
     }
     if (live) {
-      float4* ep = reinterpret_cast<float4*>(a.E + (int64_t)row * a.C + a.i + j0);
+      float4* eh = reinterpret_cast<float4*>(a.Ehi + (int64_t)row * a.C + a.i + j0);
+      float4* el = reinterpret_cast<float4*>(a.Elo + (int64_t)row * a.C + a.i + j0);
 #pragma unroll
-      for (int k = 0; k < kSB / 4; ++k)
-        ep[k] = make_float4((float)err[4 * k], (float)err[4 * k + 1], (float)err[4 * k + 2], (float)err[4 * k + 3]);
+      for (int k = 0; k < kSB / 4; ++k) {
+        float h[4], l[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) tf32x3::split_tf32((float)err[4 * k + u], h[u], l[u]);
+        eh[k] = make_float4(h[0], h[1], h[2], h[3]);
+        el[k] = make_float4(l[0], l[1], l[2], l[3]);
+      }
       uint4* cp = reinterpret_cast<uint4*>(a.codes + (int64_t)row * a.C + a.i + j0);
       cp[0] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
       cp[1] = make_uint4(cw[4], cw[5], cw[6], cw[7]);
@@ -225,27 +231,54 @@ __global__ void pack_kernel(const uint8_t* __restrict__ codes, int R, int C, int
   qweight[idx] = word;
 }
 
-// ---- contraction functors -----------------------------------------------------------------------
-struct ElemE {  // A(m, k) = E[m][kofs + k]
-  static constexpr bool kInnerContig = true;
-  const float* E; int64_t C; int kofs;
-  __device__ __forceinline__ float operator()(int m, int k) const { return E[(int64_t)m * C + kofs + k]; }
+// ---- U panel -> transposed tf32 hi / lo pair ------------------------------------------------------
+// Pt[c][r] = U[r][i2 + c] for r < rows, c < nb2 (row stride ldp): the right factor of the lazy
+// updates, transposed so the contraction index is contiguous, split so that hi + lo ~ U to 2^-22.
+__global__ void split_panel_t_kernel(const float* __restrict__ U, int C, int i2, int rows,
+                                     float* __restrict__ Phi, float* __restrict__ Plo, int64_t ldp) {
+  __shared__ float t[32][33];
+  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+  t[threadIdx.y][threadIdx.x] = U[(int64_t)(r0 + threadIdx.y) * C + i2 + c0 + threadIdx.x];
+  __syncthreads();
+  float h, l;
+  tf32x3::split_tf32(t[threadIdx.x][threadIdx.y], h, l);
+  const int64_t o = (int64_t)(c0 + threadIdx.y) * ldp + r0 + threadIdx.x;
+  Phi[o] = h; Plo[o] = l;
+  (void)rows;
+}
+
+// ---- contraction epilogues (one thread: one row, 32 consecutive columns) ------------------------
+struct FullK {
+  int K;
+  __device__ __forceinline__ bool operator()(int, int, int& k0, int& k1) const { k0 = 0; k1 = K; return K > 0; }
 };
-struct ElemU {  // B(k, n) = U[kofs + k][nofs + n]
-  static constexpr bool kInnerContig = true;
-  const float* U; int64_t C; int kofs, nofs;
-  __device__ __forceinline__ float operator()(int k, int n) const { return U[(int64_t)(kofs + k) * C + nofs + n]; }
-};
-struct EpiInitWblk {  // Wblk[m][n] = W16[m][i2 + n] - acc
+struct EpiInitWblk {  // Wblk[row][col..col+32) = W16[row][i2 + col ..] - acc
   const __half* W; int64_t C; int i2; double* Wblk; int64_t ldw;
-  __device__ __forceinline__ void operator()(int m, int n, float acc) const {
-    Wblk[(int64_t)m * ldw + n] = (double)__half2float(W[(int64_t)m * C + i2 + n]) - (double)acc;
+  __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
+    const uint4* wp = reinterpret_cast<const uint4*>(W + (int64_t)row * C + i2 + col0);
+    double2* out = reinterpret_cast<double2*>(Wblk + (int64_t)row * ldw + col0);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      uint4 u = wp[k];
+      const __half2* h = reinterpret_cast<const __half2*>(&u);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float2 f = __half22float2(h[j]);
+        out[k * 4 + j] = make_double2((double)f.x - (double)v[k * 8 + 2 * j], (double)f.y - (double)v[k * 8 + 2 * j + 1]);
+      }
+    }
   }
 };
-struct EpiSubWblk {  // Wblk[m][nofs + n] -= acc
+struct EpiSubWblk {  // Wblk[row][nofs + col ..) -= acc
   double* Wblk; int64_t ldw; int nofs;
-  __device__ __forceinline__ void operator()(int m, int n, float acc) const {
-    Wblk[(int64_t)m * ldw + nofs + n] -= (double)acc;
+  __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
+    double2* p = reinterpret_cast<double2*>(Wblk + (int64_t)row * ldw + nofs + col0);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      double2 x = p[j];
+      x.x -= (double)v[2 * j]; x.y -= (double)v[2 * j + 1];
+      p[j] = x;
+    }
   }
 };
 
@@ -267,8 +300,11 @@ extern "C" size_t gptq_quantize_workspace_bytes(int R, int C, int bits, int grou
   if (R <= 0 || C <= 0 || block <= 0 || !bits_ok(bits)) return 0;
   WsCarver w(nullptr);
   w.take<double>((size_t)R * outer_block(C, group_size, block));  // working weights of the outer block
-  w.take<float>((size_t)R * C);                                   // E, all columns
+  w.take<float>((size_t)R * C);                                   // E (tf32 high parts), all columns
+  w.take<float>((size_t)R * C);                                   // E (tf32 remainders)
   w.take<uint8_t>((size_t)R * C);                                 // unpacked codes
+  w.take<float>((size_t)C * outer_block(C, group_size, block));   // transposed panel of U, high parts
+  w.take<float>((size_t)C * outer_block(C, group_size, block));   // panel of U, remainders
   return w.off;
 }
 
@@ -297,8 +333,11 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   const int G = g > 0 ? C / g : 1;
   WsCarver w(ws);
   double* Wblk = w.take<double>((size_t)R * B2);
-  float* E = w.take<float>((size_t)R * C);
+  float* Ehi = w.take<float>((size_t)R * C);
+  float* Elo = w.take<float>((size_t)R * C);
   uint8_t* codes = w.take<uint8_t>((size_t)R * C);
+  float* Phi = w.take<float>((size_t)C * B2);
+  float* Plo = w.take<float>((size_t)C * B2);
   const int64_t ldw = B2;
   GridSpec gs{bits == GPTQ_BITS_TERNARY ? 2 : (1 << bits) - 1, (sym != 0 || bits == GPTQ_BITS_TERNARY) ? 1 : 0};
 
@@ -317,14 +356,20 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
 
   for (int i2 = 0; i2 < C; i2 += B2) {
     const int nb2 = (C - i2 < B2) ? C - i2 : B2;
+    {  // transposed tf32 hi/lo pair of U[0 : i2 + nb2, i2 : i2 + nb2] for the contractions of this outer block
+      dim3 grid(nb2 / 32, (i2 + nb2) / 32), blk(32, 32);
+      split_panel_t_kernel<<<grid, blk, 0, s>>>(U, C, i2, i2 + nb2, Phi, Plo, (int64_t)C);
+      GPTQ_LAUNCH_CHECK();
+    }
     // working weights of the outer block: original weights minus all updates from columns < i2
     if (i2 == 0) {
       int64_t total = (int64_t)R * nb2;
       wblk_from_w16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(W, R, C, nb2, Wblk, ldw);
       GPTQ_LAUNCH_CHECK();
     } else {
-      GPTQ_CUDA_TRY(launch_gemm_simt(R, nb2, 1, ElemE{E, C, 0}, ElemU{U, C, 0, i2}, FullRange{i2},
-                                     EpiInitWblk{W, C, i2, Wblk, ldw}, s));
+      tf32x3::Operand A{Ehi, Elo, R, i2, C}, Bop{Phi, Plo, nb2, i2, C};
+      gptq_status_t st = tf32x3::launch(A, Bop, R, nb2, FullK{i2}, EpiInitWblk{W, C, i2, Wblk, ldw}, dev_info, s);
+      if (st != GPTQ_OK) return st;
     }
     for (int i = i2; i < i2 + nb2; i += block) {
       const int B = (i2 + nb2 - i < block) ? i2 + nb2 - i : block;
@@ -333,15 +378,18 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
         GPTQ_LAUNCH_CHECK();
       }
       InblockArgs a{Wblk, ldw, i - i2, U, C, i, B, R, gs, g, (g > 0 && g <= B) ? 1 : 0,
-                    scales, zeros, G, E, codes, loss, dev_info};
+                    scales, zeros, G, Ehi, Elo, codes, loss, dev_info};
       if (rpb == 64) inblock_kernel<64><<<ceil_div(R, 64), 64, inblock_smem(B), s>>>(a);
       else inblock_kernel<128><<<ceil_div(R, 128), 128, inblock_smem(B), s>>>(a);
       GPTQ_LAUNCH_CHECK();
       // push this block's errors onto the remaining columns of the outer block
       const int rest = i2 + nb2 - (i + B);
-      if (rest > 0)
-        GPTQ_CUDA_TRY(launch_gemm_simt(R, rest, 1, ElemE{E, C, i}, ElemU{U, C, i, i + B}, FullRange{B},
-                                       EpiSubWblk{Wblk, ldw, i + B - i2}, s));
+      if (rest > 0) {
+        const int64_t po = (int64_t)(i + B - i2) * C + i;     // U[i][i + B] inside the transposed panel
+        tf32x3::Operand A{Ehi + i, Elo + i, R, B, C}, Bop{Phi + po, Plo + po, rest, B, C};
+        gptq_status_t st = tf32x3::launch(A, Bop, R, rest, FullK{B}, EpiSubWblk{Wblk, ldw, i + B - i2}, dev_info, s);
+        if (st != GPTQ_OK) return st;
+      }
     }
   }
   {

@@ -154,6 +154,8 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 
 }  // namespace umma
 
+int device_sm_count();
+
 // Host: encodes a 2-D tiled tensor map (row-major matrix, `inner` contiguous elements per row)
 // with 128-byte swizzle.  The driver entry point is looked up at run time, so the library does
 // not link against libcuda.
