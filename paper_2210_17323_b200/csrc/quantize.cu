@@ -82,13 +82,13 @@ __global__ void groupgrid_kernel(const double* __restrict__ Wblk, int64_t ldw, i
   if (lane == 0) find_params(mn, mx, gs, scales[(int64_t)row * G + gi], zeros[(int64_t)row * G + gi]);
 }
 
-// ---- first outer block: working weights are the original weights -------------------------------
-__global__ void wblk_from_w16_kernel(const __half* __restrict__ W, int R, int C, int nb,
+// ---- working weights of an outer block start as the original weights ---------------------------
+__global__ void wblk_from_w16_kernel(const __half* __restrict__ W, int R, int C, int i2, int nb,
                                      double* __restrict__ Wblk, int64_t ldw) {
   int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)R * nb) return;
   int r = (int)(idx / nb), c = (int)(idx % nb);
-  Wblk[(int64_t)r * ldw + c] = (double)__half2float(W[(int64_t)r * C + c]);
+  Wblk[(int64_t)r * ldw + c] = (double)__half2float(W[(int64_t)r * C + i2 + c]);
 }
 
 // ---- the in-block loop (Algorithm 1, inner FOR) -------------------------------------------------
@@ -247,38 +247,17 @@ __global__ void split_panel_t_kernel(const float* __restrict__ U, int C, int i2,
   (void)rows;
 }
 
-// ---- contraction epilogues (one thread: one row, 32 consecutive columns) ------------------------
-struct FullK {
-  int K;
-  __device__ __forceinline__ bool operator()(int, int, int& k0, int& k1) const { k0 = 0; k1 = K; return K > 0; }
-};
-struct EpiInitWblk {  // Wblk[row][col..col+32) = W16[row][i2 + col ..] - acc
-  const __half* W; int64_t C; int i2; double* Wblk; int64_t ldw;
+// ---- contraction epilogue (one thread: one row, 32 consecutive columns of a partial sum) --------
+// Wblk[row][nofs + col ..) -= partial, as fp64 reductions: partial sums of one tile may come from
+// several CTAs (one per super-chunk of the contraction).
+struct EpiSubWblk {
+  double* Wblk; int64_t ldw; int nofs; int R, N;
   __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
-    const uint4* wp = reinterpret_cast<const uint4*>(W + (int64_t)row * C + i2 + col0);
-    double2* out = reinterpret_cast<double2*>(Wblk + (int64_t)row * ldw + col0);
+    if (row >= R || col0 >= N) return;
+    double* p = Wblk + (int64_t)row * ldw + nofs + col0;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      uint4 u = wp[k];
-      const __half2* h = reinterpret_cast<const __half2*>(&u);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        float2 f = __half22float2(h[j]);
-        out[k * 4 + j] = make_double2((double)f.x - (double)v[k * 8 + 2 * j], (double)f.y - (double)v[k * 8 + 2 * j + 1]);
-      }
-    }
-  }
-};
-struct EpiSubWblk {  // Wblk[row][nofs + col ..) -= acc
-  double* Wblk; int64_t ldw; int nofs;
-  __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
-    double2* p = reinterpret_cast<double2*>(Wblk + (int64_t)row * ldw + nofs + col0);
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      double2 x = p[j];
-      x.x -= (double)v[2 * j]; x.y -= (double)v[2 * j + 1];
-      p[j] = x;
-    }
+    for (int j = 0; j < 32; ++j)
+      asm volatile("red.global.add.f64 [%0], %1;" ::"l"(p + j), "d"(-(double)v[j]) : "memory");
   }
 };
 
@@ -362,13 +341,14 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
       GPTQ_LAUNCH_CHECK();
     }
     // working weights of the outer block: original weights minus all updates from columns < i2
-    if (i2 == 0) {
+    {
       int64_t total = (int64_t)R * nb2;
-      wblk_from_w16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(W, R, C, nb2, Wblk, ldw);
+      wblk_from_w16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(W, R, C, i2, nb2, Wblk, ldw);
       GPTQ_LAUNCH_CHECK();
-    } else {
+    }
+    if (i2 > 0) {
       tf32x3::Operand A{Ehi, Elo, R, i2, C}, Bop{Phi, Plo, nb2, i2, C};
-      gptq_status_t st = tf32x3::launch(A, Bop, R, nb2, FullK{i2}, EpiInitWblk{W, C, i2, Wblk, ldw}, dev_info, s);
+      gptq_status_t st = tf32x3::launch<false, false>(A, Bop, R, nb2, EpiSubWblk{Wblk, ldw, 0, R, nb2}, dev_info, s);
       if (st != GPTQ_OK) return st;
     }
     for (int i = i2; i < i2 + nb2; i += block) {
@@ -387,7 +367,7 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
       if (rest > 0) {
         const int64_t po = (int64_t)(i + B - i2) * C + i;     // U[i][i + B] inside the transposed panel
         tf32x3::Operand A{Ehi + i, Elo + i, R, B, C}, Bop{Phi + po, Plo + po, rest, B, C};
-        gptq_status_t st = tf32x3::launch(A, Bop, R, rest, FullK{B}, EpiSubWblk{Wblk, ldw, i + B - i2}, dev_info, s);
+        gptq_status_t st = tf32x3::launch<false, false>(A, Bop, R, rest, EpiSubWblk{Wblk, ldw, i + B - i2, R, rest}, dev_info, s);
         if (st != GPTQ_OK) return st;
       }
     }
