@@ -5,10 +5,14 @@
 // and U^T U = U~^-T U~^-1 = H~^-1, so by uniqueness it is the matrix Algorithm 1 asks for, at
 // 2 C^3 / 3 flops and without ever forming H~^-1.
 //
-// Blocked with 128-wide panels: diagonal blocks are factored and inverted in fp64 in shared
-// memory by one CTA; panel and trailing products are fp32 tile GEMMs.
+// Two-level blocking.  128 x 128 diagonal blocks are factored and inverted in fp64 in shared
+// memory by one CTA; products inside a 1024-column outer panel are fp32 CUDA-core tile GEMMs;
+// everything that reaches across outer panels (almost all of the flops for large C) is a
+// left-looking fp32-accurate tensor-core contraction (3xTF32, tcgen05) over tf32 hi / lo copies
+// of the factor that are written as each panel is finalised.
 #include "common.cuh"
 #include "gemm_simt.cuh"
+#include "gemm_umma.cuh"
 
 namespace gptq {
 namespace {
@@ -106,11 +110,13 @@ __global__ void store_diag_block_kernel(float* __restrict__ U, int C, int k0, in
   }
 }
 
-struct UpperTiles {
-  int K;
+// Tiles of the M x N product that reach the part on or above the diagonal, the output columns
+// being shifted by nofs against the rows (output element (m, nofs + n)).
+struct UpperTilesOfs {
+  int K, nofs;
   __device__ __forceinline__ bool operator()(int m0, int n0, int, int, int& k0, int& k1) const {
     k0 = 0; k1 = K;
-    return m0 <= n0 + kSimtBN - 1;
+    return m0 <= nofs + n0 + kSimtBN - 1;
   }
 };
 // K starts at the tile's first row: the left factor is upper triangular.
@@ -129,12 +135,128 @@ struct StoreNegF32 {
   float* p; int64_t ld;
   __device__ __forceinline__ void operator()(int m, int n, float acc) const { p[(int64_t)m * ld + n] = -acc; }
 };
-struct SubUpperF32 {
-  float* p; int64_t ld;
+struct SubUpperOfsF32 {   // p[m][nofs + n] -= acc where that element is on or above the diagonal
+  float* p; int64_t ld; int nofs;
   __device__ __forceinline__ void operator()(int m, int n, float acc) const {
-    if (m <= n) p[(int64_t)m * ld + n] -= acc;
+    if (m <= nofs + n) p[(int64_t)m * ld + nofs + n] -= acc;
   }
 };
+
+// ---- tensor-core (3xTF32) epilogues: one thread, one row, 32 consecutive columns of a partial sum
+// dst[row][cofs + col] -= partial for elements on or above the diagonal (fp32 reductions).
+struct EpiSubUpperRed {
+  float* p; int64_t ld; int cofs; int M, N;
+  __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
+    if (row >= M || col0 >= N) return;
+    float* d = p + (int64_t)row * ld + cofs + col0;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      const int c = cofs + col0 + 4 * g;            // global column of the group's first element
+      if (c >= row) umma::red_add_v4(d + 4 * g, -v[4 * g], -v[4 * g + 1], -v[4 * g + 2], -v[4 * g + 3]);
+      else if (c + 3 >= row) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) if (c + u >= row) atomicAdd(d + 4 * g + u, -v[4 * g + u]);
+      }
+    }
+  }
+};
+// dst[row][col] -= partial over the whole rectangle (fp32 reductions).
+struct EpiSubRed {
+  float* p; int64_t ld; int M, N;
+  __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
+    if (row >= M || col0 >= N) return;
+    float* d = p + (int64_t)row * ld + col0;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) umma::red_add_v4(d + 4 * g, -v[4 * g], -v[4 * g + 1], -v[4 * g + 2], -v[4 * g + 3]);
+  }
+};
+// Stores the result as a tf32 hi / lo pair.  Only valid when the contraction is a single
+// super-chunk (K <= tf32x3::kSuperK), so that the partial sum IS the result.
+struct EpiStoreSplit {
+  float* hi; float* lo; int64_t ld; int M, N;
+  __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
+    if (row >= M || col0 >= N) return;
+    float4* h = reinterpret_cast<float4*>(hi + (int64_t)row * ld + col0);
+    float4* l = reinterpret_cast<float4*>(lo + (int64_t)row * ld + col0);
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      float4 a, b;
+      tf32x3::split_tf32(v[4 * g], a.x, b.x); tf32x3::split_tf32(v[4 * g + 1], a.y, b.y);
+      tf32x3::split_tf32(v[4 * g + 2], a.z, b.z); tf32x3::split_tf32(v[4 * g + 3], a.w, b.w);
+      h[g] = a; l[g] = b;
+    }
+  }
+};
+
+// F{hi,lo}[r][c0 + c] = split(U[r][c0 + c]) for r < rows, c < w.
+__global__ void split_block_kernel(const float* __restrict__ U, int C, int c0, int w, int rows,
+                                   float* __restrict__ Fhi, float* __restrict__ Flo) {
+  const int q = w / 4;
+  int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)rows * q) return;
+  const int r = (int)(idx / q), c = (int)(idx % q) * 4;
+  const int64_t o = (int64_t)r * C + c0 + c;
+  float4 v = *reinterpret_cast<const float4*>(U + o), h, l;
+  tf32x3::split_tf32(v.x, h.x, l.x); tf32x3::split_tf32(v.y, h.y, l.y);
+  tf32x3::split_tf32(v.z, h.z, l.z); tf32x3::split_tf32(v.w, h.w, l.w);
+  *reinterpret_cast<float4*>(Fhi + o) = h;
+  *reinterpret_cast<float4*>(Flo + o) = l;
+}
+// VT{hi,lo}[c][r] = split(U[j0 + r][j0 + c]) for r, c < w  (transpose of a diagonal block, ld = ldv).
+__global__ void split_diag_t_kernel(const float* __restrict__ U, int C, int j0,
+                                    float* __restrict__ Vhi, float* __restrict__ Vlo, int ldv) {
+  __shared__ float t[32][33];
+  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+  t[threadIdx.y][threadIdx.x] = U[(int64_t)(j0 + r0 + threadIdx.y) * C + j0 + c0 + threadIdx.x];
+  __syncthreads();
+  float h, l;
+  tf32x3::split_tf32(t[threadIdx.x][threadIdx.y], h, l);
+  const int64_t o = (int64_t)(c0 + threadIdx.y) * ldv + r0 + threadIdx.x;
+  Vhi[o] = h; Vlo[o] = l;
+}
+
+constexpr int kNB2 = 1024;   // outer panel width: contractions over everything outside it run on the tensor cores
+
+struct HinvWs {
+  double* lam; float* Dinv; float* T; float* Fhi; float* Flo; float* VThi; float* VTlo; float* TThi; float* TTlo;
+  size_t bytes;
+};
+HinvWs carve_hinv(void* ws, int C) {
+  WsCarver w(ws);
+  HinvWs o;
+  o.lam = w.take<double>(1);
+  o.Dinv = w.take<float>((size_t)ceil_div(C, kNB) * kNB * kNB);   // inverses of the 128 x 128 diagonal blocks
+  o.T = w.take<float>((size_t)C * kNB);                           // panel temporary (CUDA-core path)
+  const bool outer = C > kNB2;
+  o.Fhi = w.take<float>(outer ? (size_t)C * C : 0);               // tf32 hi / lo of the factor as it is finalised
+  o.Flo = w.take<float>(outer ? (size_t)C * C : 0);
+  o.VThi = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);        // transposed inverse of an outer diagonal block
+  o.VTlo = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);
+  o.TThi = w.take<float>(outer ? (size_t)kNB2 * C : 0);           // (U~[0:j0, J] V_JJ)^T
+  o.TTlo = w.take<float>(outer ? (size_t)kNB2 * C : 0);
+  o.bytes = w.off;
+  return o;
+}
+
+// In-place inversion of the upper-triangular w x w block at D (leading dimension C) whose 128 x 128
+// diagonal blocks already have their inverses in Dinv (first block at Dinv).  CUDA-core path.
+gptq_status_t invert_upper_block(float* D, int C, int w, float* Dinv, float* T, cudaStream_t s) {
+  for (int k0 = 0; k0 < w; k0 += kNB) {
+    const int nb = (w - k0 < kNB) ? w - k0 : kNB;
+    float* Dk = Dinv + (size_t)(k0 / kNB) * kNB * kNB;
+    if (k0 > 0) {
+      // T = U~[0:k0, blk] * V_kk
+      GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, 1, RowMajorF32{D + k0, C}, RowMajorF32{Dk, kNB},
+                                     FullRange{nb}, StoreF32{T, kNB}, s));
+      // U[0:k0, blk] = -U[0:k0, 0:k0] * T   (left factor already inverted, upper triangular)
+      GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, 1, RowMajorF32{D, C}, RowMajorF32{T, kNB},
+                                     UpperLeftFactorRange{k0}, StoreNegF32{D + k0, C}, s));
+    }
+    store_diag_block_kernel<<<8, 256, 0, s>>>(D, C, k0, nb, Dk);
+    GPTQ_LAUNCH_CHECK();
+  }
+  return GPTQ_OK;
+}
 
 }  // namespace
 }  // namespace gptq
@@ -142,11 +264,7 @@ struct SubUpperF32 {
 extern "C" size_t gptq_prepare_hinv_workspace_bytes(int C) {
   using namespace gptq;
   if (C <= 0) return 0;
-  WsCarver w(nullptr);
-  w.take<double>(1);                                        // lambda
-  w.take<float>((size_t)ceil_div(C, kNB) * kNB * kNB);      // inverses of the diagonal blocks
-  w.take<float>((size_t)C * kNB);                           // panel temporary
-  return w.off;
+  return carve_hinv(nullptr, C).bytes;
 }
 
 extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, float* U,
@@ -156,50 +274,86 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
   if (!aligned_to(H, 16) || !aligned_to(U, 16)) return GPTQ_ERR_INVALID_ARG;
   if (!ws || !aligned_to(ws, kAlign) || ws_bytes < gptq_prepare_hinv_workspace_bytes(C)) return GPTQ_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  WsCarver w(ws);
-  const int nbk = ceil_div(C, kNB);
-  double* lam = w.take<double>(1);
-  float* Dinv = w.take<float>((size_t)nbk * kNB * kNB);
-  float* T = w.take<float>((size_t)C * kNB);
+  HinvWs w = carve_hinv(ws, C);
+  gptq_status_t st;
 
   const int diag_smem = (kNB * (kNB + 1) + kNB) * (int)sizeof(double);
   GPTQ_CUDA_TRY(cudaFuncSetAttribute(rchol_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, diag_smem));
   GPTQ_CUDA_TRY(cudaMemsetAsync(dev_info, 0, 2 * sizeof(int), s));
-  lambda_kernel<<<1, 1024, 0, s>>>(H, C, damp, lam);
+  lambda_kernel<<<1, 1024, 0, s>>>(H, C, damp, w.lam);
   GPTQ_LAUNCH_CHECK();
   {
     int64_t total = (int64_t)C * C / 4;
-    init_upper_damped_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(H, U, C, lam);
+    init_upper_damped_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(H, U, C, w.lam);
     GPTQ_LAUNCH_CHECK();
   }
-  // Phase 1: backwards blocked Cholesky, H~ = U~ U~^T, in place in U's upper triangle.
-  for (int kb = nbk - 1; kb >= 0; --kb) {
-    const int k0 = kb * kNB, nb = (C - k0 < kNB) ? C - k0 : kNB;
-    float* Dk = Dinv + (size_t)kb * kNB * kNB;
-    rchol_diag_kernel<<<1, 256, diag_smem, s>>>(U, C, k0, nb, Dk, dev_info);
-    GPTQ_LAUNCH_CHECK();
-    if (k0 == 0) break;
-    // panel: U~[0:k0, blk] = A[0:k0, blk] * T_kk^-T      (out[m][n] = sum_k A[m][k0+k] V[n][k])
-    GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, 1, RowMajorF32{U + k0, C}, RowMajorF32T{Dk, kNB},
-                                   FullRange{nb}, StoreF32{U + k0, C}, s));
-    // trailing: A[0:k0, 0:k0] -= P P^T on upper tiles     (P = U~[0:k0, blk])
-    GPTQ_CUDA_TRY(launch_gemm_simt(k0, k0, 1, RowMajorF32{U + k0, C}, RowMajorF32T{U + k0, C},
-                                   UpperTiles{nb}, SubUpperF32{U, C}, s));
-  }
-  // Phase 2: U = U~^-1, column block by column block, in place.
-  for (int kb = 0; kb < nbk; ++kb) {
-    const int k0 = kb * kNB, nb = (C - k0 < kNB) ? C - k0 : kNB;
-    float* Dk = Dinv + (size_t)kb * kNB * kNB;
-    if (k0 > 0) {
-      // T = U~[0:k0, blk] * V_kk
-      GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, 1, RowMajorF32{U + k0, C}, RowMajorF32{Dk, kNB},
-                                     FullRange{nb}, StoreF32{T, kNB}, s));
-      // U[0:k0, blk] = -U[0:k0, 0:k0] * T   (left factor already inverted, upper triangular)
-      GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, 1, RowMajorF32{U, C}, RowMajorF32{T, kNB},
-                                     UpperLeftFactorRange{k0}, StoreNegF32{U + k0, C}, s));
+  const bool outer = C > kNB2;
+  const int n_outer = ceil_div(C, kNB2);
+
+  // Phase 1: backwards blocked Cholesky, H~ = U~ U~^T, in place in U's upper triangle.  Outer panels
+  // of kNB2 columns are brought up to date in one contraction over all later columns (left-looking),
+  // then factored with 128-wide steps whose updates stay inside the panel.
+  for (int J = n_outer - 1; J >= 0; --J) {
+    const int j0 = J * kNB2, wj = (C - j0 < kNB2) ? C - j0 : kNB2, rows_p = j0 + wj;
+    if (rows_p < C) {
+      // A[0:rows_p, J] -= U~[0:rows_p, later] * U~[J rows, later]^T   (upper part)
+      const int K = C - rows_p;
+      tf32x3::Operand A{w.Fhi + rows_p, w.Flo + rows_p, rows_p, K, C};
+      tf32x3::Operand B{w.Fhi + (int64_t)j0 * C + rows_p, w.Flo + (int64_t)j0 * C + rows_p, wj, K, C};
+      st = tf32x3::launch<false, false>(A, B, rows_p, wj, EpiSubUpperRed{U, C, j0, rows_p, wj}, dev_info, s);
+      if (st != GPTQ_OK) return st;
     }
-    store_diag_block_kernel<<<8, 256, 0, s>>>(U, C, k0, nb, Dk);
-    GPTQ_LAUNCH_CHECK();
+    for (int k0 = j0 + (wj - 1) / kNB * kNB; k0 >= j0; k0 -= kNB) {
+      const int nb = (rows_p - k0 < kNB) ? rows_p - k0 : kNB;
+      float* Dk = w.Dinv + (size_t)(k0 / kNB) * kNB * kNB;
+      rchol_diag_kernel<<<1, 256, diag_smem, s>>>(U, C, k0, nb, Dk, dev_info);
+      GPTQ_LAUNCH_CHECK();
+      if (k0 == 0) break;
+      // panel: U~[0:k0, blk] = A[0:k0, blk] * T_kk^-T      (out[m][n] = sum_k A[m][k0+k] V[n][k])
+      GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, 1, RowMajorF32{U + k0, C}, RowMajorF32T{Dk, kNB},
+                                     FullRange{nb}, StoreF32{U + k0, C}, s));
+      // trailing, inside the outer panel: A[0:k0, j0:k0] -= P P[j0:k0]^T on upper tiles  (P = U~[0:k0, blk])
+      if (k0 > j0)
+        GPTQ_CUDA_TRY(launch_gemm_simt(k0, k0 - j0, 1, RowMajorF32{U + k0, C}, RowMajorF32T{U + (int64_t)j0 * C + k0, C},
+                                       UpperTilesOfs{nb, j0}, SubUpperOfsF32{U, C, j0}, s));
+    }
+    if (outer && J > 0) {
+      int64_t total = (int64_t)rows_p * (wj / 4);
+      split_block_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(U, C, j0, wj, rows_p, w.Fhi, w.Flo);
+      GPTQ_LAUNCH_CHECK();
+    }
+  }
+  // Phase 2: U = U~^-1, outer panel by outer panel, in place.
+  for (int J = 0; J < n_outer; ++J) {
+    const int j0 = J * kNB2, wj = (C - j0 < kNB2) ? C - j0 : kNB2, rows_p = j0 + wj;
+    // (a) diagonal block: V_JJ = U~_JJ^-1
+    st = invert_upper_block(U + (int64_t)j0 * C + j0, C, wj, w.Dinv + (size_t)(j0 / kNB) * kNB * kNB, w.T, s);
+    if (st != GPTQ_OK) return st;
+    if (j0 > 0) {
+      // (b) rows above it: U[0:j0, J] = -U[0:j0, 0:j0] * (U~[0:j0, J] * V_JJ)
+      dim3 grid(wj / 32, wj / 32), blk(32, 32);
+      split_diag_t_kernel<<<grid, blk, 0, s>>>(U, C, j0, w.VThi, w.VTlo, kNB2);
+      GPTQ_LAUNCH_CHECK();
+      // TT = V_JJ^T * U~[0:j0, J]^T   (wj x j0), written as a hi / lo pair (single super-chunk: K = wj)
+      {
+        tf32x3::Operand A{w.VThi, w.VTlo, wj, wj, kNB2};
+        tf32x3::Operand B{w.Fhi + j0, w.Flo + j0, j0, wj, C};
+        st = tf32x3::launch<false, false>(A, B, wj, j0, EpiStoreSplit{w.TThi, w.TTlo, C, wj, j0}, dev_info, s);
+        if (st != GPTQ_OK) return st;
+      }
+      GPTQ_CUDA_TRY(cudaMemset2DAsync(U + j0, (size_t)C * 4, 0, (size_t)wj * 4, j0, s));
+      {
+        tf32x3::Operand A{w.Fhi, w.Flo, j0, j0, C};
+        tf32x3::Operand B{w.TThi, w.TTlo, wj, j0, C};
+        st = tf32x3::launch<true, false>(A, B, j0, wj, EpiSubRed{U + j0, C, j0, wj}, dev_info, s);
+        if (st != GPTQ_OK) return st;
+      }
+    }
+    if (outer && J + 1 < n_outer) {
+      int64_t total = (int64_t)rows_p * (wj / 4);
+      split_block_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(U, C, j0, wj, rows_p, w.Fhi, w.Flo);
+      GPTQ_LAUNCH_CHECK();
+    }
   }
   return GPTQ_OK;
 }

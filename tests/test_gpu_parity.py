@@ -78,9 +78,9 @@ def test_hessian_integer_inputs_bit_exact_and_chunked(B):
 
 
 # ------------------------------------------------------------------ stage 2
-@pytest.mark.parametrize("C", [32, 96, 160, 768])
+@pytest.mark.parametrize("C", [32, 96, 160, 768, 1056, 2304])
 def test_prepare_hinv_matches_oracle(B, C):
-    L = _layer(8, C, 4 * C + 100)
+    L = _layer(8, C, 2 * C + 100)
     H64 = O.hessian_accumulate(np.zeros((C, C)), L.x_bits())
     H32 = H64.astype(np.float32)
     U, info = B.gptq_prepare_hinv(torch.from_numpy(H32).cuda(), 0.01)
