@@ -52,54 +52,93 @@ __global__ void init_upper_damped_kernel(const float* __restrict__ H, float* __r
 
 // One CTA: factor the nb x nb diagonal block at (k0, k0) as A = T T^T with T upper (backwards
 // Cholesky), store T in place (fp32) and its inverse V = T^-1 (upper) to Dinv (fp32, ld = kNB).
+// Both run in fp64, fused in one sweep j = nb-1 .. 0: step j finishes column j of T and row j of
+// V (solving T V = I from the bottom row up), then applies two rank-1 updates,
+//   A[i][c] -= T[i][j] T[c][j]   (i <= c < j)      and      B[c][i] -= T[c][j] V[j][i]   (c < j <= i),
+// where B is the running right-hand side of the solve.  The whole 128 x 128 working matrix M lives
+// in REGISTERS (32 doubles per thread, element (i, c) with i = ty + 16 a, c = tx + 32 b): its upper
+// triangle holds A / T, its strictly lower triangle holds B / V transposed (M[i][c] = B[c][i]).
+// Per step only column j (scaled) passes through shared memory.
 // A non-positive pivot is reported and replaced by 1 so everything downstream stays finite.
-__global__ void __launch_bounds__(256)
+constexpr int kDiagThreads = 512;
+__global__ void __launch_bounds__(kDiagThreads)
 rchol_diag_kernel(float* __restrict__ U, int C, int k0, int nb, float* __restrict__ Dinv, int* dev_info) {
-  extern __shared__ double sm[];
-  const int LD = kNB + 1;
-  double* S = sm;               // [nb][LD]: T in the upper triangle; V^T (strictly upper part of V) in the lower
-  double* vd = sm + kNB * LD;   // [nb]: diagonal of V
-  const int tid = threadIdx.x, nt = blockDim.x;
-  for (int e = tid; e < nb * nb; e += nt) {
-    int i = e / nb, j = e % nb;
-    S[i * LD + j] = j >= i ? (double)U[(int64_t)(k0 + i) * C + k0 + j] : 0.0;
-  }
+  __shared__ double colv[kNB];   // step j: colv[i] = T[i][j] for i < j, V[j][i] for i > j
+  __shared__ double pd[kNB];     // diagonal of T
+  __shared__ double vd[kNB];     // diagonal of V
+  __shared__ double dsh;         // pivot candidate of the current step
+  const int tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
+  double M[8][4];
+#pragma unroll
+  for (int a = 0; a < 8; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int i = ty + 16 * a, c = tx + 32 * b;
+      M[a][b] = (i < nb && c < nb && c >= i) ? (double)U[(int64_t)(k0 + i) * C + k0 + c] : 0.0;
+      if (i == nb - 1 && c == nb - 1) dsh = M[a][b];
+    }
+  // which of this thread's elements lie on or above the diagonal (fixed for the whole sweep)
+  uint32_t upper_mask = 0;
+#pragma unroll
+  for (int a = 0; a < 8; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+      if (tx + 32 * b >= ty + 16 * a) upper_mask |= 1u << (a * 4 + b);
   __syncthreads();
   for (int j = nb - 1; j >= 0; --j) {
-    double d = S[j * LD + j];
-    __syncthreads();
+    double d = dsh;
     if (!(d > 0.0)) {
       if (tid == 0) report_error(dev_info, GPTQ_ERR_NOT_PD, k0 + j);
       d = 1.0;
     }
-    double piv = sqrt(d), rp = 1.0 / piv;
-    for (int i = tid; i < j; i += nt) S[i * LD + j] *= rp;
-    if (tid == 0) S[j * LD + j] = piv;
-    __syncthreads();
-    // trailing update of the leading j x j upper part: A[i][i2] -= T[i][j] T[i2][j], i <= i2 < j
-    for (int e = tid; e < j * j; e += nt) {
-      int i = e / j, i2 = e % j;
-      if (i <= i2) S[i * LD + i2] -= S[i * LD + j] * S[i2 * LD + j];
+    const double piv = sqrt(d), rp = 1.0 / piv;
+    if (tid == 0) { pd[j] = piv; vd[j] = rp; }
+    // owners of column j scale it (finishing T[:, j] above the diagonal and V[j, :] below) and publish it
+    if (tx == (j & 31)) {
+      const int bj = j >> 5;
+#pragma unroll
+      for (int a = 0; a < 8; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const int i = ty + 16 * a;
+          if (b == bj && i != j) { M[a][b] *= rp; colv[i] = M[a][b]; }
+        }
     }
     __syncthreads();
-  }
-  // V = T^-1, one column c per thread (back substitution up the column); V[i][c], i < c, is kept
-  // at S[c][i] (the unused lower triangle), V[c][c] in vd[c].
-  for (int c = tid; c < nb; c += nt) {
-    const double vcc = 1.0 / S[c * LD + c];
-    vd[c] = vcc;
-    for (int i = c - 1; i >= 0; --i) {
-      double s = S[i * LD + c] * vcc;
-      for (int k = i + 1; k < c; ++k) s += S[i * LD + k] * S[c * LD + k];
-      S[c * LD + i] = -s / S[i * LD + i];
+    // one formula for both updates: M[i][c] -= x[i] * T[c][j] for c < j and (c >= i or i >= j),
+    // with x[i] = T[i][j] for i < j and V[j][i] for i >= j
+    double x[8], cc[4];
+    bool below[8];
+#pragma unroll
+    for (int a = 0; a < 8; ++a) { const int i = ty + 16 * a; x[a] = (i == j) ? rp : colv[i]; below[a] = i >= j; }
+#pragma unroll
+    for (int b = 0; b < 4; ++b) cc[b] = colv[tx + 32 * b];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const bool left = tx + 32 * b < j;
+#pragma unroll
+      for (int a = 0; a < 8; ++a)
+        if (left && (below[a] || ((upper_mask >> (a * 4 + b)) & 1u))) M[a][b] -= x[a] * cc[b];
     }
+#pragma unroll
+    for (int a = 0; a < 8; ++a)     // next pivot candidate (flat, statically indexed: keeps M in registers)
+#pragma unroll
+      for (int b = 0; b < 4; ++b)
+        if (ty + 16 * a == j - 1 && tx + 32 * b == j - 1) dsh = M[a][b];
+    __syncthreads();
   }
-  __syncthreads();
-  for (int e = tid; e < nb * nb; e += nt) {
-    int i = e / nb, j = e % nb;
-    if (j >= i) U[(int64_t)(k0 + i) * C + k0 + j] = (float)S[i * LD + j];
-    Dinv[i * kNB + j] = j > i ? (float)S[j * LD + i] : (j == i ? (float)vd[i] : 0.f);
-  }
+#pragma unroll
+  for (int a = 0; a < 8; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int i = ty + 16 * a, c = tx + 32 * b;
+      if (i < nb && c < nb) {
+        if (c > i) U[(int64_t)(k0 + i) * C + k0 + c] = (float)M[a][b];
+        else if (c == i) { U[(int64_t)(k0 + i) * C + k0 + c] = (float)pd[i]; Dinv[i * kNB + i] = (float)vd[i]; }
+        // V[c][i] (c < i) sits in M[i][c]; strictly lower part of V is zero
+        if (c < i) { Dinv[c * kNB + i] = (float)M[a][b]; Dinv[i * kNB + c] = 0.f; }
+      }
+    }
 }
 
 __global__ void store_diag_block_kernel(float* __restrict__ U, int C, int k0, int nb,
@@ -277,8 +316,6 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
   HinvWs w = carve_hinv(ws, C);
   gptq_status_t st;
 
-  const int diag_smem = (kNB * (kNB + 1) + kNB) * (int)sizeof(double);
-  GPTQ_CUDA_TRY(cudaFuncSetAttribute(rchol_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, diag_smem));
   GPTQ_CUDA_TRY(cudaMemsetAsync(dev_info, 0, 2 * sizeof(int), s));
   lambda_kernel<<<1, 1024, 0, s>>>(H, C, damp, w.lam);
   GPTQ_LAUNCH_CHECK();
@@ -306,7 +343,7 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
     for (int k0 = j0 + (wj - 1) / kNB * kNB; k0 >= j0; k0 -= kNB) {
       const int nb = (rows_p - k0 < kNB) ? rows_p - k0 : kNB;
       float* Dk = w.Dinv + (size_t)(k0 / kNB) * kNB * kNB;
-      rchol_diag_kernel<<<1, 256, diag_smem, s>>>(U, C, k0, nb, Dk, dev_info);
+      rchol_diag_kernel<<<1, kDiagThreads, 0, s>>>(U, C, k0, nb, Dk, dev_info);
       GPTQ_LAUNCH_CHECK();
       if (k0 == 0) break;
       // panel: U~[0:k0, blk] = A[0:k0, blk] * T_kk^-T      (out[m][n] = sum_k A[m][k0+k] V[n][k])

@@ -102,29 +102,51 @@ struct InblockArgs {
   float* Ehi; float* Elo; uint8_t* codes; double* loss; int* dev_info;
 };
 
-// One thread per row.  The block's working weights sit in shared memory, column-major (thread-
-// private columns, conflict-free); 32 columns at a time are held in registers, quantized one
-// after the other with immediate feedback (W[:, j:blockend] -= E_j U[j, j:blockend]) inside the
-// registers, then their 32 errors are applied to the rest of the block in shared memory.
-template <int RPB>
-__global__ void __launch_bounds__(RPB) inblock_kernel(InblockArgs a) {
+// Four lanes per row, 32 rows per CTA.  The block's working weights sit in shared memory,
+// column-major; a lane owns every fourth column.  32 columns at a time are held in registers
+// (8 per lane) and quantized one after the other: the owner's current weight is broadcast to its
+// quad with a warp shuffle, all four lanes take the (identical) rounding decision and error, and
+// each applies the immediate feedback W[:, j:blockend] -= E_j U[j, j:blockend] to the columns it
+// owns -- first inside the registers, then, 32 errors at a time, to the rest of the block in
+// shared memory.  Min/max for group grids are quad-wide shuffle reductions.
+constexpr int kRPB = 32;                 // rows per CTA
+constexpr int kInblockThreads = 4 * kRPB;
+constexpr int kLDS = kRPB + 4;           // slab row stride (doubles): 36 % 16 == 4 keeps quad accesses conflict-free
+
+__device__ __forceinline__ double quad_min(double v) {
+  v = fmin(v, __shfl_xor_sync(0xffffffffu, v, 1));
+  return fmin(v, __shfl_xor_sync(0xffffffffu, v, 2));
+}
+__device__ __forceinline__ double quad_max(double v) {
+  v = fmax(v, __shfl_xor_sync(0xffffffffu, v, 1));
+  return fmax(v, __shfl_xor_sync(0xffffffffu, v, 2));
+}
+
+__global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a) {
   extern __shared__ double smem[];
-  const int B = a.B, LDS = RPB + 1;
-  double* slab = smem;                  // [B][LDS]
-  double* Us = smem + (size_t)B * LDS;  // [kSB][B]   rows j0..j0+31 of the B x B block of U
-  const int t = threadIdx.x, r0 = blockIdx.x * RPB, row = r0 + t;
+  const int B = a.B;
+  double* slab = smem;                    // [B][kLDS]
+  double* Us = smem + (size_t)B * kLDS;   // [kSB][B]   rows j0..j0+31 of the B x B block of U
+  const int t = threadIdx.x, l = t & 3, rl = t >> 2;
+  const int r0 = blockIdx.x * kRPB, row = r0 + rl;
   const bool live = row < a.R;
 
-  // stage the slab: coalesced along columns, transposed into shared memory
-  for (int e = t; e < RPB * B; e += RPB) {
-    int rr = e / B, c = e % B;
-    slab[c * LDS + rr] = (r0 + rr < a.R) ? a.Wblk[(int64_t)(r0 + rr) * a.ldw + a.col0 + c] : 0.0;
+  // stage the slab: coalesced 16-byte loads along columns, transposed into shared memory
+  {
+    const int half = B >> 1;
+#pragma unroll 4
+    for (int e = t; e < kRPB * half; e += kInblockThreads) {
+      const int rr = e / half, c2 = e - rr * half;
+      double2 v = make_double2(0.0, 0.0);
+      if (r0 + rr < a.R) v = *reinterpret_cast<const double2*>(a.Wblk + (int64_t)(r0 + rr) * a.ldw + a.col0 + 2 * c2);
+      slab[(2 * c2) * kLDS + rr] = v.x;
+      slab[(2 * c2 + 1) * kLDS + rr] = v.y;
+    }
   }
-  const int G = a.G;
-  const int g = a.group;
+  const int G = a.G, g = a.group;
   float scale_f = 1.f, zero_f = 0.f;
-  if (live && !(a.grid_inside)) {
-    int gi = g > 0 ? a.i / g : 0;
+  if (live && !a.grid_inside) {
+    const int gi = g > 0 ? a.i / g : 0;
     scale_f = a.scales[(int64_t)row * G + gi];
     zero_f = a.zeros[(int64_t)row * G + gi];
   }
@@ -135,82 +157,94 @@ __global__ void __launch_bounds__(RPB) inblock_kernel(InblockArgs a) {
 
   for (int j0 = 0; j0 < B; j0 += kSB) {
     __syncthreads();  // slab staged / previous sub-block's Us no longer read
-    for (int e = t; e < kSB * B; e += RPB) {
-      int jj = e / B, c = e % B;
-      Us[jj * B + c] = (c >= j0) ? (double)a.U[(int64_t)(a.i + j0 + jj) * a.C + a.i + c] : 0.0;
+    {
+      const int q4 = B >> 2;
+#pragma unroll 4
+      for (int e = t; e < kSB * q4; e += kInblockThreads) {
+        const int jj = e / q4, c = (e - jj * q4) * 4;
+        if (c + 3 >= j0) {
+          const float4 u = *reinterpret_cast<const float4*>(a.U + (int64_t)(a.i + j0 + jj) * a.C + a.i + c);
+          double* d = Us + jj * B + c;
+          d[0] = (double)u.x; d[1] = (double)u.y; d[2] = (double)u.z; d[3] = (double)u.w;
+        }
+      }
     }
     __syncthreads();
-    double w[kSB], err[kSB];
+    double w[kSB / 4], err[kSB];
     uint32_t cw[kSB / 4];
 #pragma unroll
-    for (int jj = 0; jj < kSB; ++jj) w[jj] = slab[(j0 + jj) * LDS + t];
-#pragma unroll
-    for (int k = 0; k < kSB / 4; ++k) cw[k] = 0;
+    for (int m = 0; m < kSB / 4; ++m) { w[m] = slab[(j0 + 4 * m + l) * kLDS + rl]; cw[m] = 0; }
 
-    // group grid starting at this sub-block (group a multiple of 32, within the block)
+    // grid of a group that starts at this sub-block (group a multiple of 32, inside the block)
     if (a.grid_inside && g >= kSB && ((a.i + j0) % g) == 0) {
       double mn = INFINITY, mx = -INFINITY;
-      for (int c = j0; c < j0 + g; ++c) { double v = slab[c * LDS + t]; mn = fmin(mn, v); mx = fmax(mx, v); }
-      find_params(mn, mx, a.grid, scale_f, zero_f);
+      for (int c = j0 + l; c < j0 + g; c += 4) { const double v = slab[c * kLDS + rl]; mn = fmin(mn, v); mx = fmax(mx, v); }
+      find_params(quad_min(mn), quad_max(mx), a.grid, scale_f, zero_f);
       scale = (double)scale_f; zero = (double)zero_f;
-      if (live) {
-        int gi = (a.i + j0) / g;
+      if (live && l == 0) {
+        const int gi = (a.i + j0) / g;
         a.scales[(int64_t)row * G + gi] = scale_f; a.zeros[(int64_t)row * G + gi] = zero_f;
       }
     }
 #pragma unroll
     for (int jj = 0; jj < kSB; ++jj) {
+      const int m = jj >> 2, owner = jj & 3;
       if (a.grid_inside && g < kSB && (jj % g) == 0) {   // small groups live inside the registers
         double mn = INFINITY, mx = -INFINITY;
 #pragma unroll
-        for (int kk = 0; kk < kSB; ++kk)
-          if (kk >= jj && kk < jj + g) { mn = fmin(mn, w[kk]); mx = fmax(mx, w[kk]); }
-        find_params(mn, mx, a.grid, scale_f, zero_f);
+        for (int mm = 0; mm < kSB / 4; ++mm)
+          if (4 * mm >= jj && 4 * mm < jj + g) { mn = fmin(mn, w[mm]); mx = fmax(mx, w[mm]); }
+        find_params(quad_min(mn), quad_max(mx), a.grid, scale_f, zero_f);
         scale = (double)scale_f; zero = (double)zero_f;
-        if (live) {
-          int gi = (a.i + j0 + jj) / g;
+        if (live && l == 0) {
+          const int gi = (a.i + j0 + jj) / g;
           a.scales[(int64_t)row * G + gi] = scale_f; a.zeros[(int64_t)row * G + gi] = zero_f;
         }
       }
+      const double wj = __shfl_sync(0xffffffffu, w[m], owner, 4);
       const double d = Us[jj * B + j0 + jj];
-      double q = rint(w[jj] / scale) + zero;                 // quantize column
+      double q = rint(wj / scale) + zero;                    // quantize column
       q = fmin(fmax(q, 0.0), maxq);
       const double wq = scale * (q - zero);
-      const double e = (w[jj] - wq) / d;                     // quantization error
+      const double e = (wj - wq) / d;                        // quantization error
       err[jj] = e;
       loss += e * e;
       bad |= !isfinite(e);
-      cw[jj >> 2] |= (uint32_t)q << (8 * (jj & 3));
+      cw[m] |= (uint32_t)q << (8 * owner);
+      const double* urow = Us + jj * B + j0 + l;
 #pragma unroll
-      for (int kk = jj + 1; kk < kSB; ++kk) w[kk] -= e * Us[jj * B + j0 + kk];   // update weights in block
+      for (int mm = m; mm < kSB / 4; ++mm)                   // update weights in block (own columns > jj)
+        if (mm > m || l > owner) w[mm] -= e * urow[4 * mm];
     }
-    // remaining columns of the block: apply the 32 errors of this sub-block
-    for (int c = j0 + kSB; c < B; ++c) {
-      double x = slab[c * LDS + t];
+    // remaining columns of the block: apply the 32 errors of this sub-block to the columns this lane owns
+    for (int c = j0 + kSB + l; c < B; c += 4) {
+      double x = slab[c * kLDS + rl];
 #pragma unroll
       for (int jj = 0; jj < kSB; ++jj) x -= err[jj] * Us[jj * B + c];
-      slab[c * LDS + t] = x;
+      slab[c * kLDS + rl] = x;
     }
     if (live) {
-      float4* eh = reinterpret_cast<float4*>(a.Ehi + (int64_t)row * a.C + a.i + j0);
-      float4* el = reinterpret_cast<float4*>(a.Elo + (int64_t)row * a.C + a.i + j0);
+      // lane l stores columns [8 l, 8 l + 8) of this sub-block: errors as a tf32 hi / lo pair, codes as bytes
+      float h[8], lo[8];
 #pragma unroll
-      for (int k = 0; k < kSB / 4; ++k) {
-        float h[4], l[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) tf32x3::split_tf32((float)err[4 * k + u], h[u], l[u]);
-        eh[k] = make_float4(h[0], h[1], h[2], h[3]);
-        el[k] = make_float4(l[0], l[1], l[2], l[3]);
+      for (int u = 0; u < 8; ++u) {
+        const double ev = l == 0 ? err[u] : (l == 1 ? err[8 + u] : (l == 2 ? err[16 + u] : err[24 + u]));
+        tf32x3::split_tf32((float)ev, h[u], lo[u]);
       }
-      uint4* cp = reinterpret_cast<uint4*>(a.codes + (int64_t)row * a.C + a.i + j0);
-      cp[0] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
-      cp[1] = make_uint4(cw[4], cw[5], cw[6], cw[7]);
+      const int64_t o = (int64_t)row * a.C + a.i + j0 + 8 * l;
+      float4* eh = reinterpret_cast<float4*>(a.Ehi + o);
+      float4* el = reinterpret_cast<float4*>(a.Elo + o);
+      eh[0] = make_float4(h[0], h[1], h[2], h[3]); eh[1] = make_float4(h[4], h[5], h[6], h[7]);
+      el[0] = make_float4(lo[0], lo[1], lo[2], lo[3]); el[1] = make_float4(lo[4], lo[5], lo[6], lo[7]);
+      const uint32_t c0 = l == 0 ? cw[0] : (l == 1 ? cw[2] : (l == 2 ? cw[4] : cw[6]));
+      const uint32_t c1 = l == 0 ? cw[1] : (l == 1 ? cw[3] : (l == 2 ? cw[5] : cw[7]));
+      *reinterpret_cast<uint2*>(a.codes + o) = make_uint2(c0, c1);
     }
   }
-  if (!live) loss = 0.0;
+  if (!live || l != 0) loss = 0.0;
   for (int o = 16; o > 0; o >>= 1) loss += __shfl_down_sync(0xffffffffu, loss, o);
   if ((t & 31) == 0 && loss != 0.0) atomicAdd(a.loss, loss);
-  if (live && bad) report_error(a.dev_info, GPTQ_ERR_NONFINITE, row);
+  if (live && l == 0 && bad) report_error(a.dev_info, GPTQ_ERR_NONFINITE, row);
 }
 
 // ---- pack codes: little-endian bit stream per row, field width f --------------------------------
@@ -302,7 +336,7 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   if (g > 0) {
     if (C % g != 0) return GPTQ_ERR_INVALID_ARG;
     if (g % block != 0 && block % g != 0) return GPTQ_ERR_INVALID_ARG;   // groups and blocks must nest
-    if (g % kSB != 0 && kSB % g != 0) return GPTQ_ERR_UNSUPPORTED;
+    if (g % kSB != 0 && (kSB % g != 0 || g < 4)) return GPTQ_ERR_UNSUPPORTED;   // 4, 8, 16 or a multiple of 32
   }
   if (!ws || !aligned_to(ws, kAlign) || ws_bytes < gptq_quantize_workspace_bytes(R, C, bits, group_size, block))
     return GPTQ_ERR_WORKSPACE;
@@ -326,12 +360,8 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
     rowgrid_kernel<<<ceil_div(R, 8), 256, 0, s>>>(W, R, C, gs, scales, zeros);
     GPTQ_LAUNCH_CHECK();
   }
-  const int rpb = block > 128 ? 64 : 128;
-  auto inblock_smem = [&](int B) { return (size_t)((size_t)B * (rpb + 1) + (size_t)kSB * B) * sizeof(double); };
-  GPTQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)((256 * 65 + kSB * 256) * sizeof(double))));
-  GPTQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)((128 * 129 + kSB * 128) * sizeof(double))));
+  auto inblock_smem = [&](int B) { return (size_t)((size_t)B * kLDS + (size_t)kSB * B) * sizeof(double); };
+  GPTQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)inblock_smem(256)));
 
   for (int i2 = 0; i2 < C; i2 += B2) {
     const int nb2 = (C - i2 < B2) ? C - i2 : B2;
@@ -359,8 +389,7 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
       }
       InblockArgs a{Wblk, ldw, i - i2, U, C, i, B, R, gs, g, (g > 0 && g <= B) ? 1 : 0,
                     scales, zeros, G, Ehi, Elo, codes, loss, dev_info};
-      if (rpb == 64) inblock_kernel<64><<<ceil_div(R, 64), 64, inblock_smem(B), s>>>(a);
-      else inblock_kernel<128><<<ceil_div(R, 128), 128, inblock_smem(B), s>>>(a);
+      inblock_kernel<<<ceil_div(R, kRPB), kInblockThreads, inblock_smem(B), s>>>(a);
       GPTQ_LAUNCH_CHECK();
       // push this block's errors onto the remaining columns of the outer block
       const int rest = i2 + nb2 - (i + B);
