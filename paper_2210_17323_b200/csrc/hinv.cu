@@ -56,86 +56,85 @@ __global__ void init_upper_damped_kernel(const float* __restrict__ H, float* __r
 // V (solving T V = I from the bottom row up), then applies two rank-1 updates,
 //   A[i][c] -= T[i][j] T[c][j]   (i <= c < j)      and      B[c][i] -= T[c][j] V[j][i]   (c < j <= i),
 // where B is the running right-hand side of the solve.  The whole 128 x 128 working matrix M lives
-// in REGISTERS (32 doubles per thread, element (i, c) with i = ty + 16 a, c = tx + 32 b): its upper
-// triangle holds A / T, its strictly lower triangle holds B / V transposed (M[i][c] = B[c][i]).
-// Per step only column j (scaled) passes through shared memory.
+// in REGISTERS (32 doubles per thread, element (i, c) with i = tx + 32 a, c = ty + 16 b, ty = warp):
+// its upper triangle holds A / T, its strictly lower triangle holds B / V transposed
+// (M[i][c] = B[c][i]).  With that layout both updates are the same formula
+//   M[i][c] -= x[i] * T[c][j]   for c < j and (c >= i or i >= j),   x[i] = T[i][j] (i < j), V[j][i] (i >= j),
+// column j belongs to ONE warp (which takes the square root, scales and publishes it through
+// shared memory), and "c < j" is warp-uniform.  Register arrays are only ever indexed by
+// compile-time constants (thread coordinates are compared, never loop indices).
 // A non-positive pivot is reported and replaced by 1 so everything downstream stays finite.
 constexpr int kDiagThreads = 512;
 __global__ void __launch_bounds__(kDiagThreads)
 rchol_diag_kernel(float* __restrict__ U, int C, int k0, int nb, float* __restrict__ Dinv, int* dev_info) {
-  __shared__ double colv[kNB];   // step j: colv[i] = T[i][j] for i < j, V[j][i] for i > j
+  __shared__ double colv[kNB];   // step j: colv[i] = T[i][j] for i < j, V[j][i] for i > j, V[j][j] at i == j
   __shared__ double pd[kNB];     // diagonal of T
-  __shared__ double vd[kNB];     // diagonal of V
   __shared__ double dsh;         // pivot candidate of the current step
   const int tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
-  double M[8][4];
+  double M[4][8];
 #pragma unroll
-  for (int a = 0; a < 8; ++a)
+  for (int a = 0; a < 4; ++a)
 #pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      const int i = ty + 16 * a, c = tx + 32 * b;
+    for (int b = 0; b < 8; ++b) {
+      const int i = tx + 32 * a, c = ty + 16 * b;
       M[a][b] = (i < nb && c < nb && c >= i) ? (double)U[(int64_t)(k0 + i) * C + k0 + c] : 0.0;
       if (i == nb - 1 && c == nb - 1) dsh = M[a][b];
     }
-  // which of this thread's elements lie on or above the diagonal (fixed for the whole sweep)
-  uint32_t upper_mask = 0;
-#pragma unroll
-  for (int a = 0; a < 8; ++a)
-#pragma unroll
-    for (int b = 0; b < 4; ++b)
-      if (tx + 32 * b >= ty + 16 * a) upper_mask |= 1u << (a * 4 + b);
   __syncthreads();
   for (int j = nb - 1; j >= 0; --j) {
-    double d = dsh;
-    if (!(d > 0.0)) {
-      if (tid == 0) report_error(dev_info, GPTQ_ERR_NOT_PD, k0 + j);
-      d = 1.0;
-    }
-    const double piv = sqrt(d), rp = 1.0 / piv;
-    if (tid == 0) { pd[j] = piv; vd[j] = rp; }
-    // owners of column j scale it (finishing T[:, j] above the diagonal and V[j, :] below) and publish it
-    if (tx == (j & 31)) {
-      const int bj = j >> 5;
+    if (ty == (j & 15)) {
+      // the warp that owns column j: pivot, then scale and publish the column
+      double d = dsh;
+      if (!(d > 0.0)) {
+        if (tx == 0) report_error(dev_info, GPTQ_ERR_NOT_PD, k0 + j);
+        d = 1.0;
+      }
+      const double piv = sqrt(d), rp = 1.0 / piv;
 #pragma unroll
-      for (int a = 0; a < 8; ++a)
+      for (int a = 0; a < 4; ++a)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-          const int i = ty + 16 * a;
-          if (b == bj && i != j) { M[a][b] *= rp; colv[i] = M[a][b]; }
+        for (int b = 0; b < 8; ++b) {
+          const int i = tx + 32 * a;
+          if (ty + 16 * b == j) {
+            if (i == j) { pd[j] = piv; colv[i] = rp; }
+            else { M[a][b] *= rp; colv[i] = M[a][b]; }
+          }
         }
     }
     __syncthreads();
-    // one formula for both updates: M[i][c] -= x[i] * T[c][j] for c < j and (c >= i or i >= j),
-    // with x[i] = T[i][j] for i < j and V[j][i] for i >= j
-    double x[8], cc[4];
-    bool below[8];
+    double x[4];
 #pragma unroll
-    for (int a = 0; a < 8; ++a) { const int i = ty + 16 * a; x[a] = (i == j) ? rp : colv[i]; below[a] = i >= j; }
+    for (int a = 0; a < 4; ++a) x[a] = colv[tx + 32 * a];
 #pragma unroll
-    for (int b = 0; b < 4; ++b) cc[b] = colv[tx + 32 * b];
+    for (int b = 0; b < 8; ++b) {
+      const int c = ty + 16 * b;
+      if (c < j) {                                   // warp-uniform
+        const double tc = colv[c];
 #pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      const bool left = tx + 32 * b < j;
-#pragma unroll
-      for (int a = 0; a < 8; ++a)
-        if (left && (below[a] || ((upper_mask >> (a * 4 + b)) & 1u))) M[a][b] -= x[a] * cc[b];
+        for (int a = 0; a < 4; ++a) {
+          const int i = tx + 32 * a;
+          if (i >= j || c >= i) M[a][b] -= x[a] * tc;
+        }
+      }
     }
+    if (ty == ((j - 1) & 15)) {                      // next pivot candidate, element (j-1, j-1)
 #pragma unroll
-    for (int a = 0; a < 8; ++a)     // next pivot candidate (flat, statically indexed: keeps M in registers)
+      for (int a = 0; a < 4; ++a)
 #pragma unroll
-      for (int b = 0; b < 4; ++b)
-        if (ty + 16 * a == j - 1 && tx + 32 * b == j - 1) dsh = M[a][b];
+        for (int b = 0; b < 8; ++b)
+          if (tx + 32 * a == j - 1 && ty + 16 * b == j - 1) dsh = M[a][b];
+    }
     __syncthreads();
   }
 #pragma unroll
-  for (int a = 0; a < 8; ++a)
+  for (int a = 0; a < 4; ++a)
 #pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      const int i = ty + 16 * a, c = tx + 32 * b;
+    for (int b = 0; b < 8; ++b) {
+      const int i = tx + 32 * a, c = ty + 16 * b;
       if (i < nb && c < nb) {
         if (c > i) U[(int64_t)(k0 + i) * C + k0 + c] = (float)M[a][b];
-        else if (c == i) { U[(int64_t)(k0 + i) * C + k0 + c] = (float)pd[i]; Dinv[i * kNB + i] = (float)vd[i]; }
-        // V[c][i] (c < i) sits in M[i][c]; strictly lower part of V is zero
+        else if (c == i) { U[(int64_t)(k0 + i) * C + k0 + c] = (float)pd[i]; Dinv[i * kNB + i] = (float)(1.0 / pd[i]); }
+        // V[c][i] (c < i) sits in M[i][c]; the strictly lower part of V is zero
         if (c < i) { Dinv[c * kNB + i] = (float)M[a][b]; Dinv[i * kNB + c] = 0.f; }
       }
     }
