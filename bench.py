@@ -159,7 +159,7 @@ def run_reference(args, wl):
 def run_gpu(args, wl):
     import torch
     import torch.distributed as dist
-    from paper_2210_17323_b200 import binding as B
+    from paper_2210_17323_b200 import binding as B, multi
     from paper_2210_17323_b200.synth import device as D, workloads as WL
 
     rank = int(os.environ.get("RANK", "0"))
@@ -171,7 +171,7 @@ def run_gpu(args, wl):
         dist.init_process_group("nccl", device_id=dev)
 
     # each rank solves its own copy of the layer set (block index = rank -> its own seeds)
-    layers = [WL.Layer(l.config_id, l.block_idx + rank, l.kind, l.R, l.C, l.n_tokens) for l in wl.layers]
+    layers = multi.rank_layers(wl.layers, rank)
     state = []
     ws_bytes = 256
     for L in layers:
@@ -230,8 +230,7 @@ def run_gpu(args, wl):
     launches = B.gptq_launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
     ms = t0.elapsed_time(t1)
-    if world > 1:
-        t = torch.tensor([ms], device=dev); dist.all_reduce(t, op=dist.ReduceOp.MAX); ms = t.item()
+    ms = multi.max_over_ranks(ms, dev)
     ms_per_step = ms / args.steps
     n_grids = len(wl.grids)
     weights_step = wl.weights * n_grids * world
