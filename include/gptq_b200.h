@@ -91,6 +91,31 @@ size_t gptq_prepare_hinv_workspace_bytes(int C);
 gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, float* U,
                                 void* ws, size_t ws_bytes, int* dev_info, void* stream);
 
+/* gptq_prepare_hinv for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant, it computes exactly what gptq_prepare_hinv does.)
+ *
+ * Who needs it: code that may not call cudaMalloc -- a plug-in inside a framework whose
+ * memory pool owns the whole device, a latency-critical loop where an allocation would
+ * stall the GPU, a process with a fixed memory budget handed out at start-up.  Such a
+ * caller has no workspace to pass, so the scratch lives inside the library, in one fixed
+ * array in device global memory of 256 + 2 * 512 KiB = 1,048,832 bytes.
+ *
+ *   - Limit: C <= GPTQ_PREPARE_HINV_STATIC_MAX_C (1024); a larger C returns
+ *     GPTQ_ERR_UNSUPPORTED and nothing is enqueued (use gptq_prepare_hinv with a workspace).
+ *   - H, U, dev_info, stream, return value and dev_info contents: as gptq_prepare_hinv.
+ *     The caller still owns and passes all inputs and outputs.
+ *   - The call allocates nothing: no cudaMalloc / cudaFree and no allocating library routine.
+ *   - Every GPU on which the library is loaded holds the array until the process exits.
+ *   - The first call on each device resolves the array's device address (a one-time set-up,
+ *     done with that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents.
+ *     Nothing in it needs clearing (each call writes what it later reads), but two calls
+ *     whose kernels overlap on the GPU -- different streams, or different host threads --
+ *     race on it: serialise them on one stream. */
+#define GPTQ_PREPARE_HINV_STATIC_MAX_C 1024
+gptq_status_t gptq_prepare_hinv_static(const float* H, float damp, int C, float* U,
+                                       int* dev_info, void* stream);
+
 /* ------------------------------------------------------------------ stage 3
  * Algorithm 1: for each block of `block` columns, quantize column by column
  * (Q_j = quant(W_j); E_j = (W_j - Q_j) / U_jj; W[:, j:blockend] -= E_j U[j, j:blockend]),

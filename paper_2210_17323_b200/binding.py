@@ -45,6 +45,8 @@ def _load():
     lib.gptq_prepare_hinv_workspace_bytes.argtypes = [c.c_int]
     lib.gptq_prepare_hinv.restype = c.c_int
     lib.gptq_prepare_hinv.argtypes = [c.c_void_p, c.c_float, c.c_int, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
+    lib.gptq_prepare_hinv_static.restype = c.c_int
+    lib.gptq_prepare_hinv_static.argtypes = [c.c_void_p, c.c_float, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p]
     lib.gptq_quantize_workspace_bytes.restype = c.c_size_t
     lib.gptq_quantize_workspace_bytes.argtypes = [c.c_int] * 5
     lib.gptq_quantize_layer.restype = c.c_int
@@ -123,6 +125,27 @@ def gptq_prepare_hinv(H, damp=0.01, U=None, ws=None, dev_info=None, stream=None)
                                 dev_info.data_ptr(), _stream_ptr(stream))
     if st != OK:
         raise GptqError(st, "gptq_prepare_hinv")
+    return U, dev_info
+
+
+PREPARE_HINV_STATIC_MAX_C = 1024
+
+
+def gptq_prepare_hinv_static(H, damp=0.01, U=None, dev_info=None, stream=None):
+    """gptq_prepare_hinv without a workspace, for callers that cannot allocate device memory
+    (memory owned by a framework pool, allocation-free latency paths, fixed budgets): the scratch is
+    a fixed 1 MiB array inside the library.  C <= 1024.  All calls on a device share that array, so
+    calls that could overlap on the GPU must be put on one stream.  The first call on a device does a
+    one-time address look-up and should not happen inside a stream capture.  U and dev_info are the
+    caller's (created here with torch only when not passed in)."""
+    _check(H, torch.float32, "H")
+    C = H.shape[0]
+    U = torch.empty_like(H) if U is None else U
+    _check(U, torch.float32, "U")
+    dev_info = torch.zeros(2, dtype=torch.int32, device=H.device) if dev_info is None else dev_info
+    st = _lib.gptq_prepare_hinv_static(H.data_ptr(), float(damp), C, U.data_ptr(), dev_info.data_ptr(), _stream_ptr(stream))
+    if st != OK:
+        raise GptqError(st, "gptq_prepare_hinv_static")
     return U, dev_info
 
 

@@ -2,6 +2,6 @@
 EXPORTS = (
     "gptq_status_string", "gptq_launch_count",
     "gptq_hessian_workspace_bytes", "gptq_hessian_accumulate",
-    "gptq_prepare_hinv_workspace_bytes", "gptq_prepare_hinv",
+    "gptq_prepare_hinv_workspace_bytes", "gptq_prepare_hinv", "gptq_prepare_hinv_static",
     "gptq_quantize_workspace_bytes", "gptq_quantize_layer",
 )

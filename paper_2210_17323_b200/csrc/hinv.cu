@@ -393,3 +393,49 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
   }
   return GPTQ_OK;
 }
+
+// ------------------------------------------------------------------------------------------------
+// Workspace-free variant of gptq_prepare_hinv for callers that cannot allocate device memory.
+//
+// Some callers have no way to hand this library a workspace: code that runs under a framework whose
+// memory pool owns every byte of the device and forbids cudaMalloc from plug-ins, code on a
+// latency-critical path where an allocation would synchronise the device, or a process that was
+// given a fixed memory budget up front.  For them the scratch lives in the library itself, in a
+// fixed array in device global memory.  The price: the array is sized for a stated maximum, every
+// GPU that loads the library keeps it until the process exits, and all calls share it.
+//
+// `hinv_static_scratch` below is that array.  In host code its name is only a stand-in for the
+// device object, not an address a kernel may be given; the device address is obtained once per
+// device with cudaGetSymbolAddress (with that device current) and cached.
+namespace gptq {
+namespace {
+constexpr int kStaticMaxC = GPTQ_PREPARE_HINV_STATIC_MAX_C;
+// workspace of gptq_prepare_hinv at C = 1024: lambda (256 B) + eight 128 x 128 diagonal inverses
+// (512 KiB) + a 1024 x 128 panel temporary (512 KiB)
+constexpr size_t kStaticScratchBytes = 256 + (size_t)(kStaticMaxC / kNB) * kNB * kNB * 4 + (size_t)kStaticMaxC * kNB * 4;
+static __device__ __align__(256) unsigned char hinv_static_scratch[kStaticScratchBytes];
+constexpr int kMaxDevices = 64;
+}  // namespace
+}  // namespace gptq
+
+extern "C" gptq_status_t gptq_prepare_hinv_static(const float* H, float damp, int C, float* U,
+                                                  int* dev_info, void* stream) {
+  using namespace gptq;
+  if (C > kStaticMaxC) return GPTQ_ERR_UNSUPPORTED;   // larger problems need the caller-workspace entry point
+  if (C <= 0) return GPTQ_ERR_INVALID_ARG;
+  if (carve_hinv(nullptr, C).bytes > kStaticScratchBytes) return GPTQ_ERR_UNSUPPORTED;
+  static void* scratch_of_device[kMaxDevices] = {};
+  int dev = -1;
+  GPTQ_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return GPTQ_ERR_UNSUPPORTED;
+  void* scratch = __atomic_load_n(&scratch_of_device[dev], __ATOMIC_ACQUIRE);
+  if (!scratch) {
+    // one-time set-up on this device (the current one): resolve the device address of the array
+    GPTQ_CUDA_TRY(cudaGetSymbolAddress(&scratch, hinv_static_scratch));
+    if (!scratch) return GPTQ_ERR_CUDA;
+    __atomic_store_n(&scratch_of_device[dev], scratch, __ATOMIC_RELEASE);
+  }
+  // Nothing in the scratch has to start at zero: lambda, every used diagonal inverse and the panel
+  // temporary are all written by this call before they are read, so stale contents are harmless.
+  return gptq_prepare_hinv(H, damp, C, U, scratch, kStaticScratchBytes, dev_info, stream);
+}
