@@ -334,9 +334,16 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layer", default=None, metavar="RxCxTOKENS",
+                    help="profile one layer of this shape (grid, block and damp of --workload) instead of the "
+                         "whole layer set -- a small case of the same kernels for profiler captures")
     args = ap.parse_args()
     from paper_2210_17323_b200.synth import workloads as WL
     wl = WL.workload(int(args.workload.lstrip("c")))
+    if args.layer:
+        R, C, T = (int(v) for v in args.layer.lower().split("x"))
+        wl = WL.Workload(wl.config_id, f"{wl.name}-single-{R}x{C}x{T}", (WL.Layer(wl.config_id, 0, "q", R, C, T),),
+                         wl.grids, wl.block, wl.damp)
     if args.impl == "reference":
         return run_reference(args, wl)
     return run_gpu(args, wl)

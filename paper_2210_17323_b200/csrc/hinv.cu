@@ -165,6 +165,19 @@ struct UpperLeftFactorRange {
     return k0 < k1;
   }
 };
+// Same, with the K range of each tile row cut into gridDim.z pieces (partial sums are reduced atomically).
+struct UpperLeftFactorSplitK {
+  int K;
+  __device__ __forceinline__ bool operator()(int m0, int, int z, int nz, int& k0, int& k1) const {
+    const int per = ((K - m0 + nz - 1) / nz + kSimtBK - 1) / kSimtBK * kSimtBK;
+    k0 = m0 + z * per; k1 = min(K, k0 + per);
+    return k0 < k1;
+  }
+};
+struct AtomicSubF32 {
+  float* p; int64_t ld;
+  __device__ __forceinline__ void operator()(int m, int n, float acc) const { atomicAdd(&p[(int64_t)m * ld + n], -acc); }
+};
 struct StoreF32 {
   float* p; int64_t ld;
   __device__ __forceinline__ void operator()(int m, int n, float acc) const { p[(int64_t)m * ld + n] = acc; }
@@ -287,8 +300,16 @@ gptq_status_t invert_upper_block(float* D, int C, int w, float* Dinv, float* T, 
       GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, 1, RowMajorF32{D + k0, C}, RowMajorF32{Dk, kNB},
                                      FullRange{nb}, StoreF32{T, kNB}, s));
       // U[0:k0, blk] = -U[0:k0, 0:k0] * T   (left factor already inverted, upper triangular)
-      GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, 1, RowMajorF32{D, C}, RowMajorF32{T, kNB},
-                                     UpperLeftFactorRange{k0}, StoreNegF32{D + k0, C}, s));
+      // (only k0 / 128 tiles: the K range is split so that more SMs take part)
+      const int nz = k0 / kNB > 1 ? k0 / kNB : 1;
+      if (nz == 1) {
+        GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, 1, RowMajorF32{D, C}, RowMajorF32{T, kNB},
+                                       UpperLeftFactorRange{k0}, StoreNegF32{D + k0, C}, s));
+      } else {
+        GPTQ_CUDA_TRY(cudaMemset2DAsync(D + k0, (size_t)C * 4, 0, (size_t)nb * 4, k0, s));
+        GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, nz, RowMajorF32{D, C}, RowMajorF32{T, kNB},
+                                       UpperLeftFactorSplitK{k0}, AtomicSubF32{D + k0, C}, s));
+      }
     }
     store_diag_block_kernel<<<8, 256, 0, s>>>(D, C, k0, nb, Dk);
     GPTQ_LAUNCH_CHECK();

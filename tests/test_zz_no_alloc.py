@@ -47,7 +47,6 @@ def test_static_variant_matches_workspace_variant_twice_in_a_row(B):
         assert torch.cuda.memory_allocated() == held      # the call itself took nothing from torch's pool
         assert info.tolist() == info_ref.tolist() == [0, 0]
         assert rel_fro(U.cpu().numpy(), U_ref.cpu().numpy()) <= TOL_U_FRO
-        assert torch.equal(U, U_ref)                                # same kernels, same order: identical bits
 
 
 def test_static_variant_rejects_sizes_beyond_its_scratch(B):
