@@ -52,24 +52,52 @@ __global__ void init_upper_damped_kernel(const float* __restrict__ H, float* __r
 
 // One CTA: factor the nb x nb diagonal block at (k0, k0) as A = T T^T with T upper (backwards
 // Cholesky), store T in place (fp32) and its inverse V = T^-1 (upper) to Dinv (fp32, ld = kNB).
-// Both run in fp64, fused in one sweep j = nb-1 .. 0: step j finishes column j of T and row j of
-// V (solving T V = I from the bottom row up), then applies two rank-1 updates,
+// Both run in fp64, fused in one sweep over the columns j = nb-1 .. 0: column j of T and row j of V
+// (solving T V = I from the bottom row up) are finished together, and both trailing updates,
 //   A[i][c] -= T[i][j] T[c][j]   (i <= c < j)      and      B[c][i] -= T[c][j] V[j][i]   (c < j <= i),
-// where B is the running right-hand side of the solve.  The whole 128 x 128 working matrix M lives
-// in REGISTERS (32 doubles per thread, element (i, c) with i = tx + 32 a, c = ty + 16 b, ty = warp):
-// its upper triangle holds A / T, its strictly lower triangle holds B / V transposed
-// (M[i][c] = B[c][i]).  With that layout both updates are the same formula
-//   M[i][c] -= x[i] * T[c][j]   for c < j and (c >= i or i >= j),   x[i] = T[i][j] (i < j), V[j][i] (i >= j),
-// column j belongs to ONE warp (which takes the square root, scales and publishes it through
-// shared memory), and "c < j" is warp-uniform.  Register arrays are only ever indexed by
-// compile-time constants (thread coordinates are compared, never loop indices).
+// where B is the running right-hand side of the solve, are the same formula on one working matrix M
+// whose upper triangle holds A / T and whose strictly lower triangle holds B / V transposed:
+//   M[i][c] -= x_j[i] * T[c][j]   for c < j and (c >= i or i >= j),   x_j[i] = T[i][j] (i < j), V[j][i] (i >= j).
+// M lives in REGISTERS (32 doubles per thread, element (i, c) with i = tx + 32 a, c = ty + 16 b,
+// ty = warp), so a column belongs to ONE warp.  Updates are batched lazily, four columns at a time
+// (the same idea as Algorithm 1's Step 2, one level down): inside a batch only the owning warp of
+// the next column applies the pending updates to that column, takes the pivot, scales and
+// publishes it through shared memory; after the batch every warp applies the four rank-1 updates
+// to its other elements in one pass.  Register arrays are indexed by compile-time constants only
+// (thread coordinates are compared, never loop indices).
 // A non-positive pivot is reported and replaced by 1 so everything downstream stays finite.
 constexpr int kDiagThreads = 512;
+constexpr int kDiagBatch = 4;
+// Owner warp, column j = slots M[.][B] (rows i = tx + 32 a): apply the batch's pending updates to the
+// column, take the pivot, scale the column and publish it as colv[q][.] (colv[q][j] = 1 / pivot).
+template <int B>
+__device__ __forceinline__ void diag_owner_step(double (&M)[4][8], double (*colv)[kNB], double* pd, int q, int j, int jt,
+                                                int tx, int k0, int* dev_info) {
+  double piv_c = 0.0;
+#pragma unroll
+  for (int a = 0; a < 4; ++a) {
+    const int i = tx + 32 * a;
+    for (int qq = 0; qq < q; ++qq)
+      if (i >= jt - qq || j >= i) M[a][B] -= colv[qq][i] * colv[qq][j];
+    if (i == j) piv_c = M[a][B];
+  }
+  double d = __shfl_sync(0xffffffffu, piv_c, j & 31);
+  if (!(d > 0.0)) {
+    if (tx == 0) report_error(dev_info, GPTQ_ERR_NOT_PD, k0 + j);
+    d = 1.0;
+  }
+  const double rp = rsqrt(d), piv = d * rp;
+#pragma unroll
+  for (int a = 0; a < 4; ++a) {
+    const int i = tx + 32 * a;
+    if (i == j) { pd[j] = piv; colv[q][i] = rp; }
+    else { M[a][B] *= rp; colv[q][i] = M[a][B]; }
+  }
+}
 __global__ void __launch_bounds__(kDiagThreads)
 rchol_diag_kernel(float* __restrict__ U, int C, int k0, int nb, float* __restrict__ Dinv, int* dev_info) {
-  __shared__ double colv[kNB];   // step j: colv[i] = T[i][j] for i < j, V[j][i] for i > j, V[j][j] at i == j
-  __shared__ double pd[kNB];     // diagonal of T
-  __shared__ double dsh;         // pivot candidate of the current step
+  __shared__ double colv[kDiagBatch][kNB];   // published columns of the current batch: colv[q][i] = x_{jt-q}[i]
+  __shared__ double pd[kNB];                 // diagonal of T
   const int tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
   double M[4][8];
 #pragma unroll
@@ -78,51 +106,50 @@ rchol_diag_kernel(float* __restrict__ U, int C, int k0, int nb, float* __restric
     for (int b = 0; b < 8; ++b) {
       const int i = tx + 32 * a, c = ty + 16 * b;
       M[a][b] = (i < nb && c < nb && c >= i) ? (double)U[(int64_t)(k0 + i) * C + k0 + c] : 0.0;
-      if (i == nb - 1 && c == nb - 1) dsh = M[a][b];
     }
-  __syncthreads();
-  for (int j = nb - 1; j >= 0; --j) {
-    if (ty == (j & 15)) {
-      // the warp that owns column j: pivot, then scale and publish the column
-      double d = dsh;
-      if (!(d > 0.0)) {
-        if (tx == 0) report_error(dev_info, GPTQ_ERR_NOT_PD, k0 + j);
-        d = 1.0;
-      }
-      const double piv = sqrt(d), rp = 1.0 / piv;
+  for (int jt = nb - 1; jt >= 0; jt -= kDiagBatch) {
 #pragma unroll
-      for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int b = 0; b < 8; ++b) {
-          const int i = tx + 32 * a;
-          if (ty + 16 * b == j) {
-            if (i == j) { pd[j] = piv; colv[i] = rp; }
-            else { M[a][b] *= rp; colv[i] = M[a][b]; }
-          }
+    for (int q = 0; q < kDiagBatch; ++q) {
+      const int j = jt - q;
+      if (ty == (j & 15)) {
+        // owner warp of column j (its slots have b == j >> 4): dispatch once on b so that the
+        // four slots are addressed with compile-time indices
+        switch (j >> 4) {
+          case 0: diag_owner_step<0>(M, colv, pd, q, j, jt, tx, k0, dev_info); break;
+          case 1: diag_owner_step<1>(M, colv, pd, q, j, jt, tx, k0, dev_info); break;
+          case 2: diag_owner_step<2>(M, colv, pd, q, j, jt, tx, k0, dev_info); break;
+          case 3: diag_owner_step<3>(M, colv, pd, q, j, jt, tx, k0, dev_info); break;
+          case 4: diag_owner_step<4>(M, colv, pd, q, j, jt, tx, k0, dev_info); break;
+          case 5: diag_owner_step<5>(M, colv, pd, q, j, jt, tx, k0, dev_info); break;
+          case 6: diag_owner_step<6>(M, colv, pd, q, j, jt, tx, k0, dev_info); break;
+          default: diag_owner_step<7>(M, colv, pd, q, j, jt, tx, k0, dev_info); break;
         }
+      }
+      __syncthreads();
     }
-    __syncthreads();
-    double x[4];
+    // the batch's four rank-1 updates on every element left of the batch
+    const int jlow = jt - (kDiagBatch - 1);
+    double x[kDiagBatch][4];
+    bool below[kDiagBatch][4];
 #pragma unroll
-    for (int a = 0; a < 4; ++a) x[a] = colv[tx + 32 * a];
+    for (int q = 0; q < kDiagBatch; ++q)
+#pragma unroll
+      for (int a = 0; a < 4; ++a) { const int i = tx + 32 * a; x[q][a] = colv[q][i]; below[q][a] = i >= jt - q; }
 #pragma unroll
     for (int b = 0; b < 8; ++b) {
       const int c = ty + 16 * b;
-      if (c < j) {                                   // warp-uniform
-        const double tc = colv[c];
+      if (c < jlow) {                                // warp-uniform
+        double tc[kDiagBatch];
+#pragma unroll
+        for (int q = 0; q < kDiagBatch; ++q) tc[q] = colv[q][c];
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
-          const int i = tx + 32 * a;
-          if (i >= j || c >= i) M[a][b] -= x[a] * tc;
+          const bool upper = c >= tx + 32 * a;
+#pragma unroll
+          for (int q = 0; q < kDiagBatch; ++q)
+            if (upper || below[q][a]) M[a][b] -= x[q][a] * tc[q];
         }
       }
-    }
-    if (ty == ((j - 1) & 15)) {                      // next pivot candidate, element (j-1, j-1)
-#pragma unroll
-      for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int b = 0; b < 8; ++b)
-          if (tx + 32 * a == j - 1 && ty + 16 * b == j - 1) dsh = M[a][b];
     }
     __syncthreads();
   }
