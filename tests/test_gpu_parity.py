@@ -207,3 +207,25 @@ def test_config0_end_to_end(B, D):
                zeros=out["zeros"].cpu().numpy(), loss=out["loss"].item())
     figs = check_quantize_outputs(gpu, ref, W16, grid.bits, L.C, ref["H"])
     print("config0 end-to-end:", figs)
+
+
+def test_midsize_end_to_end_grouped(B, D):
+    """2048 columns, 32768 tokens, 3-bit g128: every stage crosses several outer panels / blocks and all
+    tensor-core paths run; the oracle does the whole layer (its own H and U) for the comparison."""
+    L = _layer(192, 2048, 32768, cfg=6, kind="fc1")
+    bits_host = np.concatenate([L.x_bits(t0, t0 + 8192) for t0 in range(0, L.n_tokens, 8192)])
+    W16 = L.w()
+    ref = O.solve_layer(W16, bits_host, 3, 128, False, 128, 0.01)
+    X, W = D.fill_x(L), D.fill_w(L)
+    H = torch.zeros((L.C, L.C), dtype=torch.float32, device="cuda")
+    B.gptq_hessian_accumulate(H, X)
+    U, info = B.gptq_prepare_hinv(H, 0.01)
+    out = B.gptq_quantize_layer(W, U, 3, 128, False, 128)
+    torch.cuda.synchronize()
+    assert info.tolist()[0] == 0 and out["dev_info"].tolist()[0] == 0
+    assert rel_fro(H.cpu().numpy(), ref["H"]) <= TOL_H_FRO
+    assert rel_fro(U.cpu().numpy(), ref["U"]) <= TOL_U_FRO
+    gpu = dict(qweight=out["qweight"].cpu().numpy(), scales=out["scales"].cpu().numpy(),
+               zeros=out["zeros"].cpu().numpy(), loss=out["loss"].item())
+    figs = check_quantize_outputs(gpu, ref, W16, 3, L.C, ref["H"])
+    print("midsize end-to-end:", figs)
