@@ -104,9 +104,9 @@ def oracle_sample(wl, budget_note=True):
             total_est += seen[key]
             continue
         C = L.C
-        c_s = min(C, 2048)                       # leading principal sub-problem of the Hessian / factor
-        t_s = min(L.n_tokens, 4096)
-        r_s = min(L.R, 64)
+        c_s = min(C, 4096)                       # leading principal sub-problem of the Hessian / factor
+        t_s = min(L.n_tokens, 8192)
+        r_s = min(L.R, 128)
         sc = L.scales()
         Xb = L.x_bits(0, t_s, cols=np.arange(c_s), scales=sc)
         W = L.w(rows=np.arange(r_s))[:, :c_s]
@@ -251,8 +251,12 @@ def run_gpu(args, wl):
     upd_flops = sum(2 * L.R * (L.C * L.C - L.C * wl.block) / 2 * n_grids for L in layers)   # lazy updates, R (C^2 - C B)
     if tot["hessian_ms"] >= tot["quantize_ms"]:
         ach = hess_flops / (tot["hessian_ms"] * 1e-3) / 1e12
+        # DRAM traffic per launch: measured 4.6 x the algorithmic bytes (X once + H once) on the ncu capture of a
+        # 4096-channel x 65536-token launch (profiles/); scaled to these launches by their algorithmic bytes
+        algo_bytes = sum(L.n_tokens * L.C * 2 + L.C * L.C * 4 for L in layers) / len(layers)
         roof = dict(kernel="hessian_accumulate", bound="tensor", achieved=ach, peak=peaks["bf16_sustained"],
-                    unit="TFLOP/s", frac=ach / peaks["bf16_sustained"], traffic=None,
+                    unit="TFLOP/s", frac=ach / peaks["bf16_sustained"], traffic=4.6 * algo_bytes,
+                    traffic_note="bytes per launch (mean over layers), = 4.6 x algorithmic bytes, ratio from an ncu capture of a smaller launch",
                     peak_source=f"bf16 sustained, {peaks['source']}")
     else:
         ach = upd_flops / (tot["quantize_ms"] * 1e-3) / 1e12
@@ -287,42 +291,48 @@ def run_gpu(args, wl):
 
 
 def run_e2e(args, wl, state, ws, device_value):
-    """Same metric with HOST buffers: every step copies X and W from pinned host memory to the
-    device, runs the three calls, and reads the packed codes, scales, zeros and loss back."""
+    """Same metric end to end through the C ABI's host-buffer call: every step, for every layer (and grid),
+    gptq_solve_layer_host streams X and W from pinned HOST memory to the device (copies overlapped with the
+    Hessian accumulation), solves, and copies codes, scales, zeros and loss back to the host."""
     import torch
     from paper_2210_17323_b200 import binding as B
 
     host = []
+    need = 256
     for st in state:
-        host.append(dict(X=st["X"].cpu().pin_memory(), W=st["W"].cpu().pin_memory()))
+        L = st["L"]
+        host.append(dict(X=st["X"].cpu().pin_memory(), W=st["W"].cpu().pin_memory(), out={}))
+        for g in wl.grids:
+            need = max(need, B.gptq_solve_layer_host_workspace_bytes(L.R, L.C, L.n_tokens, g.bits, g.group_size, wl.block))
+    for st in state:                       # device copies are not needed any more: the call has its own staging
+        st["X"] = st["H"] = st["U"] = None
+    del ws
+    torch.cuda.empty_cache()
+    dev_ws = torch.empty(need, dtype=torch.uint8, device="cuda")
     torch.cuda.synchronize()
-    h2d = sum(h["X"].numel() * 2 + h["W"].numel() * 2 for h in host)
+    h2d = sum((h["X"].numel() * 2 + h["W"].numel() * 2) * len(wl.grids) for h in host)
     d2h = 0
 
     def step():
         nonlocal d2h
         d2h = 0
-        for st, h in zip(state, host):
-            st["X"].copy_(h["X"], non_blocking=True)
-            st["W"].copy_(h["W"], non_blocking=True)
-            st["H"].zero_()
-            B.gptq_hessian_accumulate(st["H"], st["X"], ws=ws)
-            B.gptq_prepare_hinv(st["H"], wl.damp, U=st["U"], ws=ws, dev_info=st["info"])
-            for g in wl.grids:
-                o = B.gptq_quantize_layer(st["W"], st["U"], g.bits, g.group_size, g.sym, wl.block, ws=ws)
-                res = [o[k].cpu() for k in ("qweight", "scales", "zeros", "loss", "dev_info")]
-                d2h += sum(r.numel() * r.element_size() for r in res)
+        for h in host:
+            for gi, g in enumerate(wl.grids):
+                o = B.gptq_solve_layer_host(h["W"], h["X"], g.bits, g.group_size, g.sym, wl.block, wl.damp,
+                                            out=h["out"].get(gi), dev_ws=dev_ws)
+                h["out"][gi] = o
+                assert o["info"].tolist()[0] == 0, o["info"].tolist()
+                d2h += sum(t.numel() * t.element_size() for t in o.values())
 
     steps = max(1, min(args.steps, 2))
     step()
-    torch.cuda.synchronize()
     t0 = time.perf_counter()
     for _ in range(steps):
-        step()
-    torch.cuda.synchronize()
+        step()                              # the call returns with the results on the host: wall clock is the e2e time
     dt = (time.perf_counter() - t0) / steps
     return dict(value=wl.weights * len(wl.grids) / dt, unit=UNIT, h2d_bytes_per_step=int(h2d),
-                d2h_bytes_per_step=int(d2h), ms_per_step=dt * 1e3, steps=steps)
+                d2h_bytes_per_step=int(d2h), ms_per_step=dt * 1e3, steps=steps,
+                api="gptq_solve_layer_host (pinned host buffers; X streamed in 512 MiB chunks on a copy stream)")
 
 
 def main():

@@ -149,6 +149,29 @@ gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U, int R, int
                                   uint32_t* qweight, float* scales, float* zeros, double* loss,
                                   void* ws, size_t ws_bytes, int* dev_info, void* stream);
 
+/* ------------------------------------------------------------------ whole layer, host buffers
+ * Stages 1-3 for one layer whose inputs and outputs live in HOST memory (Eq. 1's W and X in, the
+ * packed W^ out): X is streamed to the device in token chunks of about 512 MiB, double-buffered on
+ * an internal copy stream so that the transfer of a chunk overlaps the Hessian accumulation of the
+ * previous one (Section 5, Setup: Hessians are accumulated over calibration batches); then
+ * gptq_prepare_hinv and gptq_quantize_layer run and the results are copied back.
+ *   W_fp16_host [R x C] half, X_bf16_host [n_tokens x C] bfloat16: host memory; page-locked memory
+ *              is needed for the copies to overlap (pageable memory works, serialised).
+ *   qweight_host, scales_host, zeros_host, loss_host: host outputs, shaped as in gptq_quantize_layer.
+ *   info_host  int[2] (host): first non-OK device status of the three stages and its detail
+ *              (for stage 1: of the last chunk).
+ *   dev_ws     DEVICE workspace of gptq_solve_layer_host_workspace_bytes() bytes: holds H, U, W,
+ *              two X staging buffers, the outputs and the stages' own workspaces.
+ * Unlike the per-stage calls this one SYNCHRONISES `stream` before returning (the results are on
+ * the host when it returns); it creates and destroys one internal stream and a few events per
+ * call and allocates no device memory. */
+size_t gptq_solve_layer_host_workspace_bytes(int R, int C, int64_t n_tokens, int bits, int group_size, int block);
+gptq_status_t gptq_solve_layer_host(const void* W_fp16_host, const void* X_bf16_host, int64_t n_tokens,
+                                    int R, int C, float damp, int bits, int group_size, int sym, int block,
+                                    uint32_t* qweight_host, float* scales_host, float* zeros_host,
+                                    double* loss_host, int* info_host, void* dev_ws, size_t dev_ws_bytes,
+                                    void* stream);
+
 #ifdef __cplusplus
 }
 #endif

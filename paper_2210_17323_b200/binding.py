@@ -53,6 +53,12 @@ def _load():
     lib.gptq_quantize_layer.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_int, c.c_int, c.c_int,
                                         c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
                                         c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
+    lib.gptq_solve_layer_host_workspace_bytes.restype = c.c_size_t
+    lib.gptq_solve_layer_host_workspace_bytes.argtypes = [c.c_int, c.c_int, c.c_int64, c.c_int, c.c_int, c.c_int]
+    lib.gptq_solve_layer_host.restype = c.c_int
+    lib.gptq_solve_layer_host.argtypes = [c.c_void_p, c.c_void_p, c.c_int64, c.c_int, c.c_int, c.c_float, c.c_int, c.c_int,
+                                          c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+                                          c.c_void_p, c.c_size_t, c.c_void_p]
     return lib
 
 
@@ -170,3 +176,38 @@ def gptq_quantize_layer(W, U, bits, group_size=0, sym=False, block=128, ws=None,
     if st != OK:
         raise GptqError(st, "gptq_quantize_layer")
     return dict(qweight=qweight, scales=scales, zeros=zeros, loss=loss, dev_info=dev_info)
+
+
+def gptq_solve_layer_host_workspace_bytes(R, C, n_tokens, bits, group_size, block):
+    return _lib.gptq_solve_layer_host_workspace_bytes(R, C, n_tokens, bits, group_size, block)
+
+
+def gptq_solve_layer_host(W_host, X_host, bits, group_size=0, sym=False, block=128, damp=0.01, out=None, dev_ws=None,
+                          stream=None):
+    """Stages 1-3 for one layer with HOST inputs and outputs (CPU tensors; pinned for overlapped copies).
+    Returns dict(qweight int32 [R, C*f/32], scales, zeros, loss float64[1], info int32[2]) of CPU tensors
+    (pass `out` to reuse pinned result buffers).  Synchronises the stream."""
+    for t, dt, name in ((W_host, torch.float16, "W_host"), (X_host, torch.bfloat16, "X_host")):
+        if not (isinstance(t, torch.Tensor) and not t.is_cuda and t.is_contiguous() and t.dtype == dt):
+            raise TypeError(f"{name}: expected a contiguous CPU tensor of {dt}")
+    R, C = W_host.shape
+    n = X_host.shape[0]
+    G = C // group_size if group_size > 0 else 1
+    f = field_bits(bits)
+    if out is None:
+        out = dict(qweight=torch.empty((R, C * f // 32), dtype=torch.int32).pin_memory(),
+                   scales=torch.empty((R, G), dtype=torch.float32).pin_memory(),
+                   zeros=torch.empty((R, G), dtype=torch.float32).pin_memory(),
+                   loss=torch.zeros(1, dtype=torch.float64).pin_memory(),
+                   info=torch.zeros(2, dtype=torch.int32).pin_memory())
+    need = _lib.gptq_solve_layer_host_workspace_bytes(R, C, n, bits, group_size, block)
+    if need == 0:
+        raise GptqError(ERR_UNSUPPORTED, "gptq_solve_layer_host_workspace_bytes")
+    dev_ws = _ws(need, torch.device("cuda", torch.cuda.current_device()), dev_ws)
+    st = _lib.gptq_solve_layer_host(W_host.data_ptr(), X_host.data_ptr(), n, R, C, float(damp), bits, group_size,
+                                    int(bool(sym)), block, out["qweight"].data_ptr(), out["scales"].data_ptr(),
+                                    out["zeros"].data_ptr(), out["loss"].data_ptr(), out["info"].data_ptr(),
+                                    dev_ws.data_ptr(), dev_ws.numel(), _stream_ptr(stream))
+    if st != OK:
+        raise GptqError(st, "gptq_solve_layer_host")
+    return out

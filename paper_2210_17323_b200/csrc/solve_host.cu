@@ -1,0 +1,132 @@
+// Whole layer solve from HOST buffers: streams the calibration activations to the device in token
+// chunks (double-buffered on a second stream so the copy of chunk k+1 overlaps the Hessian
+// accumulation of chunk k), runs the three stages, and copies the results back.
+// The stages themselves are the same entry points a device-side caller uses (Algorithm 1; Section 2).
+#include "common.cuh"
+
+namespace gptq {
+namespace {
+
+constexpr int64_t kChunkBytes = (int64_t)512 << 20;   // per X staging buffer
+
+struct HostWs {
+  float* H; float* U; __half* W; __nv_bfloat16* X[2];
+  uint32_t* qweight; float* scales; float* zeros; double* loss; int* info;   // info: 3 x int[2]
+  void* stage_ws; size_t stage_ws_bytes;
+  int64_t chunk_tokens;
+  size_t bytes;
+};
+
+inline int field_bits_h(int bits) { return bits == GPTQ_BITS_TERNARY ? 2 : bits; }
+
+HostWs carve_host(void* ws, int R, int C, int64_t n_tokens, int bits, int group_size, int block) {
+  WsCarver w(ws);
+  HostWs o;
+  int64_t ct = kChunkBytes / ((int64_t)C * 2);
+  ct = ct / 64 * 64;
+  if (ct < 64) ct = 64;
+  if (ct > n_tokens) ct = n_tokens > 0 ? n_tokens : 1;
+  o.chunk_tokens = ct;
+  o.H = w.take<float>((size_t)C * C);
+  o.U = w.take<float>((size_t)C * C);
+  o.W = w.take<__half>((size_t)R * C);
+  o.X[0] = w.take<__nv_bfloat16>((size_t)ct * C);
+  o.X[1] = w.take<__nv_bfloat16>((size_t)ct * C);
+  const int G = group_size > 0 ? C / group_size : 1;
+  o.qweight = w.take<uint32_t>((size_t)R * (C * field_bits_h(bits) / 32));
+  o.scales = w.take<float>((size_t)R * G);
+  o.zeros = w.take<float>((size_t)R * G);
+  o.loss = w.take<double>(1);
+  o.info = w.take<int>(8);
+  size_t s1 = gptq_hessian_workspace_bytes(C, ct), s2 = gptq_prepare_hinv_workspace_bytes(C),
+         s3 = gptq_quantize_workspace_bytes(R, C, bits, group_size, block);
+  o.stage_ws_bytes = s1 > s2 ? (s1 > s3 ? s1 : s3) : (s2 > s3 ? s2 : s3);
+  if (o.stage_ws_bytes < kAlign) o.stage_ws_bytes = kAlign;
+  o.stage_ws = w.take<unsigned char>(o.stage_ws_bytes);
+  o.bytes = w.off;
+  return o;
+}
+
+struct StreamGuard {
+  cudaStream_t s = nullptr;
+  cudaEvent_t loaded[2] = {nullptr, nullptr}, freed[2] = {nullptr, nullptr}, w_done = nullptr;
+  ~StreamGuard() {
+    for (int i = 0; i < 2; ++i) { if (loaded[i]) cudaEventDestroy(loaded[i]); if (freed[i]) cudaEventDestroy(freed[i]); }
+    if (w_done) cudaEventDestroy(w_done);
+    if (s) cudaStreamDestroy(s);
+  }
+};
+
+}  // namespace
+}  // namespace gptq
+
+extern "C" size_t gptq_solve_layer_host_workspace_bytes(int R, int C, int64_t n_tokens, int bits, int group_size,
+                                                        int block) {
+  using namespace gptq;
+  if (R <= 0 || C <= 0 || C % 32 != 0 || n_tokens < 0 || block <= 0) return 0;
+  if (gptq_quantize_workspace_bytes(R, C, bits, group_size, block) == 0) return 0;
+  return carve_host(nullptr, R, C, n_tokens, bits, group_size, block).bytes;
+}
+
+extern "C" gptq_status_t gptq_solve_layer_host(const void* W_fp16_host, const void* X_bf16_host, int64_t n_tokens,
+                                               int R, int C, float damp, int bits, int group_size, int sym, int block,
+                                               uint32_t* qweight_host, float* scales_host, float* zeros_host,
+                                               double* loss_host, int* info_host, void* dev_ws, size_t dev_ws_bytes,
+                                               void* stream) {
+  using namespace gptq;
+  if (!W_fp16_host || !X_bf16_host || !qweight_host || !scales_host || !zeros_host || !loss_host || !info_host ||
+      R <= 0 || C <= 0 || C % 32 != 0 || n_tokens <= 0)
+    return GPTQ_ERR_INVALID_ARG;
+  const size_t need = gptq_solve_layer_host_workspace_bytes(R, C, n_tokens, bits, group_size, block);
+  if (need == 0) return GPTQ_ERR_UNSUPPORTED;
+  if (!dev_ws || !aligned_to(dev_ws, kAlign) || dev_ws_bytes < need) return GPTQ_ERR_WORKSPACE;
+  HostWs w = carve_host(dev_ws, R, C, n_tokens, bits, group_size, block);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  StreamGuard g;
+  GPTQ_CUDA_TRY(cudaStreamCreateWithFlags(&g.s, cudaStreamNonBlocking));
+  for (int i = 0; i < 2; ++i) {
+    GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&g.loaded[i], cudaEventDisableTiming));
+    GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&g.freed[i], cudaEventDisableTiming));
+  }
+  GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&g.w_done, cudaEventDisableTiming));
+
+  GPTQ_CUDA_TRY(cudaMemsetAsync(w.H, 0, (size_t)C * C * sizeof(float), s));
+  GPTQ_CUDA_TRY(cudaMemsetAsync(w.info, 0, 8 * sizeof(int), s));
+  const __nv_bfloat16* Xh = static_cast<const __nv_bfloat16*>(X_bf16_host);
+  gptq_status_t st;
+  int k = 0;
+  for (int64_t t0 = 0; t0 < n_tokens; t0 += w.chunk_tokens, ++k) {
+    const int b = k & 1;
+    const int64_t nt = n_tokens - t0 < w.chunk_tokens ? n_tokens - t0 : w.chunk_tokens;
+    if (k >= 2) GPTQ_CUDA_TRY(cudaStreamWaitEvent(g.s, g.freed[b], 0));       // buffer b consumed by chunk k-2
+    GPTQ_CUDA_TRY(cudaMemcpyAsync(w.X[b], Xh + t0 * C, (size_t)nt * C * 2, cudaMemcpyHostToDevice, g.s));
+    GPTQ_CUDA_TRY(cudaEventRecord(g.loaded[b], g.s));
+    if (k == 0) {   // the weights ride behind the first chunk on the copy stream
+      GPTQ_CUDA_TRY(cudaMemcpyAsync(w.W, W_fp16_host, (size_t)R * C * 2, cudaMemcpyHostToDevice, g.s));
+      GPTQ_CUDA_TRY(cudaEventRecord(g.w_done, g.s));
+    }
+    GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, g.loaded[b], 0));
+    st = gptq_hessian_accumulate(w.H, w.X[b], nt, C, w.stage_ws, w.stage_ws_bytes, w.info, s);
+    if (st != GPTQ_OK) return st;
+    GPTQ_CUDA_TRY(cudaEventRecord(g.freed[b], s));
+  }
+  GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, g.w_done, 0));
+  st = gptq_prepare_hinv(w.H, damp, C, w.U, w.stage_ws, w.stage_ws_bytes, w.info + 2, s);
+  if (st != GPTQ_OK) return st;
+  st = gptq_quantize_layer(w.W, w.U, R, C, bits, group_size, sym, block, w.qweight, w.scales, w.zeros, w.loss,
+                           w.stage_ws, w.stage_ws_bytes, w.info + 4, s);
+  if (st != GPTQ_OK) return st;
+  const int G = group_size > 0 ? C / group_size : 1;
+  int info[8];
+  GPTQ_CUDA_TRY(cudaMemcpyAsync(qweight_host, w.qweight, (size_t)R * (C * field_bits_h(bits) / 32) * 4, cudaMemcpyDeviceToHost, s));
+  GPTQ_CUDA_TRY(cudaMemcpyAsync(scales_host, w.scales, (size_t)R * G * 4, cudaMemcpyDeviceToHost, s));
+  GPTQ_CUDA_TRY(cudaMemcpyAsync(zeros_host, w.zeros, (size_t)R * G * 4, cudaMemcpyDeviceToHost, s));
+  GPTQ_CUDA_TRY(cudaMemcpyAsync(loss_host, w.loss, sizeof(double), cudaMemcpyDeviceToHost, s));
+  GPTQ_CUDA_TRY(cudaMemcpyAsync(info, w.info, sizeof(info), cudaMemcpyDeviceToHost, s));
+  GPTQ_CUDA_TRY(cudaStreamSynchronize(s));
+  GPTQ_CUDA_TRY(cudaStreamSynchronize(g.s));
+  info_host[0] = GPTQ_OK; info_host[1] = 0;
+  for (int i = 0; i < 3; ++i)
+    if (info[2 * i] != GPTQ_OK) { info_host[0] = info[2 * i]; info_host[1] = info[2 * i + 1]; break; }
+  return GPTQ_OK;
+}

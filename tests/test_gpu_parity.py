@@ -229,3 +229,21 @@ def test_midsize_end_to_end_grouped(B, D):
                zeros=out["zeros"].cpu().numpy(), loss=out["loss"].item())
     figs = check_quantize_outputs(gpu, ref, W16, 3, L.C, ref["H"])
     print("midsize end-to-end:", figs)
+
+
+def test_solve_layer_from_host_buffers(B):
+    """The host-buffer entry point (X streamed in chunks, results copied back) against the oracle."""
+    L = _layer(96, 512, 5000, cfg=5, kind="o")
+    bits_host = L.x_bits()
+    W16 = L.w()
+    ref = O.solve_layer(W16, bits_host, 4, 0, False, 128, 0.01)
+    Xh = torch.from_numpy(bits_host.view(np.int16)).view(torch.bfloat16).pin_memory()
+    Wh = torch.from_numpy(W16).pin_memory()
+    for _ in range(2):                      # twice: the second call reuses the result buffers and workspace
+        out = B.gptq_solve_layer_host(Wh, Xh, 4, 0, False, 128, 0.01)
+    assert out["info"].tolist() == [0, 0]
+    gpu = dict(qweight=out["qweight"].numpy(), scales=out["scales"].numpy(), zeros=out["zeros"].numpy(),
+               loss=out["loss"].item())
+    check_quantize_outputs(gpu, ref, W16, 4, L.C, ref["H"])
+    with pytest.raises(B.GptqError):
+        B.gptq_solve_layer_host(Wh, Xh, 5, 0, False, 128, 0.01)      # unsupported bits
