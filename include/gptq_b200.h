@@ -69,8 +69,9 @@ uint64_t gptq_launch_count(void);
  *   n_tokens >= 0 (0 is a no-op).
  *   dev_info int[2] or NULL: [0] = GPTQ_OK or GPTQ_ERR_TIMEOUT (a bounded wait inside the
  *            kernel ran out; H is then incomplete), [1] = which wait.
- * Products of bf16 values are exact in fp32; accumulation is fp32: at most 8192 tokens in
- * one tensor-core accumulator, chunks summed in fp32 in memory. */
+ * Products of bf16 values are exact in fp32; accumulation is fp32 and hierarchical: at most
+ * 512 tokens in one tensor-core accumulator, those sums added round-to-nearest in registers
+ * over at most 16384 tokens, and those added to H in memory. */
 size_t gptq_hessian_workspace_bytes(int C, int64_t n_tokens);
 gptq_status_t gptq_hessian_accumulate(float* H, const void* X_bf16, int64_t n_tokens, int C,
                                       void* ws, size_t ws_bytes, int* dev_info, void* stream);

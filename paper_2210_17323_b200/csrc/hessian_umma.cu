@@ -9,7 +9,7 @@
 // groups one box = 8192 B apart).
 //
 // Work decomposition: output tiles of 128 x 256 that touch the upper triangle, times super-chunks
-// of up to 8192 tokens.  Accumulation is hierarchical: 256 tokens (16 MMAs) in a TMEM accumulator,
+// of up to 16384 tokens.  Accumulation is hierarchical: 512 tokens (32 MMAs) in a TMEM accumulator,
 // chunk sums added round-to-nearest in registers over the super-chunk, super-chunk sums added to H
 // with vector reductions (red.global.add.v4.f32).
 #include "hessian_umma.cuh"
@@ -28,7 +28,7 @@ struct HessTraits {
   static constexpr int A_BYTES = (BM / 64) * BOX_BYTES;   // 16 KB
   static constexpr int B_BYTES = (BN / 64) * BOX_BYTES;   // 32 KB
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 48 KB
-  static constexpr int CHUNK_KB = 4;                      // 256 tokens = 16 MMAs per TMEM accumulation
+  static constexpr int CHUNK_KB = 8;                      // 512 tokens = 32 MMAs per TMEM accumulation
   struct Maps { CUtensorMap x; };
 
   static __device__ __forceinline__ void prefetch(const Maps& m) { umma::prefetch_tmap(&m.x); }
@@ -153,9 +153,10 @@ gptq_status_t hessian_umma(float* H, const __nv_bfloat16* X, int64_t n_tokens, i
   }
   for (int mi = 0; mi < it.tiles_m; ++mi) n_valid += it.tiles_n - (mi >> 1);
   it.total_kb = ceil_div(n_tokens, BK);
-  // tokens per super-chunk: at most 8192 (128 blocks); shorter when there are too few tiles to fill the GPU
+  // tokens per super-chunk: 16384 (256 blocks) while a super-chunk's slice of X still shares L2 with the
+  // reductions into H, 8192 beyond that; shorter when there are too few tiles to fill the GPU
   const int sms = device_sm_count();
-  int ck = 128;
+  int ck = C <= 8192 ? 256 : 128;
   while (ck > 8 && (int64_t)n_valid * ceil_div(it.total_kb, ck) < 2 * sms) ck >>= 1;
   it.sc_kb = ck;
   const int n_sc = ceil_div(it.total_kb, ck);
