@@ -14,6 +14,7 @@
 // with vector reductions (red.global.add.v4.f32).
 #include "hessian_umma.cuh"
 #include "umma_pipe.cuh"
+#include "umma_pipe2.cuh"
 
 namespace gptq {
 
@@ -71,6 +72,56 @@ struct HessItems {
     kb0 = sc * sc_kb;
     kb1 = min(total_kb, kb0 + sc_kb);
     return (mi >> 1) <= nj;          // tile touches the upper triangle: m0 <= n0 + BN - 1
+  }
+};
+
+// ---- two-CTA variant: 256 x 256 tiles, each CTA stages 128 rows of A and 128 columns of B -------
+struct HessPairTraits {
+  static constexpr int STAGES = 6;
+  static constexpr int A_BYTES = 2 * BOX_BYTES;           // 16 KB: this CTA's 128 rows
+  static constexpr int B_BYTES = 2 * BOX_BYTES;           // 16 KB: this CTA's 128 of the 256 columns
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 32 KB per CTA
+  static constexpr int CHUNK_KB = 8;
+  struct Maps { CUtensorMap x; };
+
+  static __device__ __forceinline__ void prefetch(const Maps& m) { umma::prefetch_tmap(&m.x); }
+  static __device__ __forceinline__ void load(uint8_t* s, const Maps& m, int m0, int n0, int kb, uint64_t* bar) {
+    const int y = kb * BK;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) umma::tma_load_2d_pair(s + j * BOX_BYTES, &m.x, m0 + 64 * j, y, bar);
+#pragma unroll
+    for (int j = 0; j < 2; ++j) umma::tma_load_2d_pair(s + A_BYTES + j * BOX_BYTES, &m.x, n0 + 64 * j, y, bar);
+  }
+  static __device__ __forceinline__ void mma(uint32_t d_tmem, uint32_t s, bool fresh) {
+    using namespace umma;
+    constexpr uint32_t idesc = make_idesc(kFmtBF16, true, true, 256, 256);
+#pragma unroll
+    for (int k = 0; k < BK / 16; ++k) {
+      const uint64_t da = make_desc_sw128(s + k * 2048, BOX_BYTES, 1024);
+      const uint64_t db = make_desc_sw128(s + A_BYTES + k * 2048, BOX_BYTES, 1024);
+      mma_f16_pair(d_tmem, da, db, idesc, (fresh && k == 0) ? 0u : 1u);
+    }
+  }
+};
+
+// 256 x 256 tiles on or above the diagonal, in bands of 8 tile rows, column by column inside a band.
+struct HessPairItems {
+  int tiles, n_enum, sc_kb, total_kb;
+  static constexpr int kBand = 8;
+  __device__ __forceinline__ bool operator()(int idx, int& m0, int& n0, int& kb0, int& kb1) const {
+    const int sc = idx / n_enum;
+    int t = idx % n_enum, mi = 0, nj = 0;
+    for (int s = 0; s * kBand < tiles; ++s) {
+      const int rows = min(kBand, tiles - s * kBand);
+      const int first = s * kBand;
+      const int cnt = rows * (tiles - first);
+      if (t < cnt) { nj = first + t / rows; mi = s * kBand + t % rows; break; }
+      t -= cnt;
+    }
+    m0 = mi * 256; n0 = nj * 256;
+    kb0 = sc * sc_kb;
+    kb1 = min(total_kb, kb0 + sc_kb);
+    return mi <= nj;
   }
 };
 
@@ -139,28 +190,46 @@ bool hessian_umma_supported(int C, int64_t n_tokens) {
 
 gptq_status_t hessian_umma(float* H, const __nv_bfloat16* X, int64_t n_tokens, int C, int* dev_info,
                            cudaStream_t stream) {
-  HessTraits::Maps maps;
-  gptq_status_t st = make_tmap_2d(&maps.x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)C, (uint64_t)n_tokens,
+  CUtensorMap tmap;
+  gptq_status_t st = make_tmap_2d(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)C, (uint64_t)n_tokens,
                                   (uint64_t)C * 2, 64, BK);
   if (st != GPTQ_OK) return st;
-  HessItems it;
-  it.tiles_m = ceil_div(C, BM); it.tiles_n = ceil_div(C, BN);
-  it.n_enum = 0;
-  int n_valid = 0;
-  for (int s = 0; s * SUPER_ROWS < it.tiles_m; ++s) {
-    int rows = it.tiles_m - s * SUPER_ROWS < SUPER_ROWS ? it.tiles_m - s * SUPER_ROWS : SUPER_ROWS;
-    it.n_enum += rows * (it.tiles_n - ((s * SUPER_ROWS) >> 1));
-  }
-  for (int mi = 0; mi < it.tiles_m; ++mi) n_valid += it.tiles_n - (mi >> 1);
-  it.total_kb = ceil_div(n_tokens, BK);
+  const int sms = device_sm_count();
+  const int total_kb = ceil_div(n_tokens, BK);
   // tokens per super-chunk: 16384 (256 blocks) while a super-chunk's slice of X still shares L2 with the
   // reductions into H, 8192 beyond that; shorter when there are too few tiles to fill the GPU
-  const int sms = device_sm_count();
   int ck = C <= 8192 ? 256 : 128;
-  while (ck > 8 && (int64_t)n_valid * ceil_div(it.total_kb, ck) < 2 * sms) ck >>= 1;
-  it.sc_kb = ck;
-  const int n_sc = ceil_div(it.total_kb, ck);
-  st = pipe::launch_pipe<HessTraits>(maps, (int64_t)it.n_enum * n_sc, it, EpiAddTwiceUpper{H, C}, dev_info, stream);
+  if (C >= 512) {
+    // two-CTA tiles of 256 x 256
+    HessPairTraits::Maps maps{tmap};
+    HessPairItems it;
+    it.tiles = ceil_div(C, 256);
+    it.n_enum = 0;
+    for (int s = 0; s * HessPairItems::kBand < it.tiles; ++s) {
+      int rows = it.tiles - s * HessPairItems::kBand < HessPairItems::kBand ? it.tiles - s * HessPairItems::kBand : HessPairItems::kBand;
+      it.n_enum += rows * (it.tiles - s * HessPairItems::kBand);
+    }
+    const int n_valid = it.tiles * (it.tiles + 1) / 2;
+    while (ck > 8 && (int64_t)n_valid * ceil_div(total_kb, ck) < sms) ck >>= 1;
+    it.total_kb = total_kb; it.sc_kb = ck;
+    st = pipe2::launch_pipe2<HessPairTraits>(maps, (int64_t)it.n_enum * ceil_div(total_kb, ck), it, EpiAddTwiceUpper{H, C},
+                                             dev_info, stream);
+  } else {
+    HessTraits::Maps maps{tmap};
+    HessItems it;
+    it.tiles_m = ceil_div(C, BM); it.tiles_n = ceil_div(C, BN);
+    it.n_enum = 0;
+    int n_valid = 0;
+    for (int s = 0; s * SUPER_ROWS < it.tiles_m; ++s) {
+      int rows = it.tiles_m - s * SUPER_ROWS < SUPER_ROWS ? it.tiles_m - s * SUPER_ROWS : SUPER_ROWS;
+      it.n_enum += rows * (it.tiles_n - ((s * SUPER_ROWS) >> 1));
+    }
+    for (int mi = 0; mi < it.tiles_m; ++mi) n_valid += it.tiles_n - (mi >> 1);
+    while (ck > 8 && (int64_t)n_valid * ceil_div(total_kb, ck) < 2 * sms) ck >>= 1;
+    it.total_kb = total_kb; it.sc_kb = ck;
+    st = pipe::launch_pipe<HessTraits>(maps, (int64_t)it.n_enum * ceil_div(total_kb, ck), it, EpiAddTwiceUpper{H, C},
+                                       dev_info, stream);
+  }
   if (st != GPTQ_OK) return st;
   GPTQ_CUDA_TRY(launch_mirror_upper_to_lower(H, C, stream));
   return GPTQ_OK;

@@ -51,7 +51,7 @@ def test_device_filler_matches_host_generator(D):
 
 
 # ------------------------------------------------------------------ stage 1
-@pytest.mark.parametrize("C,m", [(32, 1), (96, 77), (160, 1000), (256, 4096), (768, 8192)])
+@pytest.mark.parametrize("C,m", [(32, 1), (96, 77), (160, 1000), (256, 4096), (768, 8192), (1056, 777), (544, 1)])
 def test_hessian_matches_oracle(B, C, m):
     L = _layer(8, C, m)
     bits = L.x_bits()
@@ -168,6 +168,16 @@ def test_quantize_degenerate_inputs(B):
     Wg = ((lv - 8) * 2.0 ** -7).astype(np.float16)
     out = _run_quant(B, Wg, U32, 4, 0, False, 32)
     assert np.array_equal(O.unpack_codes(out["qweight"].view(np.uint32), 4, C), lv) and out["loss"] == 0.0
+
+
+def test_quantize_reports_nonfinite_weights(B):
+    C = 64
+    W = np.full((4, C), 0.01, np.float16)
+    W[2, 5] = np.inf
+    out = B.gptq_quantize_layer(torch.from_numpy(W).cuda(), torch.eye(C, device="cuda"), 4, 0, False, 32)
+    torch.cuda.synchronize()
+    st, where = out["dev_info"].tolist()
+    assert st == B.ERR_NONFINITE and where == 2
 
 
 def test_argument_errors_are_synchronous(B):
