@@ -127,6 +127,8 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
   const int B = a.B;
   double* slab = smem;                    // [B][kLDS]
   double* Us = smem + (size_t)B * kLDS;   // [kSB][B]   rows j0..j0+31 of the B x B block of U
+  double* esm = Us + (size_t)kSB * B;     // [kSB][kRPB] errors of the current sub-block, per row
+  double* rdiag = esm + kSB * kRPB;       // [kSB]       1 / U_jj of the current sub-block
   const int t = threadIdx.x, l = t & 3, rl = t >> 2;
   const int r0 = blockIdx.x * kRPB, row = r0 + rl;
   const bool live = row < a.R;
@@ -134,7 +136,7 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
   // stage the slab: coalesced 16-byte loads along columns, transposed into shared memory
   {
     const int half = B >> 1;
-#pragma unroll 4
+#pragma unroll 8
     for (int e = t; e < kRPB * half; e += kInblockThreads) {
       const int rr = e / half, c2 = e - rr * half;
       double2 v = make_double2(0.0, 0.0);
@@ -159,21 +161,25 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
     __syncthreads();  // slab staged / previous sub-block's Us no longer read
     {
       const int q4 = B >> 2;
-#pragma unroll 4
+#pragma unroll 8
       for (int e = t; e < kSB * q4; e += kInblockThreads) {
         const int jj = e / q4, c = (e - jj * q4) * 4;
         if (c + 3 >= j0) {
           const float4 u = *reinterpret_cast<const float4*>(a.U + (int64_t)(a.i + j0 + jj) * a.C + a.i + c);
           double* d = Us + jj * B + c;
           d[0] = (double)u.x; d[1] = (double)u.y; d[2] = (double)u.z; d[3] = (double)u.w;
+          const int dj = j0 + jj - c;                  // the diagonal entry U_jj, if it is in this quad of columns
+          if (dj >= 0 && dj < 4) rdiag[jj] = 1.0 / (double)(dj == 0 ? u.x : (dj == 1 ? u.y : (dj == 2 ? u.z : u.w)));
         }
       }
     }
     __syncthreads();
-    double w[kSB / 4], err[kSB];
-    uint32_t cw[kSB / 4];
+    // w[g]: this lane's column of group g (columns j0 + 4 g + l), rotated so that w[0] is always the group
+    // being quantized -- the loop over groups stays a real loop (small code, no instruction-cache thrash)
+    double w[kSB / 4];
 #pragma unroll
-    for (int m = 0; m < kSB / 4; ++m) { w[m] = slab[(j0 + 4 * m + l) * kLDS + rl]; cw[m] = 0; }
+    for (int m = 0; m < kSB / 4; ++m) w[m] = slab[(j0 + 4 * m + l) * kLDS + rl];
+    uint32_t c0 = 0, c1 = 0;
 
     // grid of a group that starts at this sub-block (group a multiple of 32, inside the block)
     if (a.grid_inside && g >= kSB && ((a.i + j0) % g) == 0) {
@@ -186,36 +192,46 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
         a.scales[(int64_t)row * G + gi] = scale_f; a.zeros[(int64_t)row * G + gi] = zero_f;
       }
     }
-#pragma unroll
-    for (int jj = 0; jj < kSB; ++jj) {
-      const int m = jj >> 2, owner = jj & 3;
-      if (a.grid_inside && g < kSB && (jj % g) == 0) {   // small groups live inside the registers
+#pragma unroll 1
+    for (int m = 0; m < kSB / 4; ++m) {
+      if (a.grid_inside && g < kSB && ((4 * m) % g) == 0) {   // small groups (4, 8, 16) live inside the registers
         double mn = INFINITY, mx = -INFINITY;
 #pragma unroll
-        for (int mm = 0; mm < kSB / 4; ++mm)
-          if (4 * mm >= jj && 4 * mm < jj + g) { mn = fmin(mn, w[mm]); mx = fmax(mx, w[mm]); }
+        for (int mm = 0; mm < 4; ++mm)
+          if (4 * mm < g) { mn = fmin(mn, w[mm]); mx = fmax(mx, w[mm]); }
         find_params(quad_min(mn), quad_max(mx), a.grid, scale_f, zero_f);
         scale = (double)scale_f; zero = (double)zero_f;
         if (live && l == 0) {
-          const int gi = (a.i + j0 + jj) / g;
+          const int gi = (a.i + j0 + 4 * m) / g;
           a.scales[(int64_t)row * G + gi] = scale_f; a.zeros[(int64_t)row * G + gi] = zero_f;
         }
       }
-      const double wj = __shfl_sync(0xffffffffu, w[m], owner, 4);
-      const double d = Us[jj * B + j0 + jj];
-      double q = rint(wj / scale) + zero;                    // quantize column
-      q = fmin(fmax(q, 0.0), maxq);
-      const double wq = scale * (q - zero);
-      const double e = (wj - wq) / d;                        // quantization error
-      err[jj] = e;
-      loss += e * e;
-      bad |= !isfinite(e);
-      cw[m] |= (uint32_t)q << (8 * owner);
-      const double* urow = Us + jj * B + j0 + l;
+      uint32_t packed = 0;
 #pragma unroll
-      for (int mm = m; mm < kSB / 4; ++mm)                   // update weights in block (own columns > jj)
-        if (mm > m || l > owner) w[mm] -= e * urow[4 * mm];
+      for (int o = 0; o < 4; ++o) {
+        const int jj = 4 * m + o;
+        const double wj = __shfl_sync(0xffffffffu, w[0], o, 4);
+        double q = rint(wj / scale) + zero;                    // quantize column
+        q = fmin(fmax(q, 0.0), maxq);
+        const double wq = scale * (q - zero);
+        const double e = (wj - wq) * rdiag[jj];                // quantization error (w - q) / U_jj
+        if (l == o) esm[jj * kRPB + rl] = e;
+        loss += e * e;
+        bad |= !isfinite(e);
+        packed |= (uint32_t)q << (8 * o);
+        const double* urow = Us + jj * B + j0 + 4 * m + l;
+#pragma unroll
+        for (int mm = 0; mm < kSB / 4; ++mm)                   // update weights in block (own columns > jj)
+          if (mm < kSB / 4 - m && (mm > 0 || l > o)) w[mm] -= e * urow[4 * mm];
+      }
+      if ((m >> 1) == l) { if (m & 1) c1 = packed; else c0 = packed; }
+#pragma unroll
+      for (int mm = 0; mm + 1 < kSB / 4; ++mm) w[mm] = w[mm + 1];
     }
+    __syncwarp();                                              // esm rows of this warp are complete
+    double err[kSB];
+#pragma unroll
+    for (int jj = 0; jj < kSB; ++jj) err[jj] = esm[jj * kRPB + rl];
     // remaining columns of the block: apply the 32 errors of this sub-block to the columns this lane owns
     for (int c = j0 + kSB + l; c < B; c += 4) {
       double x = slab[c * kLDS + rl];
@@ -236,8 +252,6 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
       float4* el = reinterpret_cast<float4*>(a.Elo + o);
       eh[0] = make_float4(h[0], h[1], h[2], h[3]); eh[1] = make_float4(h[4], h[5], h[6], h[7]);
       el[0] = make_float4(lo[0], lo[1], lo[2], lo[3]); el[1] = make_float4(lo[4], lo[5], lo[6], lo[7]);
-      const uint32_t c0 = l == 0 ? cw[0] : (l == 1 ? cw[2] : (l == 2 ? cw[4] : cw[6]));
-      const uint32_t c1 = l == 0 ? cw[1] : (l == 1 ? cw[3] : (l == 2 ? cw[5] : cw[7]));
       *reinterpret_cast<uint2*>(a.codes + o) = make_uint2(c0, c1);
     }
   }
@@ -360,7 +374,7 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
     rowgrid_kernel<<<ceil_div(R, 8), 256, 0, s>>>(W, R, C, gs, scales, zeros);
     GPTQ_LAUNCH_CHECK();
   }
-  auto inblock_smem = [&](int B) { return (size_t)((size_t)B * kLDS + (size_t)kSB * B) * sizeof(double); };
+  auto inblock_smem = [&](int B) { return (size_t)((size_t)B * kLDS + (size_t)kSB * B + kSB * kRPB + kSB) * sizeof(double); };
   GPTQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)inblock_smem(256)));
 
   for (int i2 = 0; i2 < C; i2 += B2) {
