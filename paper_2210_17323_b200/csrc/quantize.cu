@@ -127,8 +127,9 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
   const int B = a.B;
   double* slab = smem;                    // [B][kLDS]
   double* Us = smem + (size_t)B * kLDS;   // [kSB][B]   rows j0..j0+31 of the B x B block of U
-  double* esm = Us + (size_t)kSB * B;     // [kSB][kRPB] errors of the current sub-block, per row
-  double* rdiag = esm + kSB * kRPB;       // [kSB]       1 / U_jj of the current sub-block
+  double* rdiag = Us + (size_t)kSB * B;   // [kSB]       1 / U_jj of the current sub-block
+  float* esm = reinterpret_cast<float*>(rdiag + kSB);   // [kSB][kRPB] errors of the current sub-block, per row (fp32:
+                                                        // the precision E leaves the kernel in)
   const int t = threadIdx.x, l = t & 3, rl = t >> 2;
   const int r0 = blockIdx.x * kRPB, row = r0 + rl;
   const bool live = row < a.R;
@@ -152,7 +153,7 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
     scale_f = a.scales[(int64_t)row * G + gi];
     zero_f = a.zeros[(int64_t)row * G + gi];
   }
-  double scale = (double)scale_f, zero = (double)zero_f;
+  double scale = (double)scale_f, zero = (double)zero_f, rscale = 1.0 / scale;
   const double maxq = (double)a.grid.maxq;
   double loss = 0.0;
   bool bad = false;
@@ -186,7 +187,7 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
       double mn = INFINITY, mx = -INFINITY;
       for (int c = j0 + l; c < j0 + g; c += 4) { const double v = slab[c * kLDS + rl]; mn = fmin(mn, v); mx = fmax(mx, v); }
       find_params(quad_min(mn), quad_max(mx), a.grid, scale_f, zero_f);
-      scale = (double)scale_f; zero = (double)zero_f;
+      scale = (double)scale_f; zero = (double)zero_f; rscale = 1.0 / scale;
       if (live && l == 0) {
         const int gi = (a.i + j0) / g;
         a.scales[(int64_t)row * G + gi] = scale_f; a.zeros[(int64_t)row * G + gi] = zero_f;
@@ -200,7 +201,7 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
         for (int mm = 0; mm < 4; ++mm)
           if (4 * mm < g) { mn = fmin(mn, w[mm]); mx = fmax(mx, w[mm]); }
         find_params(quad_min(mn), quad_max(mx), a.grid, scale_f, zero_f);
-        scale = (double)scale_f; zero = (double)zero_f;
+        scale = (double)scale_f; zero = (double)zero_f; rscale = 1.0 / scale;
         if (live && l == 0) {
           const int gi = (a.i + j0 + 4 * m) / g;
           a.scales[(int64_t)row * G + gi] = scale_f; a.zeros[(int64_t)row * G + gi] = zero_f;
@@ -211,11 +212,16 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
       for (int o = 0; o < 4; ++o) {
         const int jj = 4 * m + o;
         const double wj = __shfl_sync(0xffffffffu, w[0], o, 4);
-        double q = rint(wj / scale) + zero;                    // quantize column
+        // quantize column: rne(w / scale).  The quotient is formed with the reciprocal; only when it lands within
+        // 1e-6 of a tie (where the reciprocal's last-bit error could change the rounding) is the division done.
+        const double tq = wj * rscale;
+        double q = rint(tq);
+        if (fabs(fabs(tq - q) - 0.5) < 1e-6) q = rint(wj / scale);
+        q += zero;
         q = fmin(fmax(q, 0.0), maxq);
         const double wq = scale * (q - zero);
         const double e = (wj - wq) * rdiag[jj];                // quantization error (w - q) / U_jj
-        if (l == o) esm[jj * kRPB + rl] = e;
+        if (l == o) esm[jj * kRPB + rl] = (float)e;
         loss += e * e;
         bad |= !isfinite(e);
         packed |= (uint32_t)q << (8 * o);
@@ -231,7 +237,7 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
     __syncwarp();                                              // esm rows of this warp are complete
     double err[kSB];
 #pragma unroll
-    for (int jj = 0; jj < kSB; ++jj) err[jj] = esm[jj * kRPB + rl];
+    for (int jj = 0; jj < kSB; ++jj) err[jj] = (double)esm[jj * kRPB + rl];
     // remaining columns of the block: apply the 32 errors of this sub-block to the columns this lane owns
     for (int c = j0 + kSB + l; c < B; c += 4) {
       double x = slab[c * kLDS + rl];
@@ -374,7 +380,7 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
     rowgrid_kernel<<<ceil_div(R, 8), 256, 0, s>>>(W, R, C, gs, scales, zeros);
     GPTQ_LAUNCH_CHECK();
   }
-  auto inblock_smem = [&](int B) { return (size_t)((size_t)B * kLDS + (size_t)kSB * B + kSB * kRPB + kSB) * sizeof(double); };
+  auto inblock_smem = [&](int B) { return (size_t)((size_t)B * kLDS + (size_t)kSB * B + kSB) * sizeof(double) + (size_t)kSB * kRPB * sizeof(float); };
   GPTQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)inblock_smem(256)));
 
   for (int i2 = 0; i2 < C; i2 += B2) {
