@@ -129,7 +129,9 @@ gptq_status_t gptq_prepare_hinv_static(const float* H, float damp, int C, float*
  *              > 0: g consecutive weights share a grid, taken at the group's first
  *              column from the weights as updated so far (Section 5: "always using
  *              the most current updated weights").  Must divide C, and nest with
- *              `block` (g % block == 0 or block % g == 0).
+ *              `block` (g % block == 0 or block % g == 0).  Supported sizes: 4, 8, 16
+ *              or any multiple of 32 (the paper uses 8, 32, 64, 128, 1024); anything
+ *              else returns GPTQ_ERR_UNSUPPORTED.
  *   sym        0: asymmetric min-max grid (range widened to contain 0, integer
  *              zero-point).  non-zero: symmetric grid, zero = (maxq+1)/2.
  *              The ternary grid is always symmetric.
@@ -149,6 +151,14 @@ gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U, int R, int
                                   int bits, int group_size, int sym, int block,
                                   uint32_t* qweight, float* scales, float* zeros, double* loss,
                                   void* ws, size_t ws_bytes, int* dev_info, void* stream);
+
+/* ------------------------------------------------------------------ round-to-nearest baseline
+ * RTN (Section 5, "Baselines"): every weight rounded to the nearest value of "exactly the same"
+ * grid -- per-row (group_size <= 0) or per-group min-max taken from the ORIGINAL weights -- with
+ * no error feedback.  Equals gptq_quantize_layer for a diagonal Hessian.  Arguments and output
+ * layout as in gptq_quantize_layer (any group size that divides C); no workspace, no dev_info. */
+gptq_status_t gptq_rtn_layer(const void* W_fp16, int R, int C, int bits, int group_size, int sym,
+                             uint32_t* qweight, float* scales, float* zeros, void* stream);
 
 /* ------------------------------------------------------------------ whole layer, host buffers
  * Stages 1-3 for one layer whose inputs and outputs live in HOST memory (Eq. 1's W and X in, the

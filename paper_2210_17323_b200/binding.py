@@ -59,6 +59,8 @@ def _load():
     lib.gptq_solve_layer_host.argtypes = [c.c_void_p, c.c_void_p, c.c_int64, c.c_int, c.c_int, c.c_float, c.c_int, c.c_int,
                                           c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
                                           c.c_void_p, c.c_size_t, c.c_void_p]
+    lib.gptq_rtn_layer.restype = c.c_int
+    lib.gptq_rtn_layer.argtypes = [c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
     return lib
 
 
@@ -211,3 +213,18 @@ def gptq_solve_layer_host(W_host, X_host, bits, group_size=0, sym=False, block=1
     if st != OK:
         raise GptqError(st, "gptq_solve_layer_host")
     return out
+
+
+def gptq_rtn_layer(W, bits, group_size=0, sym=False, stream=None):
+    """Round-to-nearest on the solver's grid, no error feedback.  Returns dict(qweight, scales, zeros)."""
+    _check(W, torch.float16, "W")
+    R, C = W.shape
+    G = C // group_size if group_size > 0 else 1
+    qweight = torch.empty((R, C * field_bits(bits) // 32), dtype=torch.int32, device=W.device)
+    scales = torch.empty((R, G), dtype=torch.float32, device=W.device)
+    zeros = torch.empty((R, G), dtype=torch.float32, device=W.device)
+    st = _lib.gptq_rtn_layer(W.data_ptr(), R, C, bits, group_size, int(bool(sym)), qweight.data_ptr(), scales.data_ptr(),
+                             zeros.data_ptr(), _stream_ptr(stream))
+    if st != OK:
+        raise GptqError(st, "gptq_rtn_layer")
+    return dict(qweight=qweight, scales=scales, zeros=zeros)

@@ -257,3 +257,30 @@ def test_solve_layer_from_host_buffers(B):
     check_quantize_outputs(gpu, ref, W16, 4, L.C, ref["H"])
     with pytest.raises(B.GptqError):
         B.gptq_solve_layer_host(Wh, Xh, 5, 0, False, 128, 0.01)      # unsupported bits
+
+
+@pytest.mark.parametrize("bits,group", [(4, 0), (3, 0), (3, 128), (2, 32), (4, 8), (4, 1024), (O.BITS_TERNARY, 8), (8, 64)])
+def test_rtn_layer_bit_exact_and_equals_solver_on_diagonal_hessian(B, bits, group):
+    """RTN entry point: codes, scales and zeros bit-exact against the oracle's RTN (both sides decide in
+    fp64 on fp32-rounded scales); and the solver with a diagonal H gives the same codes (Section 5, Baselines)."""
+    L = _layer(70, 2048, 64, cfg=4)
+    W16 = L.w()
+    W = torch.from_numpy(W16).cuda()
+    out = B.gptq_rtn_layer(W, bits, group, False)
+    torch.cuda.synchronize()
+    codes_ref, _ = O.rtn(W16, bits, group, False)
+    codes = O.unpack_codes(out["qweight"].cpu().numpy().view(np.uint32), bits, L.C)
+    assert np.array_equal(codes, codes_ref)
+    assert np.array_equal(O.pack_codes(codes, bits), out["qweight"].cpu().numpy().view(np.uint32))
+    g = group if group > 0 else L.C
+    for gi in range(0, L.C // g, max(1, (L.C // g) // 7)):
+        s, z = O.find_params(W16[:, gi * g:(gi + 1) * g].astype(np.float64), bits, False)
+        assert np.array_equal(out["scales"][:, gi].cpu().numpy().astype(np.float64), s)
+        assert np.array_equal(out["zeros"][:, gi].cpu().numpy().astype(np.float64), z)
+    if group == 0 or (group % 32 == 0) or group in (4, 8, 16):
+        d = np.exp(np.random.default_rng(3).normal(size=L.C)).astype(np.float32)
+        U, info = B.gptq_prepare_hinv(torch.diag(torch.from_numpy(d)).cuda(), 0.01)
+        blk = 128 if (group <= 0 or group % 128 == 0 or 128 % group == 0) else 32
+        q = B.gptq_quantize_layer(W, U, bits, group, False, blk)
+        torch.cuda.synchronize()
+        assert torch.equal(q["qweight"], out["qweight"])
