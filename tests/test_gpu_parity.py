@@ -126,6 +126,9 @@ CASES = [
     (64, 256, 4, 64, True, 64),        # symmetric grid
     (260, 2304, 4, 0, False, 128),     # several outer (lazy) blocks
     (130, 2176, 3, 128, False, 96),    # block that is not a power of two; ragged outer block
+    (64, 2048, O.BITS_TERNARY, 8, False, 128),   # the paper's ternary setting: group size 8
+    (64, 2048, 4, 1024, False, 128),             # group size 1024 (group spans eight blocks)
+    (64, 2048, 2, 32, False, 128),               # group size 32
 ]
 
 
