@@ -364,6 +364,52 @@ def run_e2e(args, wl, state, ws, device_value):
                 api="gptq_solve_layer_host (pinned host buffers; X streamed in 512 MiB chunks on a copy stream)")
 
 
+def run_inference(args, wl):
+    """Bandwidth of the inference-side kernels (packed-matrix x fp16-vector, whole-matrix dequantization) on the
+    workload's largest layer, quantized with the RTN entry point (the kernels' speed does not depend on the codes)."""
+    import torch
+    from paper_2210_17323_b200 import binding as B
+    from paper_2210_17323_b200.synth import device as D
+
+    torch.cuda.set_device(0)
+    L = max(wl.layers, key=lambda l: l.R * l.C)
+    W = D.fill_w(L)
+    peaks = _peaks()
+    rows = []
+    for g in wl.grids:
+        q = B.gptq_rtn_layer(W, g.bits, g.group_size, g.sym)
+        x = torch.randn(L.C, device="cuda").to(torch.float16)
+        y = torch.empty(L.R, dtype=torch.float32, device="cuda")
+        out = torch.empty((L.R, L.C), dtype=torch.float16, device="cuda")
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        res = {}
+        for name, fn, nbytes in (
+                ("matvec", lambda: B.gptq_matvec(q["qweight"], q["scales"], q["zeros"], x, L.C, g.bits, g.group_size, out=y),
+                 q["qweight"].numel() * 4 + q["scales"].numel() * 8 + L.C * 2 + L.R * 4),
+                ("dequantize", lambda: B.gptq_dequantize(q["qweight"], q["scales"], q["zeros"], L.C, g.bits, g.group_size, out=out),
+                 q["qweight"].numel() * 4 + q["scales"].numel() * 8 + L.R * L.C * 2)):
+            for _ in range(max(3, args.warmup)):
+                fn()
+            ts = []
+            for _ in range(max(5, args.steps)):
+                flush.zero_()                       # L2 flush between timed iterations
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            ms = statistics.median(ts)
+            res[name] = dict(ms=ms, gbs=nbytes / ms / 1e6, frac_of_hbm=nbytes / ms / 1e6 / peaks["hbm_gbs"], bytes=nbytes)
+        rows.append(dict(bits=g.bits, group_size=g.group_size, **res))
+    line = dict(metric="gptq_inference_kernel_bandwidth", unit="GB/s", value=rows[0]["matvec"]["gbs"], n_gpus=1,
+                higher_is_better=True, data="synthetic", dtype="packed codes -> f32 accumulate",
+                config=dict(workload=wl.name, layer=L.name, cache="256 MiB L2 flush between timed iterations"),
+                roofline=dict(kernel="gptq_matvec", bound="hbm", achieved=rows[0]["matvec"]["gbs"], peak=peaks["hbm_gbs"],
+                              unit="GB/s", frac=rows[0]["matvec"]["frac_of_hbm"], traffic=None,
+                              peak_source=f"STREAM-style copy, {peaks['source']}"),
+                kernels=rows)
+    print(json.dumps(line))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -374,6 +420,9 @@ def main():
     ap.add_argument("--no-graphs", action="store_true", help="issue every kernel launch from the host instead of replaying CUDA graphs")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mode", default="solver", choices=["solver", "inference"],
+                    help="solver: the layer-solver step (default, the headline metric); inference: bandwidth of the "
+                         "packed matvec / dequantize kernels")
     ap.add_argument("--layer", default=None, metavar="RxCxTOKENS",
                     help="profile one layer of this shape (grid, block and damp of --workload) instead of the "
                          "whole layer set -- a small case of the same kernels for profiler captures")
@@ -386,6 +435,8 @@ def main():
                          wl.grids, wl.block, wl.damp)
     if args.impl == "reference":
         return run_reference(args, wl)
+    if args.mode == "inference":
+        return run_inference(args, wl)
     return run_gpu(args, wl)
 
 

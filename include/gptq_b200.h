@@ -160,6 +160,23 @@ gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U, int R, int
 gptq_status_t gptq_rtn_layer(const void* W_fp16, int R, int C, int bits, int group_size, int sym,
                              uint32_t* qweight, float* scales, float* zeros, void* stream);
 
+/* ------------------------------------------------------------------ using the packed weights
+ * The two kernels the paper describes for running a quantized model (Section 5, "Practical
+ * Speedups"; appendix on kernels), reading the packed layout gptq_quantize_layer writes.
+ * Dequantized value: scales[r][gi] * (code - zeros[r][gi]), formed with one fp32 multiply.
+ * group_size as in gptq_quantize_layer (<= 0: per row); 4, 8, 16 or a multiple of 32.
+ *
+ * gptq_dequantize: the whole matrix back to fp16 (round-to-nearest-even of the fp32 product).
+ *   W_out_fp16 [R x C] half.
+ * gptq_matvec: y = W^ x for ONE fp16 vector x (batch-1 generation: "quantized-matrix
+ *   full-precision-vector product" with dequantization on the fly, never materialising W^).
+ *   x_fp16 [C] half, y [R] fp32; products and sums in fp32.  C <= 51200 (x is staged in
+ *   shared memory), else GPTQ_ERR_UNSUPPORTED. */
+gptq_status_t gptq_dequantize(const uint32_t* qweight, const float* scales, const float* zeros,
+                              int R, int C, int bits, int group_size, void* W_out_fp16, void* stream);
+gptq_status_t gptq_matvec(const uint32_t* qweight, const float* scales, const float* zeros,
+                          const void* x_fp16, int R, int C, int bits, int group_size, float* y, void* stream);
+
 /* ------------------------------------------------------------------ whole layer, host buffers
  * Stages 1-3 for one layer whose inputs and outputs live in HOST memory (Eq. 1's W and X in, the
  * packed W^ out): X is streamed to the device in token chunks of about 512 MiB, double-buffered on

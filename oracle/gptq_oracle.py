@@ -217,6 +217,27 @@ def unpack_codes(words: np.ndarray, bits: int, C: int) -> np.ndarray:
     return out
 
 
+# --------------------------------------------------------------------------- using the packed weights
+def dequantize(codes: np.ndarray, scales: np.ndarray, zeros: np.ndarray, to_fp16: bool = False) -> np.ndarray:
+    """W^ = scale * (code - zero) per row and group (Section 5: "FP16 scale and ... zero point per group").
+    to_fp16=False: the exact real-valued grid point in float64 (scales hold fp32 values).
+    to_fp16=True: the stored-model reading -- one fp32 multiply, then round-to-nearest-even to fp16."""
+    R, C = codes.shape
+    g = C // scales.shape[1]
+    s = np.repeat(scales, g, axis=1)
+    z = np.repeat(zeros, g, axis=1)
+    if not to_fp16:
+        return s.astype(np.float64) * (codes.astype(np.float64) - z.astype(np.float64))
+    d = (codes.astype(np.float32) - z.astype(np.float32)).astype(np.float32)
+    return (s.astype(np.float32) * d).astype(np.float32).astype(np.float16)
+
+
+def matvec(codes: np.ndarray, scales: np.ndarray, zeros: np.ndarray, x16: np.ndarray) -> np.ndarray:
+    """y = W^ x for one input vector (Section 5, Practical Speedups: quantized-matrix times
+    full-precision vector), in float64 on the exact grid values."""
+    return dequantize(codes, scales, zeros) @ np.asarray(x16, dtype=np.float64)
+
+
 # --------------------------------------------------------------------------- whole path
 def solve_layer(W16, Xt_bits, bits, group_size=0, sym=False, block=128, damp=0.01):
     """Stages 1-3 in sequence; returns the stage-3 dict plus H, U, lambda."""

@@ -61,6 +61,10 @@ def _load():
                                           c.c_void_p, c.c_size_t, c.c_void_p]
     lib.gptq_rtn_layer.restype = c.c_int
     lib.gptq_rtn_layer.argtypes = [c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+    lib.gptq_dequantize.restype = c.c_int
+    lib.gptq_dequantize.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p]
+    lib.gptq_matvec.restype = c.c_int
+    lib.gptq_matvec.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p]
     return lib
 
 
@@ -228,3 +232,28 @@ def gptq_rtn_layer(W, bits, group_size=0, sym=False, stream=None):
     if st != OK:
         raise GptqError(st, "gptq_rtn_layer")
     return dict(qweight=qweight, scales=scales, zeros=zeros)
+
+
+def gptq_dequantize(qweight, scales, zeros, C, bits, group_size=0, out=None, stream=None):
+    """Packed codes -> fp16 weights W^ = scales * (code - zeros)  [R x C]."""
+    _check(qweight, torch.int32, "qweight"); _check(scales, torch.float32, "scales"); _check(zeros, torch.float32, "zeros")
+    R = qweight.shape[0]
+    out = torch.empty((R, C), dtype=torch.float16, device=qweight.device) if out is None else out
+    st = _lib.gptq_dequantize(qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), R, C, bits, group_size,
+                              out.data_ptr(), _stream_ptr(stream))
+    if st != OK:
+        raise GptqError(st, "gptq_dequantize")
+    return out
+
+
+def gptq_matvec(qweight, scales, zeros, x, C, bits, group_size=0, out=None, stream=None):
+    """y = W^ x for one fp16 vector x of length C, dequantizing on the fly; y is fp32 [R]."""
+    _check(qweight, torch.int32, "qweight"); _check(scales, torch.float32, "scales"); _check(zeros, torch.float32, "zeros")
+    _check(x, torch.float16, "x")
+    R = qweight.shape[0]
+    out = torch.empty(R, dtype=torch.float32, device=qweight.device) if out is None else out
+    st = _lib.gptq_matvec(qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), x.data_ptr(), R, C, bits, group_size,
+                          out.data_ptr(), _stream_ptr(stream))
+    if st != OK:
+        raise GptqError(st, "gptq_matvec")
+    return out

@@ -5,5 +5,5 @@ EXPORTS = (
     "gptq_prepare_hinv_workspace_bytes", "gptq_prepare_hinv", "gptq_prepare_hinv_static",
     "gptq_quantize_workspace_bytes", "gptq_quantize_layer",
     "gptq_solve_layer_host_workspace_bytes", "gptq_solve_layer_host",
-    "gptq_rtn_layer",
+    "gptq_rtn_layer", "gptq_dequantize", "gptq_matvec",
 )

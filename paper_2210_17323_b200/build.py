@@ -21,7 +21,7 @@ NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 
-SOLVER_SOURCES = ["api.cu", "hessian.cu", "hessian_umma.cu", "hinv.cu", "quantize.cu", "solve_host.cu", "rtn.cu"]
+SOLVER_SOURCES = ["api.cu", "hessian.cu", "hessian_umma.cu", "hinv.cu", "quantize.cu", "solve_host.cu", "rtn.cu", "inference.cu"]
 
 
 def _newest(paths):

@@ -287,3 +287,27 @@ def test_rtn_layer_bit_exact_and_equals_solver_on_diagonal_hessian(B, bits, grou
         q = B.gptq_quantize_layer(W, U, bits, group, False, blk)
         torch.cuda.synchronize()
         assert torch.equal(q["qweight"], out["qweight"])
+
+
+@pytest.mark.parametrize("bits,group", [(4, 0), (3, 128), (2, 32), (O.BITS_TERNARY, 8), (8, 0), (3, 0)])
+def test_dequantize_and_matvec_match_oracle(B, bits, group):
+    """Inference-side kernels on the packed layout: dequantization bit-exact (fp32 product, RNE to fp16);
+    matvec within fp32 accumulation error of the fp64 definition."""
+    R, C = 300, 2048
+    L = _layer(R, C, 64, cfg=3)
+    W16 = L.w()
+    codes, _ = O.rtn(W16, bits, group, False)
+    g = group if group > 0 else C
+    scales = np.stack([O.find_params(W16[:, j:j + g].astype(np.float64), bits, False)[0] for j in range(0, C, g)], 1)
+    zeros = np.stack([O.find_params(W16[:, j:j + g].astype(np.float64), bits, False)[1] for j in range(0, C, g)], 1)
+    qw = torch.from_numpy(O.pack_codes(codes, bits).view(np.int32)).cuda()
+    sc = torch.from_numpy(scales.astype(np.float32)).cuda()
+    zr = torch.from_numpy(zeros.astype(np.float32)).cuda()
+    deq = B.gptq_dequantize(qw, sc, zr, C, bits, group)
+    ref16 = O.dequantize(codes, scales, zeros, to_fp16=True)
+    assert np.array_equal(deq.cpu().numpy().view(np.uint16), ref16.view(np.uint16))
+    x16 = (np.random.default_rng(9).normal(size=C)).astype(np.float16)
+    y = B.gptq_matvec(qw, sc, zr, torch.from_numpy(x16).cuda(), C, bits, group).cpu().numpy().astype(np.float64)
+    yref = O.matvec(codes, scales, zeros, x16)
+    bound = 4e-6 * (np.abs(O.dequantize(codes, scales, zeros)) @ np.abs(x16.astype(np.float64))) + 1e-12
+    assert (np.abs(y - yref) <= bound).all(), float(np.max(np.abs(y - yref) / bound))

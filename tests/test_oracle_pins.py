@@ -374,3 +374,23 @@ def test_rows_are_independent():
     part = O.quantize_layer(W[[2, 5, 11]], U, 3, 32, False, 32)
     assert np.array_equal(full["codes"][[2, 5, 11]], part["codes"])
     assert np.array_equal(full["scales"][[2, 5, 11]], part["scales"])
+
+
+# ------------------------------------------------------------------ dequantize / matvec (Section 5, Practical Speedups)
+def test_dequantize_and_matvec_definitions():
+    r = RNG(15)
+    W = (r.normal(size=(6, 64)) * 0.02).astype(np.float16)
+    U = np.eye(64)
+    out = O.quantize_layer(W, U, 3, 32, False, 32)
+    deq = O.dequantize(out["codes"], out["scales"], out["zeros"])
+    assert np.array_equal(deq, out["W_hat"])                    # the same grid points the solver produced
+    # hand check of one entry, and a level-by-level brute force of the whole matrix
+    s, z, q = out["scales"][2, 1], out["zeros"][2, 1], out["codes"][2, 40]
+    assert deq[2, 40] == s * (q - z)
+    x = (r.normal(size=64)).astype(np.float16)
+    y = O.matvec(out["codes"], out["scales"], out["zeros"], x)
+    want = [sum(float(deq[i, c]) * float(x[c]) for c in range(64)) for i in range(6)]
+    assert np.allclose(y, want, rtol=1e-12)
+    # fp16 storage reading: within half an fp16 ulp of the exact value
+    d16 = O.dequantize(out["codes"], out["scales"], out["zeros"], to_fp16=True)
+    assert d16.dtype == np.float16 and np.all(np.abs(d16.astype(np.float64) - deq) <= np.abs(deq) * 2.0 ** -11 + 1e-12)
