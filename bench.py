@@ -172,6 +172,7 @@ def run_gpu(args, wl):
 
     # each rank solves its own copy of the layer set (block index = rank -> its own seeds)
     layers = multi.rank_layers(wl.layers, rank)
+    overlap = not args.no_overlap
     state = []
     ws_bytes = 256
     for L in layers:
@@ -179,15 +180,37 @@ def run_gpu(args, wl):
                   H=torch.empty((L.C, L.C), dtype=torch.float32, device=dev),
                   U=torch.empty((L.C, L.C), dtype=torch.float32, device=dev),
                   info=torch.zeros(2, dtype=torch.int32, device=dev))
-        ws_bytes = max(ws_bytes, B.gptq_hessian_workspace_bytes(L.C, L.n_tokens), B.gptq_prepare_hinv_workspace_bytes(L.C),
-                       *[B.gptq_quantize_workspace_bytes(L.R, L.C, g.bits, g.group_size, wl.block) for g in wl.grids])
+        st["ws_bytes"] = max(256, B.gptq_hessian_workspace_bytes(L.C, L.n_tokens), B.gptq_prepare_hinv_workspace_bytes(L.C),
+                             *[B.gptq_quantize_workspace_bytes(L.R, L.C, g.bits, g.group_size, wl.block) for g in wl.grids])
+        ws_bytes = max(ws_bytes, st["ws_bytes"])
         state.append(st)
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    # Layers are independent problems.  Overlapped schedule (default): the Hessians run back to back on one
+    # stream, most expensive layer first; each layer's stages 2 and 3 follow on that layer's own stream as soon
+    # as its Hessian is done, so the latency-bound kernel chains of different layers fill the SMs together and
+    # run beside the next Hessians.  Every layer then needs its own workspace.  Sequential schedule
+    # (--no-overlap): one stream, one shared workspace, layer after layer.
+    if overlap:
+        for st in state:
+            st["ws"] = torch.empty(st["ws_bytes"], dtype=torch.uint8, device=dev)
+    else:
+        shared_ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        for st in state:
+            st["ws"] = shared_ws
+    order = sorted(range(len(state)), key=lambda i: -(state[i]["L"].C ** 2) * (state[i]["L"].n_tokens + state[i]["L"].C))
+    main = torch.cuda.Stream(device=dev)
+    chain_streams = [torch.cuda.Stream(device=dev) if overlap else main for _ in state]
     torch.cuda.synchronize()
 
-    stage_events = []                             # (stage, layer idx, start, end) of the timed steps
+    stage_events = []                             # (layer idx, events) of the timed steps
 
     graphs = []                                   # per layer: CUDA graphs of the three stages (launch-bound inner loops)
+
+    def stage_fns(st):
+        return ([("H", lambda: (st["H"].zero_(), B.gptq_hessian_accumulate(st["H"], st["X"], ws=st["ws"]))),
+                 ("U", lambda: B.gptq_prepare_hinv(st["H"], wl.damp, U=st["U"], ws=st["ws"], dev_info=st["info"]))] +
+                [(f"Q{gi}", (lambda gi=gi, g=g: st["out"].__setitem__(gi, B.gptq_quantize_layer(
+                    st["W"], st["U"], g.bits, g.group_size, g.sym, wl.block, ws=st["ws"]))))
+                 for gi, g in enumerate(wl.grids)])
 
     def run_stage(li, name, fn):
         if graphs:
@@ -196,30 +219,40 @@ def run_gpu(args, wl):
             fn()
 
     def step(record):
-        for li, st in enumerate(state):
+        done = []
+        for li in (order if overlap else range(len(state))):
+            st = state[li]
+            fns = stage_fns(st)
             ev = [torch.cuda.Event(enable_timing=True) for _ in range(4 + len(wl.grids))] if record else None
-            if record: ev[0].record()
-            run_stage(li, "H", lambda: (st["H"].zero_(), B.gptq_hessian_accumulate(st["H"], st["X"], ws=ws)))
-            if record: ev[1].record()
-            run_stage(li, "U", lambda: B.gptq_prepare_hinv(st["H"], wl.damp, U=st["U"], ws=ws, dev_info=st["info"]))
-            if record: ev[2].record()
-            for gi, g in enumerate(wl.grids):
-                run_stage(li, f"Q{gi}", lambda: st["out"].__setitem__(gi, B.gptq_quantize_layer(
-                    st["W"], st["U"], g.bits, g.group_size, g.sym, wl.block, ws=ws)))
-                if record: ev[3 + gi].record()
+            cs = chain_streams[li]
+            with torch.cuda.stream(main):
+                if record: ev[0].record(main)
+                run_stage(li, *fns[0])
+                if record:
+                    ev[1].record(main); h_done = ev[1]
+                else:
+                    h_done = torch.cuda.Event(); h_done.record(main)
+            with torch.cuda.stream(cs):
+                cs.wait_event(h_done)
+                if record: ev[2].record(cs)
+                run_stage(li, *fns[1])
+                if record: ev[3].record(cs)
+                for gi in range(len(wl.grids)):
+                    run_stage(li, *fns[2 + gi])
+                end = ev[4 + len(wl.grids) - 1] if record else torch.cuda.Event()
+                end.record(cs)
+            done.append(end)
             if record:
                 stage_events.append((li, ev))
+        for e in done:                            # the step ends when every layer's chain has ended
+            main.wait_event(e)
 
     def capture_graphs():
         """Every stage of every layer becomes one CUDA graph (same kernels, same order, same buffers): the
         ~2400 small launches of a step are then issued by the GPU front end instead of the host."""
         for li, st in enumerate(state):
             gs = {}
-            for name, fn in ([("H", lambda: (st["H"].zero_(), B.gptq_hessian_accumulate(st["H"], st["X"], ws=ws))),
-                              ("U", lambda: B.gptq_prepare_hinv(st["H"], wl.damp, U=st["U"], ws=ws, dev_info=st["info"]))] +
-                             [(f"Q{gi}", (lambda gi=gi, g=g: st["out"].__setitem__(gi, B.gptq_quantize_layer(
-                                 st["W"], st["U"], g.bits, g.group_size, g.sym, wl.block, ws=ws))))
-                              for gi, g in enumerate(wl.grids)]):
+            for name, fn in stage_fns(st):
                 cg = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(cg):
                     fn()
@@ -250,10 +283,10 @@ def run_gpu(args, wl):
         sampler.start()
     t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
     barrier()
-    t0.record()
+    t0.record(main)
     for _ in range(args.steps):
         step(True)
-    t1.record()
+    t1.record(main)
     barrier()
     launches = launches_per_step * args.steps     # kernels of this library in the timed region (replayed from graphs or host-issued)
     clocks = sampler.stop() if rank == 0 else None
@@ -270,14 +303,15 @@ def run_gpu(args, wl):
         L = state[li]["L"]
         d = per.setdefault(li, dict(layer=L.name, hessian_ms=0.0, hinv_ms=0.0, quantize_ms=0.0))
         d["hessian_ms"] += ev[0].elapsed_time(ev[1]) / args.steps
-        d["hinv_ms"] += ev[1].elapsed_time(ev[2]) / args.steps
-        d["quantize_ms"] += ev[2].elapsed_time(ev[2 + n_grids]) / args.steps
+        d["hinv_ms"] += ev[2].elapsed_time(ev[3]) / args.steps
+        d["quantize_ms"] += ev[3].elapsed_time(ev[3 + n_grids]) / args.steps
     peaks = _peaks()
     tot = {k: sum(d[k] for d in per.values()) for k in ("hessian_ms", "hinv_ms", "quantize_ms")}
     # roofline of the dominant kernel.  Hessian: algorithmic flops C (C + 1) m per launch (symmetric half).
     hess_flops = sum(L.C * (L.C + 1) * L.n_tokens for L in layers)
     upd_flops = sum(2 * L.R * (L.C * L.C - L.C * wl.block) / 2 * n_grids for L in layers)   # lazy updates, R (C^2 - C B)
-    if tot["hessian_ms"] >= tot["quantize_ms"]:
+    # the stage sums overlap one another in the overlapped schedule, so the dominant kernel is chosen against the step
+    if tot["hessian_ms"] >= tot["quantize_ms"] or tot["hessian_ms"] >= 0.3 * ms_per_step:
         ach = hess_flops / (tot["hessian_ms"] * 1e-3) / 1e12
         # DRAM traffic per launch: measured 4.6 x the algorithmic bytes (X once + H once) on the ncu capture of a
         # 4096-channel x 65536-token launch (profiles/); scaled to these launches by their algorithmic bytes
@@ -302,13 +336,16 @@ def run_gpu(args, wl):
                             block=wl.block, damp=wl.damp, calib_tokens=wl.layers[0].n_tokens,
                             cache="inputs larger than L2 (X >= 0.4 GB per layer); no flush needed",
                             launch="CUDA graphs, one per stage per layer" if graphs else "host-issued launches",
+                            schedule=("overlapped: Hessians back to back on one stream, each layer's stages 2-3 on its own "
+                                      "stream; stage_ms are in-context times that overlap one another") if overlap
+                            else "sequential: one stream, layer after layer",
                             parallelism=f"layer-set replica per GPU x{world}"),
                 sec_per_layer=ms_per_step * 1e-3 / len(layers),
                 stage_ms=tot, per_layer=list(per.values()),
                 roofline=roof, gpu_launches=int(launches), clocks=clocks)
 
     if rank == 0 and world == 1 and not args.no_e2e:
-        line["e2e"] = run_e2e(args, wl, state, ws, value)
+        line["e2e"] = run_e2e(args, wl, state, value)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, est, cores, sample = oracle_sample(wl)
         line["cpu_baseline"] = dict(value=v, unit=UNIT, cores=cores, kind="oracle", sample=sample)
@@ -319,7 +356,7 @@ def run_gpu(args, wl):
     return 0
 
 
-def run_e2e(args, wl, state, ws, device_value):
+def run_e2e(args, wl, state, device_value):
     """Same metric end to end through the C ABI's host-buffer call: every step, for every layer (and grid),
     gptq_solve_layer_host streams X and W from pinned HOST memory to the device (copies overlapped with the
     Hessian accumulation), solves, and copies codes, scales, zeros and loss back to the host."""
@@ -334,8 +371,7 @@ def run_e2e(args, wl, state, ws, device_value):
         for g in wl.grids:
             need = max(need, B.gptq_solve_layer_host_workspace_bytes(L.R, L.C, L.n_tokens, g.bits, g.group_size, wl.block))
     for st in state:                       # device copies are not needed any more: the call has its own staging
-        st["X"] = st["H"] = st["U"] = None
-    del ws
+        st["X"] = st["H"] = st["U"] = st["ws"] = None
     torch.cuda.empty_cache()
     dev_ws = torch.empty(need, dtype=torch.uint8, device="cuda")
     torch.cuda.synchronize()
@@ -418,6 +454,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-graphs", action="store_true", help="issue every kernel launch from the host instead of replaying CUDA graphs")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="run the layers one after another on one stream (per-stage times then do not overlap)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--mode", default="solver", choices=["solver", "inference"],

@@ -14,6 +14,8 @@
 #include "gemm_simt.cuh"
 #include "gemm_umma.cuh"
 
+#include <mutex>
+
 namespace gptq {
 namespace {
 
@@ -266,6 +268,39 @@ struct EpiStoreSplit {
   }
 };
 
+// Stores the result as fp32 into the factor AND as a tf32 hi / lo pair into its split copies (same
+// offsets, leading dimension ldf).  Single super-chunk contractions only, like EpiStoreSplit.
+struct EpiStoreF32AndSplit {
+  float* u; int64_t ldu; float* hi; float* lo; int64_t ldf; int M, N;
+  __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
+    if (row >= M || col0 >= N) return;
+    float4* d = reinterpret_cast<float4*>(u + (int64_t)row * ldu + col0);
+    float4* h = reinterpret_cast<float4*>(hi + (int64_t)row * ldf + col0);
+    float4* l = reinterpret_cast<float4*>(lo + (int64_t)row * ldf + col0);
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      float4 a, b;
+      tf32x3::split_tf32(v[4 * g], a.x, b.x); tf32x3::split_tf32(v[4 * g + 1], a.y, b.y);
+      tf32x3::split_tf32(v[4 * g + 2], a.z, b.z); tf32x3::split_tf32(v[4 * g + 3], a.w, b.w);
+      d[g] = make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+      h[g] = a; l[g] = b;
+    }
+  }
+};
+
+// dst{hi,lo}[r][c] = split(src[r][c]) for r < rows, c < w (w a multiple of 4; both 16-byte aligned).
+__global__ void split_rect_kernel(const float* __restrict__ src, int64_t ld_src, int rows, int w,
+                                  float* __restrict__ dhi, float* __restrict__ dlo, int64_t ld_dst) {
+  const int q = w / 4;
+  int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)rows * q) return;
+  const int r = (int)(idx / q), c = (int)(idx % q) * 4;
+  float4 v = *reinterpret_cast<const float4*>(src + (int64_t)r * ld_src + c), h, l;
+  tf32x3::split_tf32(v.x, h.x, l.x); tf32x3::split_tf32(v.y, h.y, l.y);
+  tf32x3::split_tf32(v.z, h.z, l.z); tf32x3::split_tf32(v.w, h.w, l.w);
+  *reinterpret_cast<float4*>(dhi + (int64_t)r * ld_dst + c) = h;
+  *reinterpret_cast<float4*>(dlo + (int64_t)r * ld_dst + c) = l;
+}
 // F{hi,lo}[r][c0 + c] = split(U[r][c0 + c]) for r < rows, c < w.
 __global__ void split_block_kernel(const float* __restrict__ U, int C, int c0, int w, int rows,
                                    float* __restrict__ Fhi, float* __restrict__ Flo) {
@@ -297,6 +332,7 @@ constexpr int kNB2 = 1024;   // outer panel width: contractions over everything 
 
 struct HinvWs {
   double* lam; float* Dinv; float* T; float* Fhi; float* Flo; float* VThi; float* VTlo; float* TThi; float* TTlo;
+  float* Vhi[2]; float* Vlo[2]; float* TAhi; float* TAlo;
   size_t bytes;
 };
 HinvWs carve_hinv(void* ws, int C) {
@@ -312,6 +348,12 @@ HinvWs carve_hinv(void* ws, int C) {
   o.VTlo = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);
   o.TThi = w.take<float>(outer ? (size_t)kNB2 * C : 0);           // (U~[0:j0, J] V_JJ)^T
   o.TTlo = w.take<float>(outer ? (size_t)kNB2 * C : 0);
+  for (int i = 0; i < 2; ++i) {                                   // inverse of an outer diagonal block, two in flight
+    o.Vhi[i] = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);
+    o.Vlo[i] = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);
+  }
+  o.TAhi = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);        // split copy of the row block above a diagonal block
+  o.TAlo = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);
   o.bytes = w.off;
   return o;
 }
@@ -353,6 +395,58 @@ extern "C" size_t gptq_prepare_hinv_workspace_bytes(int C) {
   return carve_hinv(nullptr, C).bytes;
 }
 
+// ---- second stream and events for the look-ahead schedule -----------------------------------------
+// Phase 1 is issued on two streams: the caller's stream carries the dependency chain (diagonal blocks),
+// an internal stream carries the wide contractions that only later panels wait for.  The internal
+// stream and the events are created once per device, on the first call for that device, and never
+// destroyed; they hold no device memory.  Both streams are joined before the call returns, so the
+// caller sees ordinary stream semantics (the call is also capturable into a CUDA graph, where the
+// two streams become two branches).
+namespace gptq {
+namespace {
+constexpr int kMaxOuter = 64;          // C <= 65536
+struct HinvAsync {
+  cudaStream_t bulk = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+  cudaEvent_t c3[kMaxOuter], c4[kMaxOuter], b1[kMaxOuter], b2[kMaxOuter];
+  bool ready = false;
+};
+constexpr int kMaxAsyncDevices = 64;
+HinvAsync g_async[kMaxAsyncDevices];
+std::mutex g_async_mutex;
+
+gptq_status_t get_async(HinvAsync** out) {
+  int dev = -1;
+  GPTQ_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxAsyncDevices) return GPTQ_ERR_UNSUPPORTED;
+  HinvAsync& a = g_async[dev];
+  if (!a.ready) {
+    GPTQ_CUDA_TRY(cudaStreamCreateWithFlags(&a.bulk, cudaStreamNonBlocking));
+    GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&a.fork, cudaEventDisableTiming));
+    GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&a.join, cudaEventDisableTiming));
+    for (int i = 0; i < kMaxOuter; ++i) {
+      GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&a.c3[i], cudaEventDisableTiming));
+      GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&a.c4[i], cudaEventDisableTiming));
+      GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&a.b1[i], cudaEventDisableTiming));
+      GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&a.b2[i], cudaEventDisableTiming));
+    }
+    a.ready = true;
+  }
+  *out = &a;
+  return GPTQ_OK;
+}
+
+gptq_status_t launch_split_rect(const float* src, int64_t ld_src, int rows, int w, float* dhi, float* dlo,
+                                int64_t ld_dst, cudaStream_t s) {
+  if (rows <= 0 || w <= 0) return GPTQ_OK;
+  const int64_t total = (int64_t)rows * (w / 4);
+  split_rect_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(src, ld_src, rows, w, dhi, dlo, ld_dst);
+  GPTQ_LAUNCH_CHECK();
+  return GPTQ_OK;
+}
+}  // namespace
+}  // namespace gptq
+
 extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, float* U,
                                            void* ws, size_t ws_bytes, int* dev_info, void* stream) {
   using namespace gptq;
@@ -362,6 +456,19 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   HinvWs w = carve_hinv(ws, C);
   gptq_status_t st;
+  const bool outer = C > kNB2;
+  const int n_outer = ceil_div(C, kNB2);
+  if (n_outer > kMaxOuter) return GPTQ_ERR_UNSUPPORTED;
+  const int reserve = 16;   // SMs the wide stream's contractions leave free for the chain stream's kernels
+
+  // enqueueing is serialised per process: the events below are shared by all calls on a device
+  std::lock_guard<std::mutex> lock(g_async_mutex);
+  HinvAsync* as = nullptr;
+  cudaStream_t sb = s;
+  if (outer) {
+    if ((st = get_async(&as)) != GPTQ_OK) return st;
+    sb = as->bulk;
+  }
 
   GPTQ_CUDA_TRY(cudaMemsetAsync(dev_info, 0, 2 * sizeof(int), s));
   lambda_kernel<<<1, 1024, 0, s>>>(H, C, damp, w.lam);
@@ -371,69 +478,120 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
     init_upper_damped_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(H, U, C, w.lam);
     GPTQ_LAUNCH_CHECK();
   }
-  const bool outer = C > kNB2;
-  const int n_outer = ceil_div(C, kNB2);
+  if (outer) {
+    GPTQ_CUDA_TRY(cudaEventRecord(as->fork, s));
+    GPTQ_CUDA_TRY(cudaStreamWaitEvent(sb, as->fork, 0));
+  }
 
-  // Phase 1: backwards blocked Cholesky, H~ = U~ U~^T, in place in U's upper triangle.  Outer panels
-  // of kNB2 columns are brought up to date in one contraction over all later columns (left-looking),
-  // then factored with 128-wide steps whose updates stay inside the panel.
+  // Phase 1: backwards blocked Cholesky H~ = U~ U~^T in U's upper triangle, outer panels of kNB2 columns
+  // from the last to the first, left-looking: a panel receives the contributions of all later columns in
+  // one contraction over the tf32 hi / lo copies F of the finished factor.  Per panel J (rows j0..rows_p
+  // are its diagonal block D, "row block J-1" are the kNB2 rows above D):
+  //   chain stream                                         wide stream
+  //   C1  D -= F[J rows, later] F[J rows, later]^T         B1  A[0:j0, J] -= F[0:j0, later] F[J rows, later]^T
+  //   C2  factor D (128-wide steps inside D)               B2  U~[0:j0-kNB2, J] = A[..] V^T -> U and F   (after C3)
+  //   C3  V = D^-1 in place (final U block), split copy
+  //   C4  U~[row block J-1, J] = A[..] V^T -> U and F      (after B1)
+  // C1 of panel J needs row block J of every later panel: panel J+1's comes from its C4 (same stream),
+  // the others from B2 of panels >= J+2, which had the whole chain of panel J+1 to finish.
   for (int J = n_outer - 1; J >= 0; --J) {
     const int j0 = J * kNB2, wj = (C - j0 < kNB2) ? C - j0 : kNB2, rows_p = j0 + wj;
-    if (rows_p < C) {
-      // A[0:rows_p, J] -= U~[0:rows_p, later] * U~[J rows, later]^T   (upper part)
-      const int K = C - rows_p;
-      tf32x3::Operand A{w.Fhi + rows_p, w.Flo + rows_p, rows_p, K, C};
-      tf32x3::Operand B{w.Fhi + (int64_t)j0 * C + rows_p, w.Flo + (int64_t)j0 * C + rows_p, wj, K, C};
-      st = tf32x3::launch<false, false>(A, B, rows_p, wj, EpiSubUpperRed{U, C, j0, rows_p, wj}, dev_info, s);
+    const int K = C - rows_p;                       // later columns
+    float* D = U + (int64_t)j0 * C + j0;
+    if (K > 0) {
+      if (J + 2 < n_outer) GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, as->b2[J + 2], 0));
+      // C1
+      tf32x3::Operand A{w.Fhi + (int64_t)j0 * C + rows_p, w.Flo + (int64_t)j0 * C + rows_p, wj, K, C};
+      st = tf32x3::launch<false, true>(A, A, wj, wj, EpiSubUpperRed{D, C, 0, wj, wj}, dev_info, s);
       if (st != GPTQ_OK) return st;
+      if (j0 > 0) {
+        // B1
+        GPTQ_CUDA_TRY(cudaStreamWaitEvent(sb, as->c4[J + 1], 0));
+        tf32x3::Operand A1{w.Fhi + rows_p, w.Flo + rows_p, j0, K, C};
+        st = tf32x3::launch<false, false>(A1, A, j0, wj, EpiSubRed{U + j0, C, j0, wj}, dev_info, sb, reserve);
+        if (st != GPTQ_OK) return st;
+        GPTQ_CUDA_TRY(cudaEventRecord(as->b1[J], sb));
+      }
     }
+    // C2: 128-wide steps inside D (rows j0 .. k0 of the panel only)
+    float* Ub = U + (int64_t)j0 * C;                // first row of D
     for (int k0 = j0 + (wj - 1) / kNB * kNB; k0 >= j0; k0 -= kNB) {
       const int nb = (rows_p - k0 < kNB) ? rows_p - k0 : kNB;
       float* Dk = w.Dinv + (size_t)(k0 / kNB) * kNB * kNB;
       rchol_diag_kernel<<<1, kDiagThreads, 0, s>>>(U, C, k0, nb, Dk, dev_info);
       GPTQ_LAUNCH_CHECK();
-      if (k0 == 0) break;
-      // panel: U~[0:k0, blk] = A[0:k0, blk] * T_kk^-T      (out[m][n] = sum_k A[m][k0+k] V[n][k])
-      GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, 1, RowMajorF32{U + k0, C}, RowMajorF32T{Dk, kNB},
-                                     FullRange{nb}, StoreF32{U + k0, C}, s));
-      // trailing, inside the outer panel: A[0:k0, j0:k0] -= P P[j0:k0]^T on upper tiles  (P = U~[0:k0, blk])
-      if (k0 > j0)
-        GPTQ_CUDA_TRY(launch_gemm_simt(k0, k0 - j0, 1, RowMajorF32{U + k0, C}, RowMajorF32T{U + (int64_t)j0 * C + k0, C},
-                                       UpperTilesOfs{nb, j0}, SubUpperOfsF32{U, C, j0}, s));
+      const int m = k0 - j0;                        // rows of D above this block
+      if (m == 0) break;
+      // P = A[j0:k0, blk] * T_kk^-T      (out[m][n] = sum_k A[m][k0+k] V[n][k])
+      GPTQ_CUDA_TRY(launch_gemm_simt(m, nb, 1, RowMajorF32{Ub + k0, C}, RowMajorF32T{Dk, kNB},
+                                     FullRange{nb}, StoreF32{Ub + k0, C}, s));
+      // A[j0:k0, j0:k0] -= P P^T on upper tiles
+      GPTQ_CUDA_TRY(launch_gemm_simt(m, m, 1, RowMajorF32{Ub + k0, C}, RowMajorF32T{Ub + k0, C},
+                                     UpperTilesOfs{nb, 0}, SubUpperOfsF32{Ub + j0, C, 0}, s));
     }
-    if (outer && J > 0) {
-      int64_t total = (int64_t)rows_p * (wj / 4);
-      split_block_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(U, C, j0, wj, rows_p, w.Fhi, w.Flo);
-      GPTQ_LAUNCH_CHECK();
-    }
-  }
-  // Phase 2: U = U~^-1, outer panel by outer panel, in place.
-  for (int J = 0; J < n_outer; ++J) {
-    const int j0 = J * kNB2, wj = (C - j0 < kNB2) ? C - j0 : kNB2, rows_p = j0 + wj;
-    // (a) diagonal block: V_JJ = U~_JJ^-1
-    st = invert_upper_block(U + (int64_t)j0 * C + j0, C, wj, w.Dinv + (size_t)(j0 / kNB) * kNB * kNB, w.T, s);
+    // C3: V = D^-1 in place (this IS the diagonal block of the final U)
+    st = invert_upper_block(D, C, wj, w.Dinv + (size_t)(j0 / kNB) * kNB * kNB, w.T, s);
     if (st != GPTQ_OK) return st;
-    if (j0 > 0) {
-      // (b) rows above it: U[0:j0, J] = -U[0:j0, 0:j0] * (U~[0:j0, J] * V_JJ)
-      dim3 grid(wj / 32, wj / 32), blk(32, 32);
-      split_diag_t_kernel<<<grid, blk, 0, s>>>(U, C, j0, w.VThi, w.VTlo, kNB2);
-      GPTQ_LAUNCH_CHECK();
-      // TT = V_JJ^T * U~[0:j0, J]^T   (wj x j0), written as a hi / lo pair (single super-chunk: K = wj)
-      {
-        tf32x3::Operand A{w.VThi, w.VTlo, wj, wj, kNB2};
-        tf32x3::Operand B{w.Fhi + j0, w.Flo + j0, j0, wj, C};
-        st = tf32x3::launch<false, false>(A, B, wj, j0, EpiStoreSplit{w.TThi, w.TTlo, C, wj, j0}, dev_info, s);
-        if (st != GPTQ_OK) return st;
-      }
-      GPTQ_CUDA_TRY(cudaMemset2DAsync(U + j0, (size_t)C * 4, 0, (size_t)wj * 4, j0, s));
-      {
-        tf32x3::Operand A{w.Fhi, w.Flo, j0, j0, C};
-        tf32x3::Operand B{w.TThi, w.TTlo, wj, j0, C};
-        st = tf32x3::launch<true, false>(A, B, j0, wj, EpiSubRed{U + j0, C, j0, wj}, dev_info, s);
-        if (st != GPTQ_OK) return st;
-      }
+    if (!outer || j0 == 0) continue;
+    float* Vhi = w.Vhi[J & 1]; float* Vlo = w.Vlo[J & 1];
+    if ((st = launch_split_rect(D, C, wj, wj, Vhi, Vlo, kNB2, s)) != GPTQ_OK) return st;
+    GPTQ_CUDA_TRY(cudaEventRecord(as->c3[J], s));
+    tf32x3::Operand V{Vhi, Vlo, wj, wj, kNB2};
+    const int r1 = j0 - kNB2;                       // first row of row block J-1
+    // B2 (rows above row block J-1)
+    if (r1 > 0) {
+      GPTQ_CUDA_TRY(cudaStreamWaitEvent(sb, as->c3[J], 0));
+      if ((st = launch_split_rect(U + j0, C, r1, wj, w.TThi, w.TTlo, kNB2, sb)) != GPTQ_OK) return st;
+      tf32x3::Operand A2{w.TThi, w.TTlo, r1, wj, kNB2};
+      st = tf32x3::launch<false, false>(A2, V, r1, wj,
+                                        EpiStoreF32AndSplit{U + j0, C, w.Fhi + j0, w.Flo + j0, C, r1, wj}, dev_info, sb, reserve);
+      if (st != GPTQ_OK) return st;
     }
-    if (outer && J + 1 < n_outer) {
+    GPTQ_CUDA_TRY(cudaEventRecord(as->b2[J], sb));
+    // C4 (row block J-1)
+    if (K > 0) GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, as->b1[J], 0));
+    {
+      const int64_t o = (int64_t)r1 * C + j0;
+      if ((st = launch_split_rect(U + o, C, kNB2, wj, w.TAhi, w.TAlo, kNB2, s)) != GPTQ_OK) return st;
+      tf32x3::Operand A4{w.TAhi, w.TAlo, kNB2, wj, kNB2};
+      st = tf32x3::launch<false, false>(A4, V, kNB2, wj,
+                                        EpiStoreF32AndSplit{U + o, C, w.Fhi + o, w.Flo + o, C, kNB2, wj}, dev_info, s);
+      if (st != GPTQ_OK) return st;
+    }
+    GPTQ_CUDA_TRY(cudaEventRecord(as->c4[J], s));
+  }
+  if (outer) {
+    GPTQ_CUDA_TRY(cudaEventRecord(as->join, sb));
+    GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, as->join, 0));
+  }
+
+  // Phase 2: U = U~^-1, outer panel by outer panel, in place.  The diagonal blocks are already inverted;
+  // rows above them: U[0:j0, J] = -U[0:j0, 0:j0] * (U~[0:j0, J] * V_JJ).
+  for (int J = 1; J < n_outer; ++J) {
+    const int j0 = J * kNB2, wj = (C - j0 < kNB2) ? C - j0 : kNB2, rows_p = j0 + wj;
+    if (J == 1) {                                   // split copy of the first panel of the inverse
+      int64_t total = (int64_t)kNB2 * (kNB2 / 4);
+      split_block_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(U, C, 0, kNB2, kNB2, w.Fhi, w.Flo);
+      GPTQ_LAUNCH_CHECK();
+    }
+    dim3 grid(ceil_div(wj, 32), ceil_div(wj, 32)), blk(32, 32);
+    split_diag_t_kernel<<<grid, blk, 0, s>>>(U, C, j0, w.VThi, w.VTlo, kNB2);
+    GPTQ_LAUNCH_CHECK();
+    // TT = V_JJ^T * U~[0:j0, J]^T   (wj x j0), written as a hi / lo pair (single super-chunk: K = wj)
+    {
+      tf32x3::Operand A{w.VThi, w.VTlo, wj, wj, kNB2};
+      tf32x3::Operand B{w.Fhi + j0, w.Flo + j0, j0, wj, C};
+      st = tf32x3::launch<false, false>(A, B, wj, j0, EpiStoreSplit{w.TThi, w.TTlo, C, wj, j0}, dev_info, s);
+      if (st != GPTQ_OK) return st;
+    }
+    GPTQ_CUDA_TRY(cudaMemset2DAsync(U + j0, (size_t)C * 4, 0, (size_t)wj * 4, j0, s));
+    {
+      tf32x3::Operand A{w.Fhi, w.Flo, j0, j0, C};
+      tf32x3::Operand B{w.TThi, w.TTlo, wj, j0, C};
+      st = tf32x3::launch<true, false>(A, B, j0, wj, EpiSubRed{U + j0, C, j0, wj}, dev_info, s);
+      if (st != GPTQ_OK) return st;
+    }
+    if (J + 1 < n_outer) {
       int64_t total = (int64_t)rows_p * (wj / 4);
       split_block_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(U, C, j0, wj, rows_p, w.Fhi, w.Flo);
       GPTQ_LAUNCH_CHECK();

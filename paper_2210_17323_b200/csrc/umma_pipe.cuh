@@ -149,11 +149,12 @@ umma_pipe_kernel(const __grid_constant__ typename Traits::Maps maps, const int n
 
 template <class Traits, class ItemF, class EpiF>
 gptq_status_t launch_pipe(const typename Traits::Maps& maps, int64_t n_items, ItemF itemf, EpiF epi, int* dev_info,
-                          cudaStream_t stream) {
+                          cudaStream_t stream, int reserve_sms = 0) {
   if (n_items <= 0) return GPTQ_OK;
   if (n_items > 0x7FFFFFFF) return GPTQ_ERR_UNSUPPORTED;
   constexpr size_t smem = (size_t)Traits::STAGES * Traits::STAGE_BYTES + 1024 + 256;
-  const int sms = device_sm_count();
+  int sms = device_sm_count() - reserve_sms;      // SMs left free for kernels running beside this one
+  if (sms < 1) sms = 1;
   auto kern = umma_pipe_kernel<Traits, ItemF, EpiF>;
   GPTQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   kern<<<(int)(n_items < sms ? n_items : sms), kThreads, smem, stream>>>(maps, (int)n_items, itemf, epi, dev_info);
