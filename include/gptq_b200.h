@@ -87,7 +87,14 @@ gptq_status_t gptq_hessian_accumulate(float* H, const void* X_bf16, int64_t n_to
  *            non-positive pivot.  On NOT_PD the contents of U are unspecified
  *            but finite operations continue (no trap, no hang).
  * Computed as the inverse of the upper factor of H~ = U~ U~^T, which equals
- * Cholesky(H~^-1)^T by uniqueness of the Cholesky factor. */
+ * Cholesky(H~^-1)^T by uniqueness of the Cholesky factor.
+ * Streams: for C > 1024 part of the work is enqueued on a second, internal stream (created once
+ * per device on the first such call, never destroyed, holds no device memory) that forks from
+ * `stream` after the call's first kernels and joins it again before the call returns, so the
+ * caller sees ordinary single-stream ordering and the call can be captured into a CUDA graph
+ * (make the first call for a device outside any capture).  The host-side enqueueing of
+ * concurrent calls is serialised inside the library; calls on different streams still overlap on
+ * the device as far as their workspaces are distinct. */
 size_t gptq_prepare_hinv_workspace_bytes(int C);
 gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, float* U,
                                 void* ws, size_t ws_bytes, int* dev_info, void* stream);
