@@ -189,6 +189,7 @@ def run_gpu(args, wl):
     # as its Hessian is done, so the latency-bound kernel chains of different layers fill the SMs together and
     # run beside the next Hessians.  Every layer then needs its own workspace.  Sequential schedule
     # (--no-overlap): one stream, one shared workspace, layer after layer.
+    shared_ws = None
     if overlap:
         for st in state:
             st["ws"] = torch.empty(st["ws_bytes"], dtype=torch.uint8, device=dev)
@@ -345,6 +346,8 @@ def run_gpu(args, wl):
                 roofline=roof, gpu_launches=int(launches), clocks=clocks)
 
     if rank == 0 and world == 1 and not args.no_e2e:
+        shared_ws = None                          # the host-buffer call brings its own device workspace
+        graphs.clear()
         line["e2e"] = run_e2e(args, wl, state, value)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, est, cores, sample = oracle_sample(wl)
