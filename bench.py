@@ -347,7 +347,6 @@ def run_gpu(args, wl):
 
     if rank == 0 and world == 1 and not args.no_e2e:
         shared_ws = None                          # the host-buffer call brings its own device workspace
-        graphs.clear()
         line["e2e"] = run_e2e(args, wl, state, value)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, est, cores, sample = oracle_sample(wl)
