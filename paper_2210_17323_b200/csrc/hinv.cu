@@ -12,6 +12,7 @@
 // of the factor that are written as each panel is finalised.
 #include "common.cuh"
 #include "gemm_simt.cuh"
+#include "gemm_small.cuh"
 #include "gemm_umma.cuh"
 
 #include <mutex>
@@ -406,8 +407,9 @@ namespace gptq {
 namespace {
 constexpr int kMaxOuter = 64;          // C <= 65536
 struct HinvAsync {
-  cudaStream_t bulk = nullptr;
-  cudaEvent_t fork = nullptr, join = nullptr;
+  cudaStream_t bulk = nullptr, side = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr, side_done = nullptr;
+  cudaEvent_t step[8];
   cudaEvent_t c3[kMaxOuter], c4[kMaxOuter], b1[kMaxOuter], b2[kMaxOuter];
   bool ready = false;
 };
@@ -422,6 +424,9 @@ gptq_status_t get_async(HinvAsync** out) {
   HinvAsync& a = g_async[dev];
   if (!a.ready) {
     GPTQ_CUDA_TRY(cudaStreamCreateWithFlags(&a.bulk, cudaStreamNonBlocking));
+    GPTQ_CUDA_TRY(cudaStreamCreateWithFlags(&a.side, cudaStreamNonBlocking));
+    GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&a.side_done, cudaEventDisableTiming));
+    for (int i = 0; i < 8; ++i) GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&a.step[i], cudaEventDisableTiming));
     GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&a.fork, cudaEventDisableTiming));
     GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&a.join, cudaEventDisableTiming));
     for (int i = 0; i < kMaxOuter; ++i) {
@@ -464,10 +469,10 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
   // enqueueing is serialised per process: the events below are shared by all calls on a device
   std::lock_guard<std::mutex> lock(g_async_mutex);
   HinvAsync* as = nullptr;
-  cudaStream_t sb = s;
+  cudaStream_t sb = s, ss = s;                      // a single panel (C <= 1024) stays on the caller's stream
   if (outer) {
     if ((st = get_async(&as)) != GPTQ_OK) return st;
-    sb = as->bulk;
+    sb = as->bulk; ss = as->side;
   }
 
   GPTQ_CUDA_TRY(cudaMemsetAsync(dev_info, 0, 2 * sizeof(int), s));
@@ -481,6 +486,7 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
   if (outer) {
     GPTQ_CUDA_TRY(cudaEventRecord(as->fork, s));
     GPTQ_CUDA_TRY(cudaStreamWaitEvent(sb, as->fork, 0));
+    GPTQ_CUDA_TRY(cudaStreamWaitEvent(ss, as->fork, 0));
   }
 
   // Phase 1: backwards blocked Cholesky H~ = U~ U~^T in U's upper triangle, outer panels of kNB2 columns
@@ -513,25 +519,44 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
         GPTQ_CUDA_TRY(cudaEventRecord(as->b1[J], sb));
       }
     }
-    // C2: 128-wide steps inside D (rows j0 .. k0 of the panel only)
+    // C2: 128-wide steps inside D (rows j0 .. k0 of the panel only).  C3 runs beside it on a side stream:
+    // as soon as block k is factored, row block k of V = D^-1 follows from the rows below it,
+    //   V[k, after] = -V_kk (U~[k, after] V[after, after]),
+    // in place (row block k of the factor is not read again by the factorisation).
     float* Ub = U + (int64_t)j0 * C;                // first row of D
+    const int ldt = wj;                             // leading dimension of the side stream's 128 x rem temporary
     for (int k0 = j0 + (wj - 1) / kNB * kNB; k0 >= j0; k0 -= kNB) {
       const int nb = (rows_p - k0 < kNB) ? rows_p - k0 : kNB;
       float* Dk = w.Dinv + (size_t)(k0 / kNB) * kNB * kNB;
       rchol_diag_kernel<<<1, kDiagThreads, 0, s>>>(U, C, k0, nb, Dk, dev_info);
       GPTQ_LAUNCH_CHECK();
+      if (outer) {
+        cudaEvent_t ev = as->step[(k0 - j0) / kNB];
+        GPTQ_CUDA_TRY(cudaEventRecord(ev, s));
+        GPTQ_CUDA_TRY(cudaStreamWaitEvent(ss, ev, 0));
+      }
+      const int after = k0 + nb, rem = rows_p - after;
+      if (rem > 0) {
+        float* Vaa = U + (int64_t)after * C + after;
+        float* Rk = U + (int64_t)k0 * C + after;    // row block k, columns after it
+        GPTQ_CUDA_TRY((small::launch<64, false>(Rk, C, Vaa, C, nb, rem, small::UpperRightFactor<64>{rem},
+                                                StoreF32{w.T, ldt}, ss)));
+        GPTQ_CUDA_TRY((small::launch<64, false>(Dk, kNB, w.T, ldt, nb, rem, small::AllK{nb}, StoreNegF32{Rk, C}, ss)));
+      }
+      store_diag_block_kernel<<<8, 256, 0, ss>>>(U, C, k0, nb, Dk);
+      GPTQ_LAUNCH_CHECK();
       const int m = k0 - j0;                        // rows of D above this block
       if (m == 0) break;
-      // P = A[j0:k0, blk] * T_kk^-T      (out[m][n] = sum_k A[m][k0+k] V[n][k])
-      GPTQ_CUDA_TRY(launch_gemm_simt(m, nb, 1, RowMajorF32{Ub + k0, C}, RowMajorF32T{Dk, kNB},
-                                     FullRange{nb}, StoreF32{Ub + k0, C}, s));
+      // P = A[j0:k0, blk] * T_kk^-T, in place (one tile spans the block's columns)
+      GPTQ_CUDA_TRY((small::launch<128, true>(Ub + k0, C, Dk, kNB, m, nb, small::AllK{nb}, StoreF32{Ub + k0, C}, s)));
       // A[j0:k0, j0:k0] -= P P^T on upper tiles
-      GPTQ_CUDA_TRY(launch_gemm_simt(m, m, 1, RowMajorF32{Ub + k0, C}, RowMajorF32T{Ub + k0, C},
-                                     UpperTilesOfs{nb, 0}, SubUpperOfsF32{Ub + j0, C, 0}, s));
+      GPTQ_CUDA_TRY((small::launch<64, true>(Ub + k0, C, Ub + k0, C, m, m, small::UpperTiles<64>{nb},
+                                             SubUpperOfsF32{Ub + j0, C, 0}, s)));
     }
-    // C3: V = D^-1 in place (this IS the diagonal block of the final U)
-    st = invert_upper_block(D, C, wj, w.Dinv + (size_t)(j0 / kNB) * kNB * kNB, w.T, s);
-    if (st != GPTQ_OK) return st;
+    if (outer) {
+      GPTQ_CUDA_TRY(cudaEventRecord(as->side_done, ss));
+      GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, as->side_done, 0));
+    }
     if (!outer || j0 == 0) continue;
     float* Vhi = w.Vhi[J & 1]; float* Vlo = w.Vlo[J & 1];
     if ((st = launch_split_rect(D, C, wj, wj, Vhi, Vlo, kNB2, s)) != GPTQ_OK) return st;
