@@ -88,9 +88,9 @@ gptq_status_t gptq_hessian_accumulate(float* H, const void* X_bf16, int64_t n_to
  *            but finite operations continue (no trap, no hang).
  * Computed as the inverse of the upper factor of H~ = U~ U~^T, which equals
  * Cholesky(H~^-1)^T by uniqueness of the Cholesky factor.
- * Streams: for C > 1024 part of the work is enqueued on a second, internal stream (created once
- * per device on the first such call, never destroyed, holds no device memory) that forks from
- * `stream` after the call's first kernels and joins it again before the call returns, so the
+ * Streams: for C > 1024 part of the work is enqueued on two internal streams (created once
+ * per device on the first such call, never destroyed, they hold no device memory) that fork from
+ * `stream` after the call's first kernels and join it again before the call returns, so the
  * caller sees ordinary single-stream ordering and the call can be captured into a CUDA graph
  * (make the first call for a device outside any capture).  The host-side enqueueing of
  * concurrent calls is serialised inside the library; calls on different streams still overlap on
