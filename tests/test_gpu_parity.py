@@ -289,11 +289,15 @@ def test_rtn_layer_bit_exact_and_equals_solver_on_diagonal_hessian(B, bits, grou
         assert torch.equal(q["qweight"], out["qweight"])
 
 
-@pytest.mark.parametrize("bits,group", [(4, 0), (3, 128), (2, 32), (O.BITS_TERNARY, 8), (8, 0), (3, 0)])
-def test_dequantize_and_matvec_match_oracle(B, bits, group):
+@pytest.mark.parametrize("bits,group,C", [(4, 0, 2048), (3, 128, 2048), (2, 32, 2048), (O.BITS_TERNARY, 8, 2048), (8, 0, 2048),
+                                          (3, 0, 2048), (2, 128, 2048), (4, 128, 4096), (4, 1024, 2048), (O.BITS_TERNARY, 0, 2080),
+                                          (8, 128, 1024), (3, 0, 2144), (4, 0, 96), (3, 384, 768)])
+def test_dequantize_and_matvec_match_oracle(B, bits, group, C):
     """Inference-side kernels on the packed layout: dequantization bit-exact (fp32 product, RNE to fp16);
-    matvec within fp32 accumulation error of the fp64 definition."""
-    R, C = 300, 2048
+    matvec within fp32 accumulation error of the fp64 definition.  Per-row grids and groups that are multiples
+    of 128 take the tensor-core kernel (ragged last row task, C not a multiple of 128 included), the others the
+    CUDA-core kernel."""
+    R = 300
     L = _layer(R, C, 64, cfg=3)
     W16 = L.w()
     codes, _ = O.rtn(W16, bits, group, False)
