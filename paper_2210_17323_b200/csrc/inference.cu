@@ -117,10 +117,8 @@ matvec_kernel(const uint32_t* __restrict__ qweight, const float* __restrict__ sc
 // ---- y = dequant(Q) x on the warp-level tensor path (mma.sync m16n8k16, f16 x f16 -> f32) ---------
 // For per-row grids and group sizes that are multiples of 128.  The CUDA-core kernel above spends about
 // four instructions per weight (extract, convert, multiply-add), which bounds it well below the HBM rate;
-// here two codes become one half2 register with a single logic instruction,
-//     (w >> s) & mask | 0x6400_6400  =  (1024 + k c_i, 1024 + k c_j)   in fp16,   k a power of two,
-// one half2 multiply-add removes the offset exactly (codes are small integers, exact in fp16), and the
-// multiply-adds themselves run on the tensor cores: A = 16 rows x 16 codes, B = the matching 16 entries
+// here two codes become one half2 operand with a single AND (see mma_16816 below), and the multiply-adds
+// themselves run on the tensor cores: A = 16 rows x 16 codes, B = the matching 16 entries
 // of x replicated over the 8 columns, fp32 accumulators.  Products of two fp16 values are exact in fp32;
 // the accumulator is drained into an fp32 sum after every 128 columns (8 MMAs).
 //
@@ -129,20 +127,7 @@ matvec_kernel(const uint32_t* __restrict__ qweight, const float* __restrict__ sc
 // x[chunk * 32 + perm<F>(p)].  A task is 16 consecutive rows; the 16 warps of a CTA take the 128-column
 // blocks of those rows round-robin and their partial sums meet in shared memory.
 // Per 128-column block b of group gi:  y_r += s[r][gi] * (sum_{c in b} q_c x_c - z[r][gi] * sum_{c in b} x_c).
-constexpr int kMvThreads = 512, kMvWarps = kMvThreads / 32;
-
-__device__ __forceinline__ uint32_t h2_sub(uint32_t a, uint32_t b) {
-  __half2 r = __hsub2(*reinterpret_cast<__half2*>(&a), *reinterpret_cast<__half2*>(&b));
-  return *reinterpret_cast<uint32_t*>(&r);
-}
-__device__ __forceinline__ uint32_t h2_fma(uint32_t a, uint32_t b, uint32_t c) {
-  __half2 r = __hfma2(*reinterpret_cast<__half2*>(&a), *reinterpret_cast<__half2*>(&b), *reinterpret_cast<__half2*>(&c));
-  return *reinterpret_cast<uint32_t*>(&r);
-}
-constexpr uint32_t kH1024 = 0x64006400u;                       // (1024, 1024)
-// (1024 + k c) * (1 / k) - 1024 / k = c for k = 4, 16, 64, 256: multiplier and addend as half2 bit patterns
-constexpr uint32_t kInv4 = 0x34003400u, kNeg256 = 0xDC00DC00u, kInv16 = 0x2C002C00u, kNeg64 = 0xD400D400u;
-constexpr uint32_t kInv64 = 0x24002400u, kNeg16 = 0xCC00CC00u, kInv256 = 0x1C001C00u, kNeg4 = 0xC400C400u;
+constexpr int kMvThreads = 512, kMvWarps = kMvThreads / 32, kMvDepth = 2, kMvCtasPerSm = 2;
 
 __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                           uint32_t b0, uint32_t b1) {
@@ -151,72 +136,64 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// A masked field IS an fp16 number: the bit pattern 0x000c is the subnormal c * 2^-24, and a field that
+// starts at bit s (< 10) is c * 2^(s-24).  So one AND turns two codes into a half2 operand with no offset
+// to remove; fields that sit at different bit positions carry different power-of-two factors and go to
+// separate accumulators (c1 for factor 1, c2 for the factor kMvScale2<F>), combined once per 128 columns:
+//     sum q x = 2^24 * (c1 + c2 / kMvScale2).
 // Code index (0..31 inside a 32-column chunk) whose x value sits at position p of the staged chunk.
 template <int F>
 __host__ __device__ constexpr int mv_perm(int p) {
-  if (F == 4) { return (p & ~7) + ((p & 1) ? 4 : 0) + ((p & 7) >> 1); }          // word of 8: 0 4 1 5 2 6 3 7
-  if (F == 2) { return (p & ~15) + ((p & 1) ? 8 : 0) + ((p & 15) >> 1); }        // word of 16: 0 8 1 9 ... 7 15
-  if (F == 8) { return (p & ~3) + ((p & 1) ? 2 : 0) + ((p & 3) >> 1); }          // word of 4: 0 2 1 3
+  if (F == 4) { constexpr int o[8] = {0, 4, 2, 6, 1, 5, 3, 7}; return (p & ~7) + o[p & 7]; }
+  if (F == 2) { constexpr int o[16] = {0, 8, 2, 10, 4, 12, 6, 14, 1, 9, 3, 11, 5, 13, 7, 15}; return (p & ~15) + o[p & 15]; }
+  if (F == 8) { constexpr int o[4] = {0, 2, 1, 3}; return (p & ~3) + o[p & 3]; }
   return p;                                                                        // 3-bit: natural order
 }
+template <int F> struct MvScale2 { static constexpr float inv = 0.f; };            // 1 / factor of the second accumulator
+template <> struct MvScale2<4> { static constexpr float inv = 1.f / 16.f; };
+template <> struct MvScale2<2> { static constexpr float inv = 1.f / 4.f; };
 
 // One 32-column chunk of two rows (A fragment rows g and g + 8) against the staged x: 8 MMAs.
 template <int F>
-__device__ __forceinline__ void mv_chunk(const uint32_t (&wa)[F], const uint32_t (&wb)[F], const uint4* xs, float (&c)[4]);
+__device__ __forceinline__ void mv_chunk(const uint32_t (&wa)[F], const uint32_t (&wb)[F], const uint4* xs,
+                                         float (&c1)[4], float (&c2)[4]);
 
 template <>
-__device__ __forceinline__ void mv_chunk<4>(const uint32_t (&wa)[4], const uint32_t (&wb)[4], const uint4* xs, float (&c)[4]) {
+__device__ __forceinline__ void mv_chunk<4>(const uint32_t (&wa)[4], const uint32_t (&wb)[4], const uint4* xs,
+                                            float (&c1)[4], float (&c2)[4]) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < 4; ++i) {          // word i: codes (0,4) (2,6) at factor 1, (1,5) (3,7) at factor 16
     const uint4 x = xs[i];
     const uint32_t a = wa[i], b = wb[i], a8 = a >> 8, b8 = b >> 8;
-    const uint32_t a0 = h2_sub((a & 0x000F000Fu) | kH1024, kH1024), a1 = h2_fma((a & 0x00F000F0u) | kH1024, kInv16, kNeg64);
-    const uint32_t b0 = h2_sub((b & 0x000F000Fu) | kH1024, kH1024), b1 = h2_fma((b & 0x00F000F0u) | kH1024, kInv16, kNeg64);
-    mma_16816(c, a0, b0, a1, b1, x.x, x.y);
-    const uint32_t a2 = h2_sub((a8 & 0x000F000Fu) | kH1024, kH1024), a3 = h2_fma((a8 & 0x00F000F0u) | kH1024, kInv16, kNeg64);
-    const uint32_t b2 = h2_sub((b8 & 0x000F000Fu) | kH1024, kH1024), b3 = h2_fma((b8 & 0x00F000F0u) | kH1024, kInv16, kNeg64);
-    mma_16816(c, a2, b2, a3, b3, x.z, x.w);
+    mma_16816(c1, a & 0x000F000Fu, b & 0x000F000Fu, a8 & 0x000F000Fu, b8 & 0x000F000Fu, x.x, x.y);
+    mma_16816(c2, a & 0x00F000F0u, b & 0x00F000F0u, a8 & 0x00F000F0u, b8 & 0x00F000F0u, x.z, x.w);
   }
 }
 
-// eight half2 (c_j, c_{j+8}), j = 0..7, from one word of sixteen 2-bit codes
-__device__ __forceinline__ void unpack2(uint32_t w, uint32_t (&h)[8]) {
-  const uint32_t v = w >> 10;
-  h[0] = h2_sub((w & 0x00030003u) | kH1024, kH1024);
-  h[1] = h2_fma((w & 0x000C000Cu) | kH1024, kInv4, kNeg256);
-  h[2] = h2_fma((w & 0x00300030u) | kH1024, kInv16, kNeg64);
-  h[3] = h2_fma((w & 0x00C000C0u) | kH1024, kInv64, kNeg16);
-  h[4] = h2_fma((w & 0x03000300u) | kH1024, kInv256, kNeg4);
-  h[5] = h2_sub((v & 0x00030003u) | kH1024, kH1024);
-  h[6] = h2_fma((v & 0x000C000Cu) | kH1024, kInv4, kNeg256);
-  h[7] = h2_fma((v & 0x00300030u) | kH1024, kInv16, kNeg64);
-}
 template <>
-__device__ __forceinline__ void mv_chunk<2>(const uint32_t (&wa)[2], const uint32_t (&wb)[2], const uint4* xs, float (&c)[4]) {
+__device__ __forceinline__ void mv_chunk<2>(const uint32_t (&wa)[2], const uint32_t (&wb)[2], const uint4* xs,
+                                            float (&c1)[4], float (&c2)[4]) {
 #pragma unroll
-  for (int i = 0; i < 2; ++i) {
-    uint32_t ha[8], hb[8];
-    unpack2(wa[i], ha); unpack2(wb[i], hb);
+  for (int i = 0; i < 2; ++i) {          // word i, t_s = w >> 4s: codes (2s, 2s+8) at factor 1, (2s+1, 2s+9) at factor 4
     const uint4 x0 = xs[2 * i], x1 = xs[2 * i + 1];
-    mma_16816(c, ha[0], hb[0], ha[1], hb[1], x0.x, x0.y);
-    mma_16816(c, ha[2], hb[2], ha[3], hb[3], x0.z, x0.w);
-    mma_16816(c, ha[4], hb[4], ha[5], hb[5], x1.x, x1.y);
-    mma_16816(c, ha[6], hb[6], ha[7], hb[7], x1.z, x1.w);
+    const uint32_t a = wa[i], b = wb[i], a4 = a >> 4, b4 = b >> 4, a8 = a >> 8, b8 = b >> 8, a12 = a >> 12, b12 = b >> 12;
+    mma_16816(c1, a & 0x00030003u, b & 0x00030003u, a4 & 0x00030003u, b4 & 0x00030003u, x0.x, x0.y);
+    mma_16816(c1, a8 & 0x00030003u, b8 & 0x00030003u, a12 & 0x00030003u, b12 & 0x00030003u, x0.z, x0.w);
+    mma_16816(c2, a & 0x000C000Cu, b & 0x000C000Cu, a4 & 0x000C000Cu, b4 & 0x000C000Cu, x1.x, x1.y);
+    mma_16816(c2, a8 & 0x000C000Cu, b8 & 0x000C000Cu, a12 & 0x000C000Cu, b12 & 0x000C000Cu, x1.z, x1.w);
   }
 }
 
 template <>
-__device__ __forceinline__ void mv_chunk<8>(const uint32_t (&wa)[8], const uint32_t (&wb)[8], const uint4* xs, float (&c)[4]) {
+__device__ __forceinline__ void mv_chunk<8>(const uint32_t (&wa)[8], const uint32_t (&wb)[8], const uint4* xs,
+                                            float (&c1)[4], float (&)[4]) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < 4; ++i) {          // word: codes (0,2) and (1,3); 255 * 2^-24 is still subnormal
     const uint4 x = xs[i];
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const uint32_t a = wa[2 * i + u], b = wb[2 * i + u];
-      const uint32_t a0 = h2_sub((a & 0x00FF00FFu) | kH1024, kH1024), a1 = h2_sub(((a >> 8) & 0x00FF00FFu) | kH1024, kH1024);
-      const uint32_t b0 = h2_sub((b & 0x00FF00FFu) | kH1024, kH1024), b1 = h2_sub(((b >> 8) & 0x00FF00FFu) | kH1024, kH1024);
-      mma_16816(c, a0, b0, a1, b1, u ? x.z : x.x, u ? x.w : x.y);
-    }
+    mma_16816(c1, wa[2 * i] & 0x00FF00FFu, wb[2 * i] & 0x00FF00FFu,
+              (wa[2 * i] >> 8) & 0x00FF00FFu, (wb[2 * i] >> 8) & 0x00FF00FFu, x.x, x.y);
+    mma_16816(c1, wa[2 * i + 1] & 0x00FF00FFu, wb[2 * i + 1] & 0x00FF00FFu,
+              (wa[2 * i + 1] >> 8) & 0x00FF00FFu, (wb[2 * i + 1] >> 8) & 0x00FF00FFu, x.z, x.w);
   }
 }
 
@@ -226,15 +203,16 @@ __device__ __forceinline__ uint32_t pair3(const uint32_t (&w)[3], int m) {
   const int bit = 6 * m, k = bit >> 5, o = bit & 31;
   uint32_t v = w[k] >> o;
   if (o + 6 > 32 && k + 1 < 3) v |= w[k + 1] << (32 - o);
-  return h2_sub((((v & 63u) * 0x2001u) & 0x00070007u) | kH1024, kH1024);
+  return ((v & 63u) * 0x2001u) & 0x00070007u;
 }
 template <>
-__device__ __forceinline__ void mv_chunk<3>(const uint32_t (&wa)[3], const uint32_t (&wb)[3], const uint4* xs, float (&c)[4]) {
+__device__ __forceinline__ void mv_chunk<3>(const uint32_t (&wa)[3], const uint32_t (&wb)[3], const uint4* xs,
+                                            float (&c1)[4], float (&)[4]) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const uint4 x = xs[i];
-    mma_16816(c, pair3(wa, 4 * i), pair3(wb, 4 * i), pair3(wa, 4 * i + 1), pair3(wb, 4 * i + 1), x.x, x.y);
-    mma_16816(c, pair3(wa, 4 * i + 2), pair3(wb, 4 * i + 2), pair3(wa, 4 * i + 3), pair3(wb, 4 * i + 3), x.z, x.w);
+    mma_16816(c1, pair3(wa, 4 * i), pair3(wb, 4 * i), pair3(wa, 4 * i + 1), pair3(wb, 4 * i + 1), x.x, x.y);
+    mma_16816(c1, pair3(wa, 4 * i + 2), pair3(wb, 4 * i + 2), pair3(wa, 4 * i + 3), pair3(wb, 4 * i + 3), x.z, x.w);
   }
 }
 
@@ -258,10 +236,10 @@ __device__ __forceinline__ void mv_load(const uint32_t* p, bool valid, uint32_t 
   }
 }
 
-// grid: min(tasks, 2 x SMs) CTAs of 512 threads; dynamic shared memory: staged x (fp16, C rounded up to 128),
+// grid: min(tasks, kMvCtasPerSm x SMs) CTAs of 512 threads; dynamic shared memory: staged x (fp16, C rounded up to 128),
 // per-128-column sums of x (fp32), and two buffers of 16 warps x 16 rows partial sums.
 template <int F>
-__global__ void __launch_bounds__(kMvThreads, 2)
+__global__ void __launch_bounds__(kMvThreads, kMvCtasPerSm)
 matvec_mma_kernel(const uint32_t* __restrict__ qweight, const float* __restrict__ scales, const float* __restrict__ zeros,
                   const __half* __restrict__ x, int R, int C, int g, int G, float* __restrict__ y) {
   extern __shared__ uint4 mv_smem[];
@@ -292,54 +270,69 @@ matvec_mma_kernel(const uint32_t* __restrict__ qweight, const float* __restrict_
 
   const int gq = lane >> 2, t4 = lane & 3;                               // fragment row and k-quarter of this lane
   const int n_tasks = (R + 15) / 16;
+  const int my_tasks = blockIdx.x < n_tasks ? (n_tasks - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+  const int per_task = (n_blk + kMvWarps - 1) / kMvWarps;                // blocks per warp and task (the same for all warps)
   const bool per_block = g < C;                                          // grouped: scale and zero change along the row
-  int par = 0;
-  for (int task = blockIdx.x; task < n_tasks; task += gridDim.x, par ^= 1) {
+  const int chunk_bytes_w = F;                                           // words per chunk
+
+  // The (task, block) pairs of this warp form one stream; the codes of the next kMvDepth pairs are in flight in
+  // a register ring (indexed by compile-time constants only) while one block is unpacked and multiplied, also
+  // across task boundaries.
+  uint32_t wa[kMvDepth][F], wb[kMvDepth][F];
+  int lk = 0, lj = 0;                                                    // load cursor: task number, block number
+  auto issue = [&](uint32_t (&ua)[F], uint32_t (&ub)[F]) {
+    const int task = blockIdx.x + lk * gridDim.x, blk = warp + lj * kMvWarps, ch = blk * 4 + t4;
+    const bool ok = lk < my_tasks && ch < chunks;
     const int ra = min(task * 16 + gq, R - 1), rb = min(task * 16 + gq + 8, R - 1);   // clamped: loads stay in range
-    const uint32_t* pa = qweight + (int64_t)ra * chunks * F;
-    const uint32_t* pb = qweight + (int64_t)rb * chunks * F;
-    const float* sa = scales + (int64_t)ra * G; const float* za = zeros + (int64_t)ra * G;
-    const float* sb = scales + (int64_t)rb * G; const float* zb = zeros + (int64_t)rb * G;
-    float ya = 0.f, yb = 0.f;                                            // grouped: finished sums; per-row: sum of q x
-    float xsum = 0.f;                                                    // per-row: sum of x over this warp's blocks
-    // software pipeline: the codes of the next block are in flight while this block is unpacked and multiplied
-    uint32_t wa[F], wb[F];
-    {
-      const int ch = warp * 4 + t4;
-      mv_load<F>(pa + (int64_t)ch * F, warp < n_blk && ch < chunks, wa);
-      mv_load<F>(pb + (int64_t)ch * F, warp < n_blk && ch < chunks, wb);
-    }
-    for (int blk = warp; blk < n_blk; blk += kMvWarps) {
-      const int ch = blk * 4 + t4, chn = ch + 4 * kMvWarps;
-      uint32_t na[F], nb[F];
-      mv_load<F>(pa + (int64_t)chn * F, blk + kMvWarps < n_blk && chn < chunks, na);
-      mv_load<F>(pb + (int64_t)chn * F, blk + kMvWarps < n_blk && chn < chunks, nb);
-      float c[4] = {0.f, 0.f, 0.f, 0.f};
-      mv_chunk<F>(wa, wb, reinterpret_cast<const uint4*>(xs + ch * 32), c);
-      if (per_block) {
-        const int gi = (blk * 128) / g;
-        const float bx = sx[blk];
-        ya = fmaf(__ldg(sa + gi), c[0] - __ldg(za + gi) * bx, ya);
-        yb = fmaf(__ldg(sb + gi), c[2] - __ldg(zb + gi) * bx, yb);
-      } else {
-        ya += c[0]; yb += c[2]; xsum += sx[blk];
+    mv_load<F>(qweight + ((int64_t)ra * chunks + ch) * chunk_bytes_w, ok, ua);
+    mv_load<F>(qweight + ((int64_t)rb * chunks + ch) * chunk_bytes_w, ok, ub);
+    if (++lj == per_task) { lj = 0; ++lk; }
+  };
+#pragma unroll
+  for (int d = 0; d < kMvDepth; ++d) issue(wa[d], wb[d]);
+
+  int k = 0, j = 0, par = 0;
+  float ya = 0.f, yb = 0.f, xsum = 0.f;                                  // grouped: finished sums; per-row: sums of q x and of x
+  const int total = my_tasks * per_task;
+  for (int it0 = 0; it0 < total; it0 += kMvDepth) {
+#pragma unroll
+    for (int d = 0; d < kMvDepth; ++d) {
+      if (it0 + d < total) {                                             // uniform over the CTA
+        const int task = blockIdx.x + k * gridDim.x, blk = warp + j * kMvWarps, ch = blk * 4 + t4;
+        const int ra = min(task * 16 + gq, R - 1), rb = min(task * 16 + gq + 8, R - 1);
+        float c1[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};
+        if (blk < n_blk) mv_chunk<F>(wa[d], wb[d], reinterpret_cast<const uint4*>(xs + ch * 32), c1, c2);
+        issue(wa[d], wb[d]);
+        if (blk < n_blk) {
+          const float da = (c1[0] + c2[0] * MvScale2<F>::inv) * 16777216.f;  // sum of q x over the block, rows a and b
+          const float db = (c1[2] + c2[2] * MvScale2<F>::inv) * 16777216.f;
+          const float bx = sx[blk];
+          if (per_block) {
+            const int gi = (blk * 128) / g;
+            ya = fmaf(__ldg(scales + (int64_t)ra * G + gi), da - __ldg(zeros + (int64_t)ra * G + gi) * bx, ya);
+            yb = fmaf(__ldg(scales + (int64_t)rb * G + gi), db - __ldg(zeros + (int64_t)rb * G + gi) * bx, yb);
+          } else {
+            ya += da; yb += db; xsum += bx;
+          }
+        }
+        if (++j == per_task) {                                           // the task is complete: combine the warps' partial sums
+          if (!per_block) {
+            ya = __ldg(scales + ra) * (ya - __ldg(zeros + ra) * xsum);
+            yb = __ldg(scales + rb) * (yb - __ldg(zeros + rb) * xsum);
+          }
+          float* rp = red + (par * kMvWarps + warp) * 16;
+          if (t4 == 0) { rp[gq] = ya; rp[gq + 8] = yb; }
+          __syncthreads();
+          if (threadIdx.x < 16) {
+            float t = 0.f;
+#pragma unroll
+            for (int w = 0; w < kMvWarps; ++w) t += red[(par * kMvWarps + w) * 16 + threadIdx.x];
+            const int r = task * 16 + threadIdx.x;
+            if (r < R) y[r] = t;
+          }
+          j = 0; ++k; par ^= 1; ya = yb = xsum = 0.f;
+        }
       }
-#pragma unroll
-      for (int k = 0; k < F; ++k) { wa[k] = na[k]; wb[k] = nb[k]; }
-    }
-    if (!per_block) {
-      ya = __ldg(sa) * (ya - __ldg(za) * xsum);
-      yb = __ldg(sb) * (yb - __ldg(zb) * xsum);
-    }
-    float* rp = red + (par * kMvWarps + warp) * 16;
-    if (t4 == 0) { rp[gq] = ya; rp[gq + 8] = yb; }
-    __syncthreads();
-    if (threadIdx.x < 16) {
-      float t = 0.f;
-#pragma unroll
-      for (int w = 0; w < kMvWarps; ++w) t += red[(par * kMvWarps + w) * 16 + threadIdx.x];
-      const int r = task * 16 + threadIdx.x;
-      if (r < R) y[r] = t;
     }
   }
 }
@@ -372,9 +365,9 @@ gptq_status_t launch_matvec(const uint32_t* qweight, const float* scales, const 
     const int n_blk = (C + 127) / 128;
     const size_t smem = (size_t)n_blk * 128 * sizeof(__half) + (size_t)((n_blk + 3) & ~3) * sizeof(float) +
                         (size_t)2 * gptq::kMvWarps * 16 * sizeof(float);
-    if (smem > 110 * 1024) return GPTQ_ERR_UNSUPPORTED;               // two CTAs per SM
+    if (smem > 220 * 1024 / gptq::kMvCtasPerSm) return GPTQ_ERR_UNSUPPORTED;
     const int tasks = (R + 15) / 16;
-    int grid = 2 * gptq::device_sm_count_inference();
+    int grid = gptq::kMvCtasPerSm * gptq::device_sm_count_inference();
     if (grid > tasks) grid = tasks;
     GPTQ_CUDA_TRY(cudaFuncSetAttribute(gptq::matvec_mma_kernel<F>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     gptq::matvec_mma_kernel<F><<<grid, gptq::kMvThreads, smem, s>>>(qweight, scales, zeros, x, R, C, g, G, y);
