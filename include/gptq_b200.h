@@ -177,8 +177,11 @@ gptq_status_t gptq_rtn_layer(const void* W_fp16, int R, int C, int bits, int gro
  *   W_out_fp16 [R x C] half.
  * gptq_matvec: y = W^ x for ONE fp16 vector x (batch-1 generation: "quantized-matrix
  *   full-precision-vector product" with dequantization on the fly, never materialising W^).
- *   x_fp16 [C] half, y [R] fp32; products and sums in fp32.  C <= 51200 (x is staged in
- *   shared memory), else GPTQ_ERR_UNSUPPORTED. */
+ *   x_fp16 [C] half, y [R] fp32; products exact, sums in fp32: per group the kernel forms
+ *   sum q x and zero * sum x and combines them with the scale, so its rounding error is
+ *   fp32-level relative to sum scale * (q + zero) * |x|.  Per-row grids and group sizes that
+ *   are multiples of 128 run on the tensor cores (mma.sync f16), other group sizes on the
+ *   CUDA cores.  C <= 51200 (x is staged in shared memory), else GPTQ_ERR_UNSUPPORTED. */
 gptq_status_t gptq_dequantize(const uint32_t* qweight, const float* scales, const float* zeros,
                               int R, int C, int bits, int group_size, void* W_out_fp16, void* stream);
 gptq_status_t gptq_matvec(const uint32_t* qweight, const float* scales, const float* zeros,
