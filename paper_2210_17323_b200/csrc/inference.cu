@@ -17,30 +17,42 @@ __device__ __forceinline__ uint32_t code_at(const uint32_t (&w)[F], int i) {
   return v & ((1u << F) - 1u);
 }
 
-// ---- whole-matrix dequantization: one thread per 32 columns ------------------------------------
+// ---- whole-matrix dequantization: one thread per 8 columns --------------------------------------
+// A warp reads 32 F consecutive bytes of codes and writes 512 consecutive bytes of fp16 with one 16-byte
+// streaming store per lane.  A thread keeps its 8 columns and walks down the rows (blockIdx.y, grid-stride), so
+// the bit offset, the word index and the group index are computed once.
 template <int F>
-__global__ void dequantize_kernel(const uint32_t* __restrict__ qweight, const float* __restrict__ scales,
-                                  const float* __restrict__ zeros, int R, int C, int g, int G,
-                                  __half* __restrict__ out) {
-  const int chunks = C / 32;
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (int64_t)R * chunks) return;
-  const int r = (int)(idx / chunks), ch = (int)(idx % chunks);
-  uint32_t w[F];
-  const uint32_t* p = qweight + ((int64_t)r * chunks + ch) * F;
+__global__ void __launch_bounds__(256)
+dequantize_kernel(const uint32_t* __restrict__ qweight, const float* __restrict__ scales,
+                  const float* __restrict__ zeros, int R, int C, int g, int G, __half* __restrict__ out) {
+  const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * 8;
+  if (c0 >= C) return;
+  // the 8 codes are 8 F bits of the row's bit stream, starting at bit c0 * F (a multiple of 8)
+  const int bit = c0 * F, k = bit >> 5, o = bit & 31;
+  const bool two = o + 8 * F > 32;
+  const int gi0 = c0 / g;
+  const int64_t wpr = (int64_t)(C / 32) * F;                  // words per row
+  for (int r = blockIdx.y; r < R; r += gridDim.y) {
+    const uint32_t* rowp = qweight + r * wpr;
+    uint64_t v = __ldg(rowp + k);
+    if (two) v |= (uint64_t)__ldg(rowp + k + 1) << 32;
+    v >>= o;
+    __align__(16) __half h[8];
+    if (g >= 8) {
+      const float s = __ldg(scales + (int64_t)r * G + gi0), z = __ldg(zeros + (int64_t)r * G + gi0);
 #pragma unroll
-  for (int k = 0; k < F; ++k) w[k] = p[k];
-  __align__(16) __half h[32];
+      for (int i = 0; i < 8; ++i)
+        h[i] = __float2half_rn(__fmul_rn(s, (float)(uint32_t)((v >> (i * F)) & ((1u << F) - 1u)) - z));
+    } else {
 #pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    const int gi = (ch * 32 + i) / g;
-    const float s = scales[(int64_t)r * G + gi], z = zeros[(int64_t)r * G + gi];
-    h[i] = __float2half_rn(__fmul_rn(s, (float)code_at<F>(w, i) - z));
+      for (int i = 0; i < 8; ++i) {
+        const int gi = (c0 + i) / g;
+        const float s = __ldg(scales + (int64_t)r * G + gi), z = __ldg(zeros + (int64_t)r * G + gi);
+        h[i] = __float2half_rn(__fmul_rn(s, (float)(uint32_t)((v >> (i * F)) & ((1u << F) - 1u)) - z));
+      }
+    }
+    __stcs(reinterpret_cast<uint4*>(out + (int64_t)r * C + c0), *reinterpret_cast<const uint4*>(h));
   }
-  uint4* o = reinterpret_cast<uint4*>(out + (int64_t)r * C + ch * 32);
-  const uint4* hv = reinterpret_cast<const uint4*>(h);
-#pragma unroll
-  for (int k = 0; k < 4; ++k) o[k] = hv[k];
 }
 
 // ---- y = dequant(Q) x for one fp16 vector x: one warp per row -------------------------------------
@@ -351,8 +363,12 @@ inline int device_sm_count_inference() {
 template <int F>
 gptq_status_t launch_dequantize(const uint32_t* qweight, const float* scales, const float* zeros, int R, int C, int g,
                                 int G, __half* out, cudaStream_t s) {
-  const int64_t total = (int64_t)R * (C / 32);
-  gptq::dequantize_kernel<F><<<(unsigned)((total + 127) / 128), 128, 0, s>>>(qweight, scales, zeros, R, C, g, G, out);
+  const int gx = (C / 8 + 255) / 256;
+  int gy = gptq::device_sm_count_inference() * 32 / gx;                  // about 32 CTAs per SM in total
+  if (gy < 1) gy = 1;
+  if (gy > R) gy = R;
+  if (gy > 65535) gy = 65535;
+  gptq::dequantize_kernel<F><<<dim3(gx, gy), 256, 0, s>>>(qweight, scales, zeros, R, C, g, G, out);
   GPTQ_LAUNCH_CHECK();
   return GPTQ_OK;
 }
