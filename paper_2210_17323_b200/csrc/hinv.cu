@@ -5,13 +5,14 @@
 // and U^T U = U~^-T U~^-1 = H~^-1, so by uniqueness it is the matrix Algorithm 1 asks for, at
 // 2 C^3 / 3 flops and without ever forming H~^-1.
 //
-// Two-level blocking.  128 x 128 diagonal blocks are factored and inverted in fp64 in shared
-// memory by one CTA; products inside a 1024-column outer panel are fp32 CUDA-core tile GEMMs;
-// everything that reaches across outer panels (almost all of the flops for large C) is a
-// left-looking fp32-accurate tensor-core contraction (3xTF32, tcgen05) over tf32 hi / lo copies
-// of the factor that are written as each panel is finalised.
+// Two-level blocking.  128 x 128 diagonal blocks are factored and inverted in fp64 (registers) by
+// one CTA; products inside a 1024-column outer panel are small fp32 CUDA-core GEMMs
+// (gemm_small.cuh); everything that reaches across outer panels (almost all of the flops for
+// large C) is a left-looking fp32-accurate tensor-core contraction (3xTF32, tcgen05) over tf32
+// hi / lo copies of the factor that are written as each panel is finalised.  The launches of one
+// call go to three streams (dependency chain, wide contractions, diagonal-block inverses): see
+// gptq_prepare_hinv below.
 #include "common.cuh"
-#include "gemm_simt.cuh"
 #include "gemm_small.cuh"
 #include "gemm_umma.cuh"
 
@@ -178,36 +179,6 @@ __global__ void store_diag_block_kernel(float* __restrict__ U, int C, int k0, in
   }
 }
 
-// Tiles of the M x N product that reach the part on or above the diagonal, the output columns
-// being shifted by nofs against the rows (output element (m, nofs + n)).
-struct UpperTilesOfs {
-  int K, nofs;
-  __device__ __forceinline__ bool operator()(int m0, int n0, int, int, int& k0, int& k1) const {
-    k0 = 0; k1 = K;
-    return m0 <= nofs + n0 + kSimtBN - 1;
-  }
-};
-// K starts at the tile's first row: the left factor is upper triangular.
-struct UpperLeftFactorRange {
-  int K;
-  __device__ __forceinline__ bool operator()(int m0, int, int, int, int& k0, int& k1) const {
-    k0 = m0; k1 = K;
-    return k0 < k1;
-  }
-};
-// Same, with the K range of each tile row cut into gridDim.z pieces (partial sums are reduced atomically).
-struct UpperLeftFactorSplitK {
-  int K;
-  __device__ __forceinline__ bool operator()(int m0, int, int z, int nz, int& k0, int& k1) const {
-    const int per = ((K - m0 + nz - 1) / nz + kSimtBK - 1) / kSimtBK * kSimtBK;
-    k0 = m0 + z * per; k1 = min(K, k0 + per);
-    return k0 < k1;
-  }
-};
-struct AtomicSubF32 {
-  float* p; int64_t ld;
-  __device__ __forceinline__ void operator()(int m, int n, float acc) const { atomicAdd(&p[(int64_t)m * ld + n], -acc); }
-};
 struct StoreF32 {
   float* p; int64_t ld;
   __device__ __forceinline__ void operator()(int m, int n, float acc) const { p[(int64_t)m * ld + n] = acc; }
@@ -357,34 +328,6 @@ HinvWs carve_hinv(void* ws, int C) {
   o.TAlo = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);
   o.bytes = w.off;
   return o;
-}
-
-// In-place inversion of the upper-triangular w x w block at D (leading dimension C) whose 128 x 128
-// diagonal blocks already have their inverses in Dinv (first block at Dinv).  CUDA-core path.
-gptq_status_t invert_upper_block(float* D, int C, int w, float* Dinv, float* T, cudaStream_t s) {
-  for (int k0 = 0; k0 < w; k0 += kNB) {
-    const int nb = (w - k0 < kNB) ? w - k0 : kNB;
-    float* Dk = Dinv + (size_t)(k0 / kNB) * kNB * kNB;
-    if (k0 > 0) {
-      // T = U~[0:k0, blk] * V_kk
-      GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, 1, RowMajorF32{D + k0, C}, RowMajorF32{Dk, kNB},
-                                     FullRange{nb}, StoreF32{T, kNB}, s));
-      // U[0:k0, blk] = -U[0:k0, 0:k0] * T   (left factor already inverted, upper triangular)
-      // (only k0 / 128 tiles: the K range is split so that more SMs take part)
-      const int nz = k0 / kNB > 1 ? k0 / kNB : 1;
-      if (nz == 1) {
-        GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, 1, RowMajorF32{D, C}, RowMajorF32{T, kNB},
-                                       UpperLeftFactorRange{k0}, StoreNegF32{D + k0, C}, s));
-      } else {
-        GPTQ_CUDA_TRY(cudaMemset2DAsync(D + k0, (size_t)C * 4, 0, (size_t)nb * 4, k0, s));
-        GPTQ_CUDA_TRY(launch_gemm_simt(k0, nb, nz, RowMajorF32{D, C}, RowMajorF32{T, kNB},
-                                       UpperLeftFactorSplitK{k0}, AtomicSubF32{D + k0, C}, s));
-      }
-    }
-    store_diag_block_kernel<<<8, 256, 0, s>>>(D, C, k0, nb, Dk);
-    GPTQ_LAUNCH_CHECK();
-  }
-  return GPTQ_OK;
 }
 
 }  // namespace
