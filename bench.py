@@ -172,7 +172,9 @@ def run_gpu(args, wl):
 
     # each rank solves its own copy of the layer set (block index = rank -> its own seeds)
     layers = multi.rank_layers(wl.layers, rank)
-    overlap = not args.no_overlap
+    if args.no_overlap:
+        args.schedule = "sequential"
+    overlap = args.schedule != "sequential"
     state = []
     ws_bytes = 256
     for L in layers:
@@ -221,20 +223,25 @@ def run_gpu(args, wl):
 
     def step(record):
         done = []
-        for li in (order if overlap else range(len(state))):
-            st = state[li]
-            fns = stage_fns(st)
-            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4 + len(wl.grids))] if record else None
-            cs = chain_streams[li]
+        layer_order = order if overlap else range(len(state))
+        evs = {li: ([torch.cuda.Event(enable_timing=True) for _ in range(4 + len(wl.grids))] if record else None)
+               for li in layer_order}
+        h_done = {}
+
+        def hessian(li):
+            ev = evs[li]
             with torch.cuda.stream(main):
                 if record: ev[0].record(main)
-                run_stage(li, *fns[0])
+                run_stage(li, *stage_fns(state[li])[0])
                 if record:
-                    ev[1].record(main); h_done = ev[1]
+                    ev[1].record(main); h_done[li] = ev[1]
                 else:
-                    h_done = torch.cuda.Event(); h_done.record(main)
+                    h_done[li] = torch.cuda.Event(); h_done[li].record(main)
+
+        def chain(li, after):
+            ev, cs, fns = evs[li], chain_streams[li], stage_fns(state[li])
             with torch.cuda.stream(cs):
-                cs.wait_event(h_done)
+                cs.wait_event(after)
                 if record: ev[2].record(cs)
                 run_stage(li, *fns[1])
                 if record: ev[3].record(cs)
@@ -245,6 +252,17 @@ def run_gpu(args, wl):
             done.append(end)
             if record:
                 stage_events.append((li, ev))
+
+        if args.schedule == "hessians-first":
+            for li in layer_order:
+                hessian(li)
+            last = h_done[list(layer_order)[-1]]
+            for li in layer_order:
+                chain(li, last)
+        else:
+            for li in layer_order:
+                hessian(li)
+                chain(li, h_done[li])
         for e in done:                            # the step ends when every layer's chain has ended
             main.wait_event(e)
 
@@ -337,9 +355,11 @@ def run_gpu(args, wl):
                             block=wl.block, damp=wl.damp, calib_tokens=wl.layers[0].n_tokens,
                             cache="inputs larger than L2 (X >= 0.4 GB per layer); no flush needed",
                             launch="CUDA graphs, one per stage per layer" if graphs else "host-issued launches",
-                            schedule=("overlapped: Hessians back to back on one stream, each layer's stages 2-3 on its own "
-                                      "stream; stage_ms are in-context times that overlap one another") if overlap
-                            else "sequential: one stream, layer after layer",
+                            schedule={"pipelined": "pipelined: Hessians back to back on one stream, each layer's stages 2-3 on its own "
+                                                   "stream as soon as its Hessian is done; stage_ms are in-context times that overlap",
+                                      "hessians-first": "hessians-first: all Hessians on one stream, then every layer's stages 2-3 side by "
+                                                        "side on its own stream; stage 2-3 times overlap one another",
+                                      "sequential": "sequential: one stream, layer after layer"}[args.schedule],
                             parallelism=f"layer-set replica per GPU x{world}"),
                 sec_per_layer=ms_per_step * 1e-3 / len(layers),
                 stage_ms=tot, per_layer=list(per.values()),
@@ -456,8 +476,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-graphs", action="store_true", help="issue every kernel launch from the host instead of replaying CUDA graphs")
-    ap.add_argument("--no-overlap", action="store_true",
-                    help="run the layers one after another on one stream (per-stage times then do not overlap)")
+    ap.add_argument("--schedule", default="pipelined", choices=["pipelined", "hessians-first", "sequential"],
+                    help="pipelined: Hessians back to back on one stream, each layer's stages 2-3 on its own stream as soon as "
+                         "its Hessian is done; hessians-first: all Hessians, then all layers' stages 2-3 side by side; "
+                         "sequential: one stream, layer after layer")
+    ap.add_argument("--no-overlap", action="store_true", help="same as --schedule sequential")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--mode", default="solver", choices=["solver", "inference"],
