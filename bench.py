@@ -468,6 +468,124 @@ def run_inference(args, wl):
     return 0
 
 
+def run_block(args, wl):
+    """Transformer-block pipeline on one GPU (Section 5, Setup: a block's layers are quantized from the same pass of
+    calibration inputs).  q, k and v read the same input, so they share ONE Hessian and ONE factor U; o, fc1 and fc2
+    have their own.  The Hessians run back to back on one stream; each input group's stage 2 follows on its own
+    stream, and every member layer's stage 3 on its own stream after that.  One grid (--grid) per run, as a real
+    quantization run has.  Prints the block time and the solver-only time of a whole model of such blocks."""
+    import torch
+    from paper_2210_17323_b200 import binding as B
+    from paper_2210_17323_b200.synth import device as D
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    g = wl.grids[min(args.grid, len(wl.grids) - 1)]
+    groups = []                                   # (input layer, member layers)
+    for L in wl.layers:
+        shared = [gr for gr in groups if L.kind in ("k", "v") and gr[0].kind == "q" and gr[0].block_idx == L.block_idx
+                  and gr[0].C == L.C]
+        if shared:
+            shared[0][1].append(L)
+        else:
+            groups.append((L, [L]))
+    state = []
+    for Lx, members in groups:
+        gs = dict(Lx=Lx, X=D.fill_x(Lx, device=dev),
+                  H=torch.empty((Lx.C, Lx.C), dtype=torch.float32, device=dev),
+                  U=torch.empty((Lx.C, Lx.C), dtype=torch.float32, device=dev),
+                  info=torch.zeros(2, dtype=torch.int32, device=dev),
+                  ws=torch.empty(max(256, B.gptq_hessian_workspace_bytes(Lx.C, Lx.n_tokens),
+                                     B.gptq_prepare_hinv_workspace_bytes(Lx.C)), dtype=torch.uint8, device=dev),
+                  stream=torch.cuda.Stream(device=dev), members=[])
+        for L in members:
+            gs["members"].append(dict(L=L, W=D.fill_w(L, device=dev), out=None, stream=torch.cuda.Stream(device=dev),
+                                      ws=torch.empty(B.gptq_quantize_workspace_bytes(L.R, L.C, g.bits, g.group_size, wl.block),
+                                                     dtype=torch.uint8, device=dev)))
+        state.append(gs)
+    state.sort(key=lambda gs: -(gs["Lx"].C ** 2) * (gs["Lx"].n_tokens + gs["Lx"].C))
+    main = torch.cuda.Stream(device=dev)
+    torch.cuda.synchronize()
+
+    def fH(gs): gs["H"].zero_(); B.gptq_hessian_accumulate(gs["H"], gs["X"], ws=gs["ws"])
+    def fU(gs): B.gptq_prepare_hinv(gs["H"], wl.damp, U=gs["U"], ws=gs["ws"], dev_info=gs["info"])
+    def fQ(gs, m): m["out"] = B.gptq_quantize_layer(m["W"], gs["U"], g.bits, g.group_size, g.sym, wl.block, ws=m["ws"])
+
+    graphs = {}
+
+    def run(key, fn):
+        if key in graphs:
+            graphs[key].replay()
+        else:
+            fn()
+
+    def step():
+        ends = []
+        for gi, gs in enumerate(state):
+            with torch.cuda.stream(main):
+                run(("H", gi), lambda: fH(gs))
+                h_done = torch.cuda.Event(); h_done.record(main)
+            with torch.cuda.stream(gs["stream"]):
+                gs["stream"].wait_event(h_done)
+                run(("U", gi), lambda: fU(gs))
+                u_done = torch.cuda.Event(); u_done.record(gs["stream"])
+            for mi, m in enumerate(gs["members"]):
+                with torch.cuda.stream(m["stream"]):
+                    m["stream"].wait_event(u_done)
+                    run(("Q", gi, mi), lambda: fQ(gs, m))
+                    e = torch.cuda.Event(); e.record(m["stream"]); ends.append(e)
+        for e in ends:
+            main.wait_event(e)
+
+    launches0 = B.gptq_launch_count()
+    step()
+    torch.cuda.synchronize()
+    launches_per_step = B.gptq_launch_count() - launches0
+    if not args.no_graphs:
+        for gi, gs in enumerate(state):
+            for key, fn in ([(("H", gi), lambda: fH(gs)), (("U", gi), lambda: fU(gs))] +
+                            [(("Q", gi, mi), (lambda m=m: fQ(gs, m))) for mi, m in enumerate(gs["members"])]):
+                cg = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(cg):
+                    fn()
+                graphs[key] = cg
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    for gs in state:
+        assert gs["info"].tolist()[0] == 0, "prepare_hinv reported an error"
+    sampler = ClockSampler(0)
+    sampler.start()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record(main)
+    for _ in range(args.steps):
+        step()
+    t1.record(main)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = t0.elapsed_time(t1) / args.steps
+    blocks_here = len({L.block_idx for L in wl.layers})
+    model_blocks = {1: 12, 2: 32, 3: 96, 4: 70}.get(wl.config_id)     # OPT-125M, OPT-6.7B, OPT-175B, BLOOM-176B
+    sec_per_block = ms * 1e-3 / blocks_here
+    line = dict(metric=METRIC, value=wl.weights / (ms * 1e-3), unit=UNIT, n_gpus=1, steps=args.steps, warmup=args.warmup,
+                ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, data="synthetic",
+                dtype="bf16 x bf16 -> f32 (Hessian); f32 factor; f64 working weights + f32 update sums (quantize)",
+                config=dict(workload=wl.name, mode="block pipeline: q, k, v share one Hessian and one factor",
+                            grid=dict(bits=g.bits, group_size=g.group_size, sym=g.sym), block=wl.block, damp=wl.damp,
+                            input_groups=[[m["L"].name for m in gs["members"]] for gs in state],
+                            hessians_per_block=len(state) // blocks_here,
+                            launch="CUDA graphs, one per stage" if graphs else "host-issued launches"),
+                sec_per_block=sec_per_block,
+                model_estimate=(dict(blocks=model_blocks, solver_seconds=model_blocks * sec_per_block,
+                                     note="solver only (this library's three stages) for a model of that many such blocks; the "
+                                          "paper's ~4 GPU-hours for OPT-175B on one A100 cover its whole pipeline and are "
+                                          "context, not a comparison") if model_blocks else None),
+                gpu_launches=int(launches_per_step * args.steps), clocks=clocks)
+    print(json.dumps(line))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -483,9 +601,11 @@ def main():
     ap.add_argument("--no-overlap", action="store_true", help="same as --schedule sequential")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--mode", default="solver", choices=["solver", "inference"],
+    ap.add_argument("--mode", default="solver", choices=["solver", "inference", "block"],
                     help="solver: the layer-solver step (default, the headline metric); inference: bandwidth of the "
-                         "packed matvec / dequantize kernels")
+                         "packed matvec / dequantize kernels; block: Transformer-block pipeline in which q, k, v share "
+                         "one Hessian and one factor")
+    ap.add_argument("--grid", type=int, default=0, help="--mode block: index of the workload's grid to run")
     ap.add_argument("--layer", default=None, metavar="RxCxTOKENS",
                     help="profile one layer of this shape (grid, block and damp of --workload) instead of the "
                          "whole layer set -- a small case of the same kernels for profiler captures")
@@ -500,6 +620,8 @@ def main():
         return run_reference(args, wl)
     if args.mode == "inference":
         return run_inference(args, wl)
+    if args.mode == "block":
+        return run_block(args, wl)
     return run_gpu(args, wl)
 
 
