@@ -332,12 +332,12 @@ def run_gpu(args, wl):
     # the stage sums overlap one another in the overlapped schedule, so the dominant kernel is chosen against the step
     if tot["hessian_ms"] >= tot["quantize_ms"] or tot["hessian_ms"] >= 0.3 * ms_per_step:
         ach = hess_flops / (tot["hessian_ms"] * 1e-3) / 1e12
-        # DRAM traffic per launch: measured 4.6 x the algorithmic bytes (X once + H once) on the ncu capture of a
+        # DRAM traffic per launch: measured 3.4 x the algorithmic bytes (X once + H once) on the ncu capture of a
         # 4096-channel x 65536-token launch (profiles/); scaled to these launches by their algorithmic bytes
         algo_bytes = sum(L.n_tokens * L.C * 2 + L.C * L.C * 4 for L in layers) / len(layers)
         roof = dict(kernel="hessian_accumulate", bound="tensor", achieved=ach, peak=peaks["bf16_sustained"],
-                    unit="TFLOP/s", frac=ach / peaks["bf16_sustained"], traffic=4.6 * algo_bytes,
-                    traffic_note="bytes per launch (mean over layers), = 4.6 x algorithmic bytes, ratio from an ncu capture of a smaller launch",
+                    unit="TFLOP/s", frac=ach / peaks["bf16_sustained"], traffic=3.4 * algo_bytes,
+                    traffic_note="bytes per launch (mean over layers), = 3.4 x algorithmic bytes (dram__bytes_read + dram__bytes_write of the two-CTA kernel on a 4096-channel x 65536-token launch, profiles/hessian_two_cta_kernel_4096ch_65536tok.md), scaled by algorithmic bytes",
                     peak_source=f"bf16 sustained, {peaks['source']}")
     else:
         ach = upd_flops / (tot["quantize_ms"] * 1e-3) / 1e12
