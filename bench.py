@@ -332,12 +332,19 @@ def run_gpu(args, wl):
     # the stage sums overlap one another in the overlapped schedule, so the dominant kernel is chosen against the step
     if tot["hessian_ms"] >= tot["quantize_ms"] or tot["hessian_ms"] >= 0.3 * ms_per_step:
         ach = hess_flops / (tot["hessian_ms"] * 1e-3) / 1e12
-        # DRAM traffic per launch: measured 3.4 x the algorithmic bytes (X once + H once) on the ncu capture of a
-        # 4096-channel x 65536-token launch (profiles/); scaled to these launches by their algorithmic bytes
+        # DRAM traffic per launch: dram__bytes_read + dram__bytes_write of this kernel were captured on two smaller
+        # launches (profiles/hessian_two_cta_kernel_4096ch_65536tok.md): 2.4 x the algorithmic bytes (X once + H once) at
+        # 4096 channels and 10.9 x at 16384 channels (every band of tile rows streams the column strips to its right
+        # again); the ratio is interpolated linearly in C between them and extrapolated beyond, and scaled to these
+        # launches by their algorithmic bytes
+        def traffic_ratio(C):
+            return 2.4 if C <= 4096 else 2.4 + (10.9 - 2.4) * (C - 4096) / (16384 - 4096)
         algo_bytes = sum(L.n_tokens * L.C * 2 + L.C * L.C * 4 for L in layers) / len(layers)
+        est_traffic = sum(traffic_ratio(L.C) * (L.n_tokens * L.C * 2 + L.C * L.C * 4) for L in layers) / len(layers)
         roof = dict(kernel="hessian_accumulate", bound="tensor", achieved=ach, peak=peaks["bf16_sustained"],
-                    unit="TFLOP/s", frac=ach / peaks["bf16_sustained"], traffic=3.4 * algo_bytes,
-                    traffic_note="bytes per launch (mean over layers), = 3.4 x algorithmic bytes (dram__bytes_read + dram__bytes_write of the two-CTA kernel on a 4096-channel x 65536-token launch, profiles/hessian_two_cta_kernel_4096ch_65536tok.md), scaled by algorithmic bytes",
+                    unit="TFLOP/s", frac=ach / peaks["bf16_sustained"], traffic=est_traffic,
+                    traffic_note=f"bytes per launch, mean over layers = {est_traffic / algo_bytes:.1f} x algorithmic bytes; from ncu "
+                                 "captures of 4096- and 16384-channel launches (2.4 x and 10.9 x), interpolated in C",
                     peak_source=f"bf16 sustained, {peaks['source']}")
     else:
         ach = upd_flops / (tot["quantize_ms"] * 1e-3) / 1e12
