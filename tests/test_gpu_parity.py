@@ -262,6 +262,43 @@ def test_solve_layer_from_host_buffers(B):
         B.gptq_solve_layer_host(Wh, Xh, 5, 0, False, 128, 0.01)      # unsupported bits
 
 
+def test_two_host_buffer_calls_in_flight_match_the_oracle(B):
+    """Two host threads, each with its own stream and device workspace, solve different layers at the same time
+    (the benchmark's end-to-end leg does this).  Stage 2 shares its internal streams and events between the calls;
+    both results must still match the oracle.  The wider layer has several outer panels, so those streams are used."""
+    import threading
+    cases = [(_layer(64, 2304, 3000, cfg=7, kind="fc2"), 3, 128), (_layer(96, 1280, 4000, cfg=8, kind="q"), 4, 0)]
+    refs, inputs = [], []
+    for L, bits, group in cases:
+        xb, W16 = L.x_bits(), L.w()
+        refs.append((O.solve_layer(W16, xb, bits, group, False, 128, 0.01), W16, bits, L))
+        inputs.append((torch.from_numpy(W16).pin_memory(), torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()))
+    dev = torch.cuda.current_device()
+    outs, errs = [None, None], []
+
+    def work(i):
+        try:
+            torch.cuda.set_device(dev)
+            stream = torch.cuda.Stream()
+            _, bits, group = cases[i][0], cases[i][1], cases[i][2]
+            for _ in range(3):              # several rounds so that the two calls really overlap
+                outs[i] = B.gptq_solve_layer_host(inputs[i][0], inputs[i][1], bits, group, False, 128, 0.01, stream=stream)
+        except Exception as e:
+            errs.append(e)
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errs, errs
+    for out, (ref, W16, bits, L) in zip(outs, refs):
+        assert out["info"].tolist() == [0, 0]
+        gpu = dict(qweight=out["qweight"].numpy(), scales=out["scales"].numpy(), zeros=out["zeros"].numpy(),
+                   loss=out["loss"].item())
+        check_quantize_outputs(gpu, ref, W16, bits, L.C, ref["H"])
+
+
 @pytest.mark.parametrize("bits,group", [(4, 0), (3, 0), (3, 128), (2, 32), (4, 8), (4, 1024), (O.BITS_TERNARY, 8), (8, 64)])
 def test_rtn_layer_bit_exact_and_equals_solver_on_diagonal_hessian(B, bits, group):
     """RTN entry point: codes, scales and zeros bit-exact against the oracle's RTN (both sides decide in
