@@ -202,7 +202,9 @@ gptq_status_t gptq_matvec(const uint32_t* qweight, const float* scales, const fl
  *              two X staging buffers, the outputs and the stages' own workspaces.
  * Unlike the per-stage calls this one SYNCHRONISES `stream` before returning (the results are on
  * the host when it returns); it creates and destroys one internal stream and a few events per
- * call and allocates no device memory. */
+ * call and allocates no device memory.  Calls from different host threads may be in flight at
+ * the same time if each has its own `stream` and `dev_ws` (one layer's X then crosses PCIe while
+ * another layer is factored and quantized). */
 size_t gptq_solve_layer_host_workspace_bytes(int R, int C, int64_t n_tokens, int bits, int group_size, int block);
 gptq_status_t gptq_solve_layer_host(const void* W_fp16_host, const void* X_bf16_host, int64_t n_tokens,
                                     int R, int C, float damp, int bits, int group_size, int sym, int block,
