@@ -125,7 +125,7 @@ CASES = [
     (64, 256, 8, 0, False, 128),
     (64, 256, 4, 64, True, 64),        # symmetric grid
     (260, 2304, 4, 0, False, 128),     # several outer (lazy) blocks
-    (130, 2176, 3, 128, False, 96),    # block that is not a power of two; ragged outer block
+    (130, 2176, 3, 32, False, 96),     # block that is not a power of two (groups of 32 nest in it); ragged outer block
     (64, 2048, O.BITS_TERNARY, 8, False, 128),   # the paper's ternary setting: group size 8
     (64, 2048, 4, 1024, False, 128),             # group size 1024 (group spans eight blocks)
     (64, 2048, 2, 32, False, 128),               # group size 32
@@ -134,8 +134,7 @@ CASES = [
 
 @pytest.mark.parametrize("R,C,bits,group,sym,block", CASES)
 def test_quantize_layer_matches_oracle(B, R, C, bits, group, sym, block):
-    if group and (group % block and block % group):
-        pytest.skip("not nested")
+    assert not (group and (group % block and block % group)), "cases must have nested group and block sizes"
     L = _layer(R, C, 2 * C + 64, cfg=8)
     W16 = L.w()
     H = O.hessian_accumulate(np.zeros((C, C)), L.x_bits())
@@ -192,7 +191,8 @@ def test_argument_errors_are_synchronous(B):
     W = torch.zeros((4, 64), dtype=torch.float16, device="cuda")
     U = torch.eye(64, device="cuda")
     for kw, st in ((dict(bits=5), B.ERR_UNSUPPORTED), (dict(bits=4, block=48), B.ERR_UNSUPPORTED),
-                   (dict(bits=4, group_size=48), B.ERR_INVALID_ARG), (dict(bits=4, block=0), B.ERR_INVALID_ARG)):
+                   (dict(bits=4, group_size=48), B.ERR_INVALID_ARG), (dict(bits=4, block=0), B.ERR_INVALID_ARG),
+                   (dict(bits=4, group_size=64, block=96), B.ERR_INVALID_ARG)):      # group and block do not nest
         with pytest.raises(B.GptqError) as e:
             B.gptq_quantize_layer(W, U, **kw)
         assert e.value.status == st
