@@ -26,7 +26,7 @@ sys.path.insert(0, ROOT)
 
 METRIC = "gptq_weights_quantized_per_second"
 UNIT = "weights/s"
-DEFAULT_WORKLOAD = "c2"
+DEFAULT_WORKLOAD = "c3"
 
 
 def _peaks():

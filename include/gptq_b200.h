@@ -25,6 +25,9 @@
  *   - Matrices are dense row-major.  The paper's X is d_col x m; this API takes
  *     its transpose, token-major: X[t][c], t < n_tokens, c < C.
  *   - C must be a multiple of 32.
+ *   - The device that owns the buffers and `stream` must be the CURRENT device of the calling
+ *     thread (cudaSetDevice) for every call: per-device state inside the library (internal
+ *     streams, SM count, the static scratch of gptq_prepare_hinv_static) is looked up by it.
  */
 #ifndef GPTQ_B200_H_
 #define GPTQ_B200_H_
@@ -63,7 +66,7 @@ uint64_t gptq_launch_count(void);
  *                                               Algorithm 1 caption: 2 X X^T)
  *   H        [C x C] fp32, in/out.  The caller zeroes it before the first call;
  *            calls add, so calibration batches may arrive in any chunking
- *            (Section 5, Setup: "accumulate the layer-Hessians").  Both
+ *            (Section 5, Setup: Hessians are summed over calibration batches).  Both
  *            triangles are valid on return.  No 1/m normalisation.
  *   X_bf16   [n_tokens x C] bfloat16, row-major, 16-byte aligned.
  *   n_tokens >= 0 (0 is a no-op).
@@ -134,8 +137,8 @@ gptq_status_t gptq_prepare_hinv_static(const float* H, float damp, int C, float*
  *   group_size <= 0: one grid per row, fixed from the original row before the
  *              process (Section 2; Section 5 Setup: per-row asymmetric min-max).
  *              > 0: g consecutive weights share a grid, taken at the group's first
- *              column from the weights as updated so far (Section 5: "always using
- *              the most current updated weights").  Must divide C, and nest with
+ *              column from the weights as updated so far (Section 5, grouping).
+ *              Must divide C, and nest with
  *              `block` (g % block == 0 or block % g == 0).  Supported sizes: 4, 8, 16
  *              or any multiple of 32 (the paper uses 8, 32, 64, 128, 1024); anything
  *              else returns GPTQ_ERR_UNSUPPORTED.
@@ -160,7 +163,7 @@ gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U, int R, int
                                   void* ws, size_t ws_bytes, int* dev_info, void* stream);
 
 /* ------------------------------------------------------------------ round-to-nearest baseline
- * RTN (Section 5, "Baselines"): every weight rounded to the nearest value of "exactly the same"
+ * RTN (Section 5, Baselines): every weight rounded to the nearest value of the solver's own
  * grid -- per-row (group_size <= 0) or per-group min-max taken from the ORIGINAL weights -- with
  * no error feedback.  Equals gptq_quantize_layer for a diagonal Hessian.  Arguments and output
  * layout as in gptq_quantize_layer (any group size that divides C); no workspace, no dev_info. */
@@ -175,8 +178,8 @@ gptq_status_t gptq_rtn_layer(const void* W_fp16, int R, int C, int bits, int gro
  *
  * gptq_dequantize: the whole matrix back to fp16 (round-to-nearest-even of the fp32 product).
  *   W_out_fp16 [R x C] half.
- * gptq_matvec: y = W^ x for ONE fp16 vector x (batch-1 generation: "quantized-matrix
- *   full-precision-vector product" with dequantization on the fly, never materialising W^).
+ * gptq_matvec: y = W^ x for ONE fp16 vector x (batch-1 generation: packed matrix times
+ *   fp16 vector with dequantization on the fly, never materialising W^).
  *   x_fp16 [C] half, y [R] fp32; products exact, sums in fp32: per group the kernel forms
  *   sum q x and zero * sum x and combines them with the scale, so its rounding error is
  *   fp32-level relative to sum scale * (q + zero) * |x|.  Per-row grids and group sizes that
@@ -197,7 +200,7 @@ gptq_status_t gptq_matvec(const uint32_t* qweight, const float* scales, const fl
  *              is needed for the copies to overlap (pageable memory works, serialised).
  *   qweight_host, scales_host, zeros_host, loss_host: host outputs, shaped as in gptq_quantize_layer.
  *   info_host  int[2] (host): first non-OK device status of the three stages and its detail
- *              (for stage 1: of the last chunk).
+ *              (for stage 1: of the first chunk that reported one).
  *   dev_ws     DEVICE workspace of gptq_solve_layer_host_workspace_bytes() bytes: holds H, U, W,
  *              two X staging buffers, the outputs and the stages' own workspaces.
  * Unlike the per-stage calls this one SYNCHRONISES `stream` before returning (the results are on

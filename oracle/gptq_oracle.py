@@ -12,6 +12,7 @@ arrive as the transposed, token-major array Xt (m x C).  H = 2 X X^T.
 U is the upper-triangular matrix Algorithm 1 calls "Cholesky(H^-1)^T".
 
 Pins (tests/test_oracle_pins.py): diagonal H reduces to round-to-nearest;
+group grids equal the min-max grid of the trajectory-reconstructed current weights;
 block-size invariance; equivalence with the sequential OBQ recursion (Eq. 2,
 Eq. 3) for d_col <= 16; exhaustive search on d_col <= 8 at 2 bits never beaten;
 loss identity sum(E^2) = 2||dW X||^2 + lambda ||dW||^2; 2x2 closed form of U;
@@ -50,8 +51,8 @@ def hessian_accumulate(H: np.ndarray, Xt_bits: np.ndarray, chunk: int = 4096) ->
 
 # --------------------------------------------------------------------------- stage 2
 def dampen(H: np.ndarray, damp: float) -> tuple[np.ndarray, float]:
-    """H~ = H + lambda I, lambda = damp * mean(diag H)  (Section 3, Step 3:
-    "1% of the average diagonal value")."""
+    """H~ = H + lambda I with lambda = damp x the mean of H's diagonal (Section 3, Step 3; the
+    paper's setting is damp = 0.01)."""
     lam = float(damp) * float(np.mean(np.diag(H)))
     Ht = H.copy()
     Ht[np.diag_indices_from(Ht)] += lam
@@ -82,10 +83,10 @@ def field_bits_of(bits: int) -> int:
 
 
 def find_params(v: np.ndarray, bits: int, sym: bool):
-    """Min-max grid of each row of v (Section 5, Setup: "uniform per-row asymmetric
-    quantization on the min-max grid"; grouping applies the same to g consecutive
-    weights).  The range is widened to contain 0 so the zero-point is an integer
-    code (Section 5, Extreme Quantization: "2-bit zero point per group").  An
+    """Min-max grid of each row of v (Section 5, Setup: asymmetric uniform grid spanning the
+    row's minimum and maximum; grouping applies the same to g consecutive weights).
+    The range is widened to contain 0 so the zero-point is an integer code (Section 5,
+    Extreme Quantization, counts a b-bit zero-point per group in its storage figures).  An
     all-zero row gets [-1, 1].  Symmetric / ternary: half-range a = max|v|,
     scale = 2a/maxq, zero = (maxq+1)//2.  The scale is rounded to fp32 -- the
     precision it is returned in -- and used as that value.
@@ -114,50 +115,69 @@ def quant(w: np.ndarray, scale: np.ndarray, zero: np.ndarray, maxq: int):
 
 
 # --------------------------------------------------------------------------- stage 3
+def _fix_group_grid(W, j, g, bits, sym, scales, zeros):
+    """Column j opens a group: its g columns, in the state the error feedback of all earlier
+    columns has left them, decide the group's scale and zero-point (Section 5, grouping)."""
+    scales[:, j // g], zeros[:, j // g] = find_params(W[:, j:j + g], bits, sym)
+
+
+def _round_column_and_feed_back(W, U, j, stop, s, z, maxq):
+    """Algorithm 1, one pass of the inner loop for column j (all rows at once): pick the grid
+    point, form the scaled error (w - quant(w)) / U_jj, and subtract error x U[j, j:stop] from
+    columns j .. stop-1 (which also sets column j itself to its grid point).
+    Returns (codes, grid values, scaled errors) of the column."""
+    q, wq = quant(W[:, j], s, z, maxq)
+    err = (W[:, j] - wq) / U[j, j]
+    W[:, j:stop] -= np.outer(err, U[j, j:stop])
+    return q.astype(np.int32), wq, err
+
+
+def _push_block_errors(W, U, E, i, stop):
+    """Algorithm 1, last line of the outer loop: the block's errors reach every later column in
+    one product, W[:, stop:] -= E U[i:stop, stop:] (the lazy batch update of Section 3, Step 2)."""
+    W[:, stop:] -= E @ U[i:stop, stop:]
+
+
 def quantize_layer(W16: np.ndarray, U: np.ndarray, bits: int, group_size: int = 0,
                    sym: bool = False, block: int = 128):
     """Algorithm 1 with lazy batch updates of `block` columns.
 
     W16: (R x C) fp16 (promoted exactly to double); U: (C x C) upper factor.
-    Per-row grid (group_size <= 0): fixed from the original row before the
-    process (Section 2, "grid ... fixed before the process").  Grouped: at every
-    column j that starts a group the grid of W[:, j:j+g] is taken from the
-    weights as currently updated (Section 5, "always using the most current
-    updated weights").
+    One grid per row (group_size <= 0): decided once from the untouched row, before any column
+    is processed (Section 2 takes the grid as given in advance).  Grouped: decided per group
+    when its first column is reached, from the weights as updated up to then (Section 5).
     Returns dict(codes int32 RxC, scales RxG, zeros RxG, loss, W_hat RxC, E RxC)."""
     W = np.asarray(W16, dtype=np.float64).copy()
     R, C = W.shape
     maxq = maxq_of(bits)
-    g = group_size if group_size > 0 else C
+    grouped = group_size > 0
+    g = group_size if grouped else C
     if C % g != 0:
         raise ValueError("group size must divide d_col")
-    if group_size > 0 and g % block != 0 and block % g != 0:
-        # a group cut by a block end would see some columns before and some after
-        # the lazy update; groups and blocks must nest for "most current" to be defined
+    if grouped and g % block != 0 and block % g != 0:
+        # a group cut by a block end would see some of its columns before and some after the
+        # lazy update; only nested groups and blocks give "the weights as updated so far" a meaning
         raise ValueError("group size and block size must nest")
     G = C // g
-    Q = np.zeros((R, C))                        # quantized output (dequantized values)
+    W_hat = np.zeros((R, C))
     codes = np.zeros((R, C), dtype=np.int32)
     scales = np.zeros((R, G))
     zeros = np.zeros((R, G))
     E_all = np.zeros((R, C))
-    if group_size <= 0:
+    if not grouped:
         scales[:, 0], zeros[:, 0] = find_params(W, bits, sym)
     for i in range(0, C, block):
-        i2 = min(i + block, C)
-        E = np.zeros((R, i2 - i))               # block quantization errors
-        for j in range(i, i2):
-            if group_size > 0 and j % g == 0:
-                scales[:, j // g], zeros[:, j // g] = find_params(W[:, j:j + g], bits, sym)
-            s, z = scales[:, j // g], zeros[:, j // g]
-            q, Q[:, j] = quant(W[:, j], s, z, maxq)                     # quantize column
-            codes[:, j] = q.astype(np.int32)
-            E[:, j - i] = (W[:, j] - Q[:, j]) / U[j, j]                 # quantization error
-            W[:, j:i2] -= np.outer(E[:, j - i], U[j, j:i2])             # update weights in block
-        W[:, i2:] -= E @ U[i:i2, i2:]                                   # update all remaining weights
-        E_all[:, i:i2] = E
+        stop = min(i + block, C)
+        E = np.zeros((R, stop - i))
+        for j in range(i, stop):
+            if grouped and j % g == 0:
+                _fix_group_grid(W, j, g, bits, sym, scales, zeros)
+            codes[:, j], W_hat[:, j], E[:, j - i] = _round_column_and_feed_back(
+                W, U, j, stop, scales[:, j // g], zeros[:, j // g], maxq)
+        _push_block_errors(W, U, E, i, stop)
+        E_all[:, i:stop] = E
     loss = float(np.sum(E_all * E_all))
-    return dict(codes=codes, scales=scales, zeros=zeros, loss=loss, W_hat=Q, E=E_all)
+    return dict(codes=codes, scales=scales, zeros=zeros, loss=loss, W_hat=W_hat, E=E_all)
 
 
 def rtn(W16: np.ndarray, bits: int, group_size: int = 0, sym: bool = False):
@@ -219,7 +239,7 @@ def unpack_codes(words: np.ndarray, bits: int, C: int) -> np.ndarray:
 
 # --------------------------------------------------------------------------- using the packed weights
 def dequantize(codes: np.ndarray, scales: np.ndarray, zeros: np.ndarray, to_fp16: bool = False) -> np.ndarray:
-    """W^ = scale * (code - zero) per row and group (Section 5: "FP16 scale and ... zero point per group").
+    """W^ = scale * (code - zero) per row and group (Section 5, Extreme Quantization: one scale and one zero-point per group).
     to_fp16=False: the exact real-valued grid point in float64 (scales hold fp32 values).
     to_fp16=True: the stored-model reading -- one fp32 multiply, then round-to-nearest-even to fp16."""
     R, C = codes.shape

@@ -6,6 +6,7 @@ Function names and argument order follow include/gptq_b200.h.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
 import os
 
@@ -84,6 +85,18 @@ def _stream_ptr(stream):
     return ctypes.c_void_p(s.cuda_stream)
 
 
+@contextlib.contextmanager
+def _alloc_on(stream):
+    """Temporaries and outputs a wrapper creates (workspace, dev_info, result tensors) are allocated
+    and initialised with `stream` current, so torch's caching allocator orders their reuse, and their
+    zero-fill, on the stream the library's kernels run on -- not on whatever stream is current."""
+    if stream is None:
+        yield
+    else:
+        with torch.cuda.stream(stream):
+            yield
+
+
 def _check(t, dtype, name):
     if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype):
         raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
@@ -113,31 +126,33 @@ def gptq_quantize_workspace_bytes(R, C, bits, group_size, block):
 
 def gptq_hessian_accumulate(H, X, n_tokens=None, ws=None, dev_info=None, stream=None):
     """H += 2 X^T X for token-major bf16 X (n_tokens x C).  H: C x C fp32, zeroed by the caller first."""
-    _check(H, torch.float32, "H")
-    _check(X, torch.bfloat16, "X")
-    C = H.shape[0]
-    n = X.shape[0] if n_tokens is None else int(n_tokens)
-    ws = _ws(_lib.gptq_hessian_workspace_bytes(C, n), H.device, ws)
-    st = _lib.gptq_hessian_accumulate(H.data_ptr(), X.data_ptr(), n, C, ws.data_ptr(), ws.numel(),
-                                      None if dev_info is None else dev_info.data_ptr(), _stream_ptr(stream))
-    if st != OK:
-        raise GptqError(st, "gptq_hessian_accumulate")
-    return H
+    with _alloc_on(stream):
+        _check(H, torch.float32, "H")
+        _check(X, torch.bfloat16, "X")
+        C = H.shape[0]
+        n = X.shape[0] if n_tokens is None else int(n_tokens)
+        ws = _ws(_lib.gptq_hessian_workspace_bytes(C, n), H.device, ws)
+        st = _lib.gptq_hessian_accumulate(H.data_ptr(), X.data_ptr(), n, C, ws.data_ptr(), ws.numel(),
+                                          None if dev_info is None else dev_info.data_ptr(), _stream_ptr(stream))
+        if st != OK:
+            raise GptqError(st, "gptq_hessian_accumulate")
+        return H
 
 
 def gptq_prepare_hinv(H, damp=0.01, U=None, ws=None, dev_info=None, stream=None):
     """U = Cholesky((H + damp*mean(diag H) I)^-1)^T.  Returns (U, dev_info); dev_info is read by the caller after a sync."""
-    _check(H, torch.float32, "H")
-    C = H.shape[0]
-    U = torch.empty_like(H) if U is None else U
-    _check(U, torch.float32, "U")
-    dev_info = torch.zeros(2, dtype=torch.int32, device=H.device) if dev_info is None else dev_info
-    ws = _ws(_lib.gptq_prepare_hinv_workspace_bytes(C), H.device, ws)
-    st = _lib.gptq_prepare_hinv(H.data_ptr(), float(damp), C, U.data_ptr(), ws.data_ptr(), ws.numel(),
-                                dev_info.data_ptr(), _stream_ptr(stream))
-    if st != OK:
-        raise GptqError(st, "gptq_prepare_hinv")
-    return U, dev_info
+    with _alloc_on(stream):
+        _check(H, torch.float32, "H")
+        C = H.shape[0]
+        U = torch.empty_like(H) if U is None else U
+        _check(U, torch.float32, "U")
+        dev_info = torch.zeros(2, dtype=torch.int32, device=H.device) if dev_info is None else dev_info
+        ws = _ws(_lib.gptq_prepare_hinv_workspace_bytes(C), H.device, ws)
+        st = _lib.gptq_prepare_hinv(H.data_ptr(), float(damp), C, U.data_ptr(), ws.data_ptr(), ws.numel(),
+                                    dev_info.data_ptr(), _stream_ptr(stream))
+        if st != OK:
+            raise GptqError(st, "gptq_prepare_hinv")
+        return U, dev_info
 
 
 PREPARE_HINV_STATIC_MAX_C = 1024
@@ -150,38 +165,40 @@ def gptq_prepare_hinv_static(H, damp=0.01, U=None, dev_info=None, stream=None):
     calls that could overlap on the GPU must be put on one stream.  The first call on a device does a
     one-time address look-up and should not happen inside a stream capture.  U and dev_info are the
     caller's (created here with torch only when not passed in)."""
-    _check(H, torch.float32, "H")
-    C = H.shape[0]
-    U = torch.empty_like(H) if U is None else U
-    _check(U, torch.float32, "U")
-    dev_info = torch.zeros(2, dtype=torch.int32, device=H.device) if dev_info is None else dev_info
-    st = _lib.gptq_prepare_hinv_static(H.data_ptr(), float(damp), C, U.data_ptr(), dev_info.data_ptr(), _stream_ptr(stream))
-    if st != OK:
-        raise GptqError(st, "gptq_prepare_hinv_static")
-    return U, dev_info
+    with _alloc_on(stream):
+        _check(H, torch.float32, "H")
+        C = H.shape[0]
+        U = torch.empty_like(H) if U is None else U
+        _check(U, torch.float32, "U")
+        dev_info = torch.zeros(2, dtype=torch.int32, device=H.device) if dev_info is None else dev_info
+        st = _lib.gptq_prepare_hinv_static(H.data_ptr(), float(damp), C, U.data_ptr(), dev_info.data_ptr(), _stream_ptr(stream))
+        if st != OK:
+            raise GptqError(st, "gptq_prepare_hinv_static")
+        return U, dev_info
 
 
 def gptq_quantize_layer(W, U, bits, group_size=0, sym=False, block=128, ws=None, dev_info=None, stream=None):
     """Algorithm 1 on fp16 W (R x C) with U from gptq_prepare_hinv.
     Returns dict(qweight uint32 [R, C*f/32] (as int32 tensor), scales [R,G], zeros [R,G], loss double[1], dev_info)."""
-    _check(W, torch.float16, "W")
-    _check(U, torch.float32, "U")
-    R, C = W.shape
-    G = C // group_size if group_size > 0 else 1
-    f = field_bits(bits)
-    dev = W.device
-    qweight = torch.empty((R, C * f // 32), dtype=torch.int32, device=dev)
-    scales = torch.empty((R, G), dtype=torch.float32, device=dev)
-    zeros = torch.empty((R, G), dtype=torch.float32, device=dev)
-    loss = torch.zeros(1, dtype=torch.float64, device=dev)
-    dev_info = torch.zeros(2, dtype=torch.int32, device=dev) if dev_info is None else dev_info
-    ws = _ws(_lib.gptq_quantize_workspace_bytes(R, C, bits, group_size, block), dev, ws)
-    st = _lib.gptq_quantize_layer(W.data_ptr(), U.data_ptr(), R, C, bits, group_size, int(bool(sym)), block,
-                                  qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), loss.data_ptr(),
-                                  ws.data_ptr(), ws.numel(), dev_info.data_ptr(), _stream_ptr(stream))
-    if st != OK:
-        raise GptqError(st, "gptq_quantize_layer")
-    return dict(qweight=qweight, scales=scales, zeros=zeros, loss=loss, dev_info=dev_info)
+    with _alloc_on(stream):
+        _check(W, torch.float16, "W")
+        _check(U, torch.float32, "U")
+        R, C = W.shape
+        G = C // group_size if group_size > 0 else 1
+        f = field_bits(bits)
+        dev = W.device
+        qweight = torch.empty((R, C * f // 32), dtype=torch.int32, device=dev)
+        scales = torch.empty((R, G), dtype=torch.float32, device=dev)
+        zeros = torch.empty((R, G), dtype=torch.float32, device=dev)
+        loss = torch.zeros(1, dtype=torch.float64, device=dev)
+        dev_info = torch.zeros(2, dtype=torch.int32, device=dev) if dev_info is None else dev_info
+        ws = _ws(_lib.gptq_quantize_workspace_bytes(R, C, bits, group_size, block), dev, ws)
+        st = _lib.gptq_quantize_layer(W.data_ptr(), U.data_ptr(), R, C, bits, group_size, int(bool(sym)), block,
+                                      qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), loss.data_ptr(),
+                                      ws.data_ptr(), ws.numel(), dev_info.data_ptr(), _stream_ptr(stream))
+        if st != OK:
+            raise GptqError(st, "gptq_quantize_layer")
+        return dict(qweight=qweight, scales=scales, zeros=zeros, loss=loss, dev_info=dev_info)
 
 
 def gptq_solve_layer_host_workspace_bytes(R, C, n_tokens, bits, group_size, block):
@@ -221,39 +238,42 @@ def gptq_solve_layer_host(W_host, X_host, bits, group_size=0, sym=False, block=1
 
 def gptq_rtn_layer(W, bits, group_size=0, sym=False, stream=None):
     """Round-to-nearest on the solver's grid, no error feedback.  Returns dict(qweight, scales, zeros)."""
-    _check(W, torch.float16, "W")
-    R, C = W.shape
-    G = C // group_size if group_size > 0 else 1
-    qweight = torch.empty((R, C * field_bits(bits) // 32), dtype=torch.int32, device=W.device)
-    scales = torch.empty((R, G), dtype=torch.float32, device=W.device)
-    zeros = torch.empty((R, G), dtype=torch.float32, device=W.device)
-    st = _lib.gptq_rtn_layer(W.data_ptr(), R, C, bits, group_size, int(bool(sym)), qweight.data_ptr(), scales.data_ptr(),
-                             zeros.data_ptr(), _stream_ptr(stream))
-    if st != OK:
-        raise GptqError(st, "gptq_rtn_layer")
-    return dict(qweight=qweight, scales=scales, zeros=zeros)
+    with _alloc_on(stream):
+        _check(W, torch.float16, "W")
+        R, C = W.shape
+        G = C // group_size if group_size > 0 else 1
+        qweight = torch.empty((R, C * field_bits(bits) // 32), dtype=torch.int32, device=W.device)
+        scales = torch.empty((R, G), dtype=torch.float32, device=W.device)
+        zeros = torch.empty((R, G), dtype=torch.float32, device=W.device)
+        st = _lib.gptq_rtn_layer(W.data_ptr(), R, C, bits, group_size, int(bool(sym)), qweight.data_ptr(), scales.data_ptr(),
+                                 zeros.data_ptr(), _stream_ptr(stream))
+        if st != OK:
+            raise GptqError(st, "gptq_rtn_layer")
+        return dict(qweight=qweight, scales=scales, zeros=zeros)
 
 
 def gptq_dequantize(qweight, scales, zeros, C, bits, group_size=0, out=None, stream=None):
     """Packed codes -> fp16 weights W^ = scales * (code - zeros)  [R x C]."""
-    _check(qweight, torch.int32, "qweight"); _check(scales, torch.float32, "scales"); _check(zeros, torch.float32, "zeros")
-    R = qweight.shape[0]
-    out = torch.empty((R, C), dtype=torch.float16, device=qweight.device) if out is None else out
-    st = _lib.gptq_dequantize(qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), R, C, bits, group_size,
-                              out.data_ptr(), _stream_ptr(stream))
-    if st != OK:
-        raise GptqError(st, "gptq_dequantize")
-    return out
+    with _alloc_on(stream):
+        _check(qweight, torch.int32, "qweight"); _check(scales, torch.float32, "scales"); _check(zeros, torch.float32, "zeros")
+        R = qweight.shape[0]
+        out = torch.empty((R, C), dtype=torch.float16, device=qweight.device) if out is None else out
+        st = _lib.gptq_dequantize(qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), R, C, bits, group_size,
+                                  out.data_ptr(), _stream_ptr(stream))
+        if st != OK:
+            raise GptqError(st, "gptq_dequantize")
+        return out
 
 
 def gptq_matvec(qweight, scales, zeros, x, C, bits, group_size=0, out=None, stream=None):
     """y = W^ x for one fp16 vector x of length C, dequantizing on the fly; y is fp32 [R]."""
-    _check(qweight, torch.int32, "qweight"); _check(scales, torch.float32, "scales"); _check(zeros, torch.float32, "zeros")
-    _check(x, torch.float16, "x")
-    R = qweight.shape[0]
-    out = torch.empty(R, dtype=torch.float32, device=qweight.device) if out is None else out
-    st = _lib.gptq_matvec(qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), x.data_ptr(), R, C, bits, group_size,
-                          out.data_ptr(), _stream_ptr(stream))
-    if st != OK:
-        raise GptqError(st, "gptq_matvec")
-    return out
+    with _alloc_on(stream):
+        _check(qweight, torch.int32, "qweight"); _check(scales, torch.float32, "scales"); _check(zeros, torch.float32, "zeros")
+        _check(x, torch.float16, "x")
+        R = qweight.shape[0]
+        out = torch.empty(R, dtype=torch.float32, device=qweight.device) if out is None else out
+        st = _lib.gptq_matvec(qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), x.data_ptr(), R, C, bits, group_size,
+                              out.data_ptr(), _stream_ptr(stream))
+        if st != OK:
+            raise GptqError(st, "gptq_matvec")
+        return out

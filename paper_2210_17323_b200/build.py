@@ -19,7 +19,7 @@ SYNTH = os.path.join(HERE, "synth")
 LIB = os.path.join(HERE, "lib")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-         "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
+         "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"] + os.environ.get("GPTQ_NVCC_EXTRA", "").split()
 
 SOLVER_SOURCES = ["api.cu", "hessian.cu", "hessian_umma.cu", "hinv.cu", "quantize.cu", "solve_host.cu", "rtn.cu", "inference.cu"]
 

@@ -443,6 +443,7 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
   //   C4  U~[row block J-1, J] = A[..] V^T -> U and F      (after B1)
   // C1 of panel J needs row block J of every later panel: panel J+1's comes from its C4 (same stream),
   // the others from B2 of panels >= J+2, which had the whole chain of panel J+1 to finish.
+  auto phase1 = [&]() -> gptq_status_t {
   for (int J = n_outer - 1; J >= 0; --J) {
     const int j0 = J * kNB2, wj = (C - j0 < kNB2) ? C - j0 : kNB2, rows_p = j0 + wj;
     const int K = C - rows_p;                       // later columns
@@ -528,10 +529,18 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
     }
     GPTQ_CUDA_TRY(cudaEventRecord(as->c4[J], s));
   }
+  return GPTQ_OK;
+  };
+  st = phase1();
   if (outer) {
-    GPTQ_CUDA_TRY(cudaEventRecord(as->join, sb));
-    GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, as->join, 0));
+    // Join the internal streams into the caller's stream whether or not phase 1 was enqueued completely:
+    // an error return must not leave work on them that the caller's stream does not wait for (inside a
+    // stream capture that would invalidate the capture; outside, later calls share these streams).
+    const cudaError_t j1 = cudaEventRecord(as->join, sb), j2 = cudaStreamWaitEvent(s, as->join, 0);
+    const cudaError_t j3 = cudaEventRecord(as->side_done, ss), j4 = cudaStreamWaitEvent(s, as->side_done, 0);
+    if (st == GPTQ_OK && (j1 != cudaSuccess || j2 != cudaSuccess || j3 != cudaSuccess || j4 != cudaSuccess)) st = GPTQ_ERR_CUDA;
   }
+  if (st != GPTQ_OK) return st;
 
   // Phase 2: U = U~^-1, outer panel by outer panel, in place.  The diagonal blocks are already inverted;
   // rows above them: U[0:j0, J] = -U[0:j0, 0:j0] * (U~[0:j0, J] * V_JJ).

@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
       for (int o = 0; o < 4; ++o) {
         const int jj = 4 * m + o;
         const double wj = __shfl_sync(0xffffffffu, w[0], o, 4);
-        // quantize column: rne(w / scale).  The quotient is formed with the reciprocal; only when it lands within
+        // code of this weight: rne(w / scale).  The quotient is formed with the reciprocal; only when it lands within
         // 1e-6 of a tie (where the reciprocal's last-bit error could change the rounding) is the division done.
         const double tq = wj * rscale;
         double q = rint(tq);
@@ -220,14 +220,14 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
         q += zero;
         q = fmin(fmax(q, 0.0), maxq);
         const double wq = scale * (q - zero);
-        const double e = (wj - wq) * rdiag[jj];                // quantization error (w - q) / U_jj
+        const double e = (wj - wq) * rdiag[jj];                // scaled error (w - q) / U_jj
         if (l == o) esm[jj * kRPB + rl] = (float)e;
         loss += e * e;
         bad |= !isfinite(e);
         packed |= (uint32_t)q << (8 * o);
         const double* urow = Us + jj * B + j0 + 4 * m + l;
 #pragma unroll
-        for (int mm = 0; mm < kSB / 4; ++mm)                   // update weights in block (own columns > jj)
+        for (int mm = 0; mm < kSB / 4; ++mm)                   // immediate feedback onto own columns > jj
           if (mm < kSB / 4 - m && (mm > 0 || l > o)) w[mm] -= e * urow[4 * mm];
       }
       if ((m >> 1) == l) { if (m & 1) c1 = packed; else c0 = packed; }

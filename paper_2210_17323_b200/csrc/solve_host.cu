@@ -47,6 +47,12 @@ HostWs carve_host(void* ws, int R, int C, int64_t n_tokens, int bits, int group_
   return o;
 }
 
+// First error wins across the Hessian calls of one solve: each call reports into `src` (which it clears
+// first); a non-OK report is moved into `dst` unless `dst` already holds one.
+__global__ void fold_info_kernel(int* __restrict__ dst, const int* __restrict__ src) {
+  if (dst[0] == GPTQ_OK && src[0] != GPTQ_OK) { dst[1] = src[1]; dst[0] = src[0]; }
+}
+
 struct StreamGuard {
   cudaStream_t s = nullptr;
   cudaEvent_t loaded[2] = {nullptr, nullptr}, freed[2] = {nullptr, nullptr}, w_done = nullptr;
@@ -67,6 +73,15 @@ extern "C" size_t gptq_solve_layer_host_workspace_bytes(int R, int C, int64_t n_
   if (gptq_quantize_workspace_bytes(R, C, bits, group_size, block) == 0) return 0;
   return carve_host(nullptr, R, C, n_tokens, bits, group_size, block).bytes;
 }
+
+namespace gptq {
+namespace {
+gptq_status_t solve_layer_host_enqueue(const HostWs& w, StreamGuard& g, cudaStream_t s, const void* W_fp16_host,
+                                       const void* X_bf16_host, int64_t n_tokens, int R, int C, float damp, int bits,
+                                       int group_size, int sym, int block, uint32_t* qweight_host, float* scales_host,
+                                       float* zeros_host, double* loss_host, int* info8_host);
+}  // namespace
+}  // namespace gptq
 
 extern "C" gptq_status_t gptq_solve_layer_host(const void* W_fp16_host, const void* X_bf16_host, int64_t n_tokens,
                                                int R, int C, float damp, int bits, int group_size, int sym, int block,
@@ -90,6 +105,26 @@ extern "C" gptq_status_t gptq_solve_layer_host(const void* W_fp16_host, const vo
   }
   GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&g.w_done, cudaEventDisableTiming));
 
+  int info[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  gptq_status_t st = solve_layer_host_enqueue(w, g, s, W_fp16_host, X_bf16_host, n_tokens, R, C, damp, bits, group_size,
+                                              sym, block, qweight_host, scales_host, zeros_host, loss_host, info);
+  // Whatever happened, nothing of this call may still be in flight when it returns: the caller may free the host
+  // buffers the copy stream reads, and the guard destroys that stream and its events.
+  const cudaError_t e1 = cudaStreamSynchronize(s), e2 = cudaStreamSynchronize(g.s);
+  if (st != GPTQ_OK) return st;
+  if (e1 != cudaSuccess || e2 != cudaSuccess) return GPTQ_ERR_CUDA;
+  info_host[0] = GPTQ_OK; info_host[1] = 0;
+  for (int i = 0; i < 3; ++i)
+    if (info[2 * i] != GPTQ_OK) { info_host[0] = info[2 * i]; info_host[1] = info[2 * i + 1]; break; }
+  return GPTQ_OK;
+}
+
+namespace gptq {
+namespace {
+gptq_status_t solve_layer_host_enqueue(const HostWs& w, StreamGuard& g, cudaStream_t s, const void* W_fp16_host,
+                                       const void* X_bf16_host, int64_t n_tokens, int R, int C, float damp, int bits,
+                                       int group_size, int sym, int block, uint32_t* qweight_host, float* scales_host,
+                                       float* zeros_host, double* loss_host, int* info8_host) {
   GPTQ_CUDA_TRY(cudaMemsetAsync(w.H, 0, (size_t)C * C * sizeof(float), s));
   GPTQ_CUDA_TRY(cudaMemsetAsync(w.info, 0, 8 * sizeof(int), s));
   const __nv_bfloat16* Xh = static_cast<const __nv_bfloat16*>(X_bf16_host);
@@ -106,8 +141,11 @@ extern "C" gptq_status_t gptq_solve_layer_host(const void* W_fp16_host, const vo
       GPTQ_CUDA_TRY(cudaEventRecord(g.w_done, g.s));
     }
     GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, g.loaded[b], 0));
-    st = gptq_hessian_accumulate(w.H, w.X[b], nt, C, w.stage_ws, w.stage_ws_bytes, w.info, s);
+    // every chunk reports into the spare slot info[6..7]; the first non-OK report is kept in info[0..1]
+    st = gptq_hessian_accumulate(w.H, w.X[b], nt, C, w.stage_ws, w.stage_ws_bytes, w.info + 6, s);
     if (st != GPTQ_OK) return st;
+    fold_info_kernel<<<1, 1, 0, s>>>(w.info, w.info + 6);
+    GPTQ_LAUNCH_CHECK();
     GPTQ_CUDA_TRY(cudaEventRecord(g.freed[b], s));
   }
   GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, g.w_done, 0));
@@ -117,16 +155,12 @@ extern "C" gptq_status_t gptq_solve_layer_host(const void* W_fp16_host, const vo
                            w.stage_ws, w.stage_ws_bytes, w.info + 4, s);
   if (st != GPTQ_OK) return st;
   const int G = group_size > 0 ? C / group_size : 1;
-  int info[8];
   GPTQ_CUDA_TRY(cudaMemcpyAsync(qweight_host, w.qweight, (size_t)R * (C * field_bits_h(bits) / 32) * 4, cudaMemcpyDeviceToHost, s));
   GPTQ_CUDA_TRY(cudaMemcpyAsync(scales_host, w.scales, (size_t)R * G * 4, cudaMemcpyDeviceToHost, s));
   GPTQ_CUDA_TRY(cudaMemcpyAsync(zeros_host, w.zeros, (size_t)R * G * 4, cudaMemcpyDeviceToHost, s));
   GPTQ_CUDA_TRY(cudaMemcpyAsync(loss_host, w.loss, sizeof(double), cudaMemcpyDeviceToHost, s));
-  GPTQ_CUDA_TRY(cudaMemcpyAsync(info, w.info, sizeof(info), cudaMemcpyDeviceToHost, s));
-  GPTQ_CUDA_TRY(cudaStreamSynchronize(s));
-  GPTQ_CUDA_TRY(cudaStreamSynchronize(g.s));
-  info_host[0] = GPTQ_OK; info_host[1] = 0;
-  for (int i = 0; i < 3; ++i)
-    if (info[2 * i] != GPTQ_OK) { info_host[0] = info[2 * i]; info_host[1] = info[2 * i + 1]; break; }
+  GPTQ_CUDA_TRY(cudaMemcpyAsync(info8_host, w.info, 8 * sizeof(int), cudaMemcpyDeviceToHost, s));
   return GPTQ_OK;
 }
+}  // namespace
+}  // namespace gptq

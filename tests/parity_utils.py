@@ -44,3 +44,55 @@ def check_quantize_outputs(gpu, ref, W16, bits, C, H=None, min_identical=TOL_COD
     assert abs(loss - ref["loss"]) <= TOL_RECON * ref["loss"] + 1e-30, f"loss {loss} vs {ref['loss']}"
     out["loss_ratio"] = loss / ref["loss"] if ref["loss"] else 1.0
     return out
+
+
+# ---- checks that work at any size (H and U are CUDA tensors; torch is imported lazily) -----------------
+def check_hessian_sampled(L, H, n_cols=24):
+    """Sampled entries of H against the definition 2 sum_t x_ti x_tj, from host-generated columns of X."""
+    import torch
+    r = np.random.default_rng(5 + L.C)
+    cols = np.unique(np.concatenate([r.integers(0, L.C, n_cols), [0, L.C - 1, 127, 128, 255, 256]]))
+    sc = L.scales()
+    Xc = np.concatenate([O.bf16_bits_to_f64(L.x_bits(t0, min(t0 + 32768, L.n_tokens), cols=cols, scales=sc))
+                         for t0 in range(0, L.n_tokens, 32768)])
+    ref = 2.0 * (Xc.T @ Xc)
+    idx = torch.from_numpy(cols).cuda()
+    got = H[idx][:, idx].cpu().numpy().astype(np.float64)
+    fro = float(np.linalg.norm(got - ref) / np.linalg.norm(ref))
+    assert fro <= TOL_H_FRO, fro
+    assert np.abs(got - ref).max() <= 1e-5 * np.abs(ref).max()
+    d = np.diag(ref)
+    assert (np.abs(np.diag(got) - d) <= 5e-6 * d).all()
+    return fro
+
+
+def check_factor_on_device(H, U, damp, k_tail=512, n_probe=4, blk=2048):
+    """U upper with positive diagonal; probe residual of U^T U = (H + lambda I)^-1 in fp64 (device, row blocks);
+    last rows of U against the oracle's literal route on the trailing principal block of H~."""
+    import torch
+    C = H.shape[0]
+    assert bool((torch.diagonal(U) > 0).all())
+    for r0 in range(0, C, blk):                              # strict lower triangle is exactly zero
+        r1 = min(C, r0 + blk)
+        assert not bool(torch.tril(U[r0:r1, :r1], diagonal=r0 - 1).any()), r0
+    lam = damp * float(torch.diagonal(H).double().mean().item())
+    g = torch.Generator(device="cuda").manual_seed(6)
+    z = torch.randn((C, n_probe), dtype=torch.float64, device="cuda", generator=g)
+    y = torch.empty_like(z)
+    for r0 in range(0, C, blk):
+        y[r0:r0 + blk] = U[r0:r0 + blk].double() @ z
+    w = torch.zeros_like(z)
+    for r0 in range(0, C, blk):
+        w += U[r0:r0 + blk].double().T @ y[r0:r0 + blk]
+    v = lam * w
+    for r0 in range(0, C, blk):
+        v[r0:r0 + blk] += H[r0:r0 + blk].double() @ w
+    res = float(((v - z).norm(dim=0) / z.norm(dim=0)).max().item())
+    assert res <= 5e-5, res
+    Ht_tail = H[C - k_tail:, C - k_tail:].cpu().numpy().astype(np.float64)
+    Ht_tail[np.diag_indices_from(Ht_tail)] += lam
+    Uref = O.cholesky_inverse_upper(Ht_tail)
+    Ut = U[C - k_tail:, C - k_tail:].cpu().numpy().astype(np.float64)
+    err = float((np.linalg.norm(Ut - Uref, axis=1) / np.linalg.norm(Uref, axis=1)).max())
+    assert err <= 1e-4, err
+    return res, err

@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 
 from oracle import gptq_oracle as O
 from paper_2210_17323_b200.synth import workloads as WL
-from tests.parity_utils import check_quantize_outputs
+from tests.parity_utils import check_factor_on_device, check_hessian_sampled, check_quantize_outputs
 
 
 @pytest.fixture(scope="module")
@@ -111,6 +111,8 @@ def test_config4_block_size_sweep_full_size(B):
     W = D.fill_w(L)
     torch.cuda.synchronize()
     assert info.tolist()[0] == 0
+    check_hessian_sampled(L, H)
+    check_factor_on_device(H, U, wl.damp)
     rows = np.sort(np.random.default_rng(8).choice(L.R, 16, replace=False))
     W16 = L.w(rows=rows)
     U64 = U.cpu().numpy().astype(np.float64)
@@ -131,4 +133,7 @@ def test_config4_block_size_sweep_full_size(B):
             gpu = dict(qweight=qw[rows].cpu().numpy(), scales=out["scales"][rows].cpu().numpy(),
                        zeros=out["zeros"][rows].cpu().numpy(), loss=ref["loss"])
             figs = check_quantize_outputs(gpu, ref, W16, g.bits, L.C)
+            # the layer's loss against the sampled rows' share of it (rows are i.i.d.)
+            per_row = ref["loss"] / len(rows)
+            assert 0.5 * per_row * L.R <= out["loss"].item() <= 2.0 * per_row * L.R
             print(f"c4 bits={g.bits} B={blk}:", figs, "words identical to B=32:", 1.0 if base is qw else same)

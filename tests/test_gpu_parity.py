@@ -244,6 +244,37 @@ def test_midsize_end_to_end_grouped(B, D):
     print("midsize end-to-end:", figs)
 
 
+def test_calls_on_a_non_current_stream_with_library_made_temporaries(B):
+    """Stages 2 and 3 launched on a stream that is NOT torch's current stream, with the wrapper creating the
+    workspace, dev_info and outputs itself, while the current stream keeps allocating and overwriting memory:
+    the temporaries must be ordered on the launch stream, so the results still match the oracle."""
+    C, R = 1280, 96                                  # two outer panels: stage 2 also uses its internal streams
+    L = _layer(R, C, 3000, cfg=5, kind="k")
+    W16 = L.w()
+    H64 = O.hessian_accumulate(np.zeros((C, C)), L.x_bits())
+    H32 = H64.astype(np.float32)
+    Uref = O.cholesky_inverse_upper(O.dampen(H32.astype(np.float64), 0.01)[0])
+    Hd, Wd = torch.from_numpy(H32).cuda(), torch.from_numpy(W16).cuda()
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    need = max(B.gptq_prepare_hinv_workspace_bytes(C), B.gptq_quantize_workspace_bytes(R, C, 3, 128, 128))
+    for _ in range(3):
+        U, info = B.gptq_prepare_hinv(Hd, 0.01, stream=side)
+        junk = [torch.full((need // 4 + 64,), float("nan"), device="cuda") for _ in range(3)]   # current stream
+        out = B.gptq_quantize_layer(Wd, U, 3, 128, False, 128, stream=side)
+        junk += [torch.full((need // 4 + 64,), float("nan"), device="cuda") for _ in range(3)]
+        junk += [torch.full((16,), -1, dtype=torch.int32, device="cuda") for _ in range(64)]
+        side.synchronize()
+        torch.cuda.synchronize()
+        del junk
+        assert info.tolist() == [0, 0] and out["dev_info"].tolist()[0] == 0
+        assert rel_fro(U.cpu().numpy(), Uref) <= TOL_U_FRO
+        ref = O.quantize_layer(W16, U.cpu().numpy().astype(np.float64), 3, 128, False, 128)
+        gpu = dict(qweight=out["qweight"].cpu().numpy(), scales=out["scales"].cpu().numpy(),
+                   zeros=out["zeros"].cpu().numpy(), loss=out["loss"].item())
+        check_quantize_outputs(gpu, ref, W16, 3, C, H64)
+
+
 def test_solve_layer_from_host_buffers(B):
     """The host-buffer entry point (X streamed in chunks, results copied back) against the oracle."""
     L = _layer(96, 512, 5000, cfg=5, kind="o")

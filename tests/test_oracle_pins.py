@@ -48,7 +48,7 @@ def test_hessian_integer_exact_and_additive():
     H = O.hessian_accumulate(np.zeros((C, C)), bits)
     exact = 2 * (Xi.T.astype(np.int64) @ Xi.astype(np.int64))
     assert np.array_equal(H, exact.astype(np.float64))
-    # additive over any chunking of the tokens ("accumulate the layer-Hessians", Section 5 Setup)
+    # additive over any chunking of the tokens (Section 5 Setup: Hessians are summed over batches)
     H2 = np.zeros((C, C))
     for a, b in ((0, 7), (7, 128), (128, 300)):
         O.hessian_accumulate(H2, bits[a:b])
@@ -312,6 +312,46 @@ def test_error_feedback_beats_rtn_on_correlated_inputs():
     out = O.quantize_layer(W, U, 4, 0, False, block=16)
     _, What_rtn = O.rtn(W, 4, 0, False)
     assert O.reconstruction_error(W, out["W_hat"], H) < 0.5 * O.reconstruction_error(W, What_rtn, H)
+
+
+# ------------------------------------------------------------------ grouped grids come from the UPDATED weights (Section 5)
+@pytest.mark.parametrize("bits,group,block", [(4, 16, 16), (3, 16, 32), (2, 32, 16), (3, 8, 64)])
+def test_group_grid_is_taken_from_current_weights(bits, group, block):
+    """Section 5 (grouping): a group's grid is fixed when its first column is reached, from the
+    weights as the error feedback of all earlier columns has left them -- not from the original
+    weights.  By the trajectory identity W0 - W^ = E U (pinned above), the weights of group
+    [j, j+g) at that moment are W0[:, j:j+g] - E[:, :j] U[:j, j:j+g]; the returned scale and
+    zero-point must be the min-max grid of THAT slice (endpoints checked by brute force over the
+    slice), and on strongly correlated inputs they must differ from the original slice's grid."""
+    r = RNG(31)
+    R, C, m = 12, 64, 400
+    Z = r.normal(size=(m, 8)) @ r.normal(size=(8, C)) + 0.05 * r.normal(size=(m, C))
+    Xt = _bf16_bits(Z)
+    W = (r.normal(size=(R, C)) * 0.02).astype(np.float16)
+    H = O.hessian_accumulate(np.zeros((C, C)), Xt)
+    U = O.cholesky_inverse_upper(O.dampen(H, 0.01)[0])
+    out = O.quantize_layer(W, U, bits, group, False, block=block)
+    W0 = W.astype(np.float64)
+    maxq = 2 ** bits - 1
+    differs = 0
+    for j in range(0, C, group):
+        gi = j // group
+        cur = W0[:, j:j + group] - out["E"][:, :j] @ U[:j, j:j + group]
+        s, z = out["scales"][:, gi], out["zeros"][:, gi]
+        for rr in range(R):
+            lo = min(min(cur[rr]), 0.0)                  # brute force over the slice
+            hi = max(max(cur[rr]), 0.0)
+            assert s[rr] == np.float64(np.float32((hi - lo) / maxq)), (j, rr)
+            # the integer zero-point puts the grid's lower end within half a step of lo
+            assert z[rr] == int(z[rr]) and 0 <= z[rr] <= maxq
+            assert abs(s[rr] * (0 - z[rr]) - lo) <= 0.5 * s[rr] * (1 + 1e-9)
+            lo0 = min(min(W0[rr, j:j + group]), 0.0)
+            hi0 = max(max(W0[rr, j:j + group]), 0.0)
+            if j > 0 and np.float32((hi0 - lo0) / maxq) != np.float32(s[rr]):
+                differs += 1
+    # the feedback moves the weights by a good fraction of a step here, so nearly every later
+    # group's range differs from the original slice's: a solver that took the grids from W0 fails
+    assert differs >= 0.9 * R * (C // group - 1)
 
 
 # ------------------------------------------------------------------ P8: packed layout

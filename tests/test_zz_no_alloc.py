@@ -13,6 +13,7 @@ import pytest
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
+from oracle import gptq_oracle as O
 from paper_2210_17323_b200.synth import workloads as WL
 from tests.parity_utils import TOL_U_FRO, rel_fro
 
@@ -47,6 +48,9 @@ def test_static_variant_matches_workspace_variant_twice_in_a_row(B):
         assert torch.cuda.memory_allocated() == held      # the call itself took nothing from torch's pool
         assert info.tolist() == info_ref.tolist() == [0, 0]
         assert rel_fro(U.cpu().numpy(), U_ref.cpu().numpy()) <= TOL_U_FRO
+        # and directly against the oracle's factor of the same (fp32) Hessian
+        U_oracle = O.cholesky_inverse_upper(O.dampen(H.cpu().numpy().astype(np.float64), 0.01)[0])
+        assert rel_fro(U.cpu().numpy(), U_oracle) <= TOL_U_FRO
 
 
 def test_static_variant_rejects_sizes_beyond_its_scratch(B):
