@@ -81,11 +81,7 @@ struct HessPairTraits {
   static constexpr int A_BYTES = 2 * BOX_BYTES;           // 16 KB: this CTA's 128 rows
   static constexpr int B_BYTES = 2 * BOX_BYTES;           // 16 KB: this CTA's 128 of the 256 columns
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 32 KB per CTA
-#ifdef GPTQ_EXP_CHUNK
-  static constexpr int CHUNK_KB = GPTQ_EXP_CHUNK;
-#else
   static constexpr int CHUNK_KB = 8;
-#endif
   struct Maps { CUtensorMap x; };
 
   static __device__ __forceinline__ void prefetch(const Maps& m) { umma::prefetch_tmap(&m.x); }
@@ -93,10 +89,8 @@ struct HessPairTraits {
     const int y = kb * BK;
 #pragma unroll
     for (int j = 0; j < 2; ++j) umma::tma_load_2d_pair(s + j * BOX_BYTES, &m.x, m0 + 64 * j, y, bar);
-#ifndef GPTQ_EXP_SKIP_B
 #pragma unroll
     for (int j = 0; j < 2; ++j) umma::tma_load_2d_pair(s + A_BYTES + j * BOX_BYTES, &m.x, n0 + 64 * j, y, bar);
-#endif
   }
   static __device__ __forceinline__ void mma(uint32_t d_tmem, uint32_t s, bool fresh) {
     using namespace umma;
@@ -104,11 +98,7 @@ struct HessPairTraits {
 #pragma unroll
     for (int k = 0; k < BK / 16; ++k) {
       const uint64_t da = make_desc_sw128(s + k * 2048, BOX_BYTES, 1024);
-#ifdef GPTQ_EXP_SKIP_B
-      const uint64_t db = da;
-#else
       const uint64_t db = make_desc_sw128(s + A_BYTES + k * 2048, BOX_BYTES, 1024);
-#endif
       mma_f16_pair(d_tmem, da, db, idesc, (fresh && k == 0) ? 0u : 1u);
     }
   }

@@ -10,11 +10,17 @@
 //   * Inside an outer block the paper's loop runs with the caller's block size B: the in-block
 //     kernel quantizes B columns with immediate error feedback, then the block's errors are
 //     pushed onto the remaining columns of the outer block.
-//   * Working weights of the current outer block are fp64; E is kept in fp32 (as a tf32 hi/lo
-//     pair); update sums come from the tensor cores with fp32 accuracy (3xTF32).  Each weight therefore meets one rounding at fp32 level (its update sum)
-//     instead of one per preceding block.
+//   * Working weights of the current outer block are fp64; E is kept at fp32 level (as an fp16 hi/lo
+//     pair of a power-of-two-scaled copy); update sums come from the tensor cores with fp32 accuracy
+//     (three fp16 products per term, gemm_umma_f16.cuh).  Each weight therefore meets one rounding at
+//     fp32 level (its update sum) instead of one per preceding block.
+//   * Scaling for the fp16 pairs (all factors are powers of two, so scaling is exact):
+//       E'[r][k] = E[r][k] * sK[k] * sE[r],   U'[k][c] = U[k][c] / sK[k] * sC[c],   sum_k E U = (sum_k E' U') / (sE[r] sC[c])
+//     sK[k] ~ U_kk (then E * sK = (w - q) / mantissa(U_kk) has the size of a weight), sE[r] ~ 2^11 / max|W[r][:]|,
+//     sC[c] ~ 2^13 / max_k |U[k][c] / sK[k]|.  An E' beyond fp16's range (an error thousands of times the
+//     row's largest weight) is saturated and reported as GPTQ_ERR_NONFINITE.
 #include "common.cuh"
-#include "gemm_umma.cuh"
+#include "gemm_umma_f16.cuh"
 
 namespace gptq {
 namespace {
@@ -99,7 +105,9 @@ struct InblockArgs {
   int group;        // group size (<= 0: one grid per row)
   int grid_inside;  // 1: grids of groups that start in this block are computed here (group <= B)
   float* scales; float* zeros; int G;
-  float* Ehi; float* Elo; uint8_t* codes; double* loss; int* dev_info;
+  __half* Ehi; __half* Elo;             // scaled errors E' = E * sK[column] * sE[row] as an fp16 hi / lo pair
+  const float* sK; const float* sE;
+  uint8_t* codes; double* loss; int* dev_info;
 };
 
 // Four lanes per row, 32 rows per CTA.  The block's working weights sit in shared memory,
@@ -130,6 +138,7 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
   double* rdiag = Us + (size_t)kSB * B;   // [kSB]       1 / U_jj of the current sub-block
   float* esm = reinterpret_cast<float*>(rdiag + kSB);   // [kSB][kRPB] errors of the current sub-block, per row (fp32:
                                                         // the precision E leaves the kernel in)
+  float* sks = esm + kSB * kRPB;          // [kSB]       column scales sK of the current sub-block
   const int t = threadIdx.x, l = t & 3, rl = t >> 2;
   const int r0 = blockIdx.x * kRPB, row = r0 + rl;
   const bool live = row < a.R;
@@ -147,6 +156,7 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
     }
   }
   const int G = a.G, g = a.group;
+  const float se_row = live ? a.sE[row] : 1.f;
   float scale_f = 1.f, zero_f = 0.f;
   if (live && !a.grid_inside) {
     const int gi = g > 0 ? a.i / g : 0;
@@ -160,6 +170,7 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
 
   for (int j0 = 0; j0 < B; j0 += kSB) {
     __syncthreads();  // slab staged / previous sub-block's Us no longer read
+    if (t < kSB) sks[t] = a.sK[a.i + j0 + t];
     {
       const int q4 = B >> 2;
 #pragma unroll 8
@@ -246,18 +257,23 @@ __global__ void __launch_bounds__(kInblockThreads) inblock_kernel(InblockArgs a)
       slab[c * kLDS + rl] = x;
     }
     if (live) {
-      // lane l stores columns [8 l, 8 l + 8) of this sub-block: errors as a tf32 hi / lo pair, codes as bytes
-      float h[8], lo[8];
+      // lane l stores columns [8 l, 8 l + 8) of this sub-block: scaled errors as an fp16 hi / lo pair, codes as bytes
+      uint32_t hw[4], lw[4];
+      bool sat = false;
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const double ev = l == 0 ? err[u] : (l == 1 ? err[8 + u] : (l == 2 ? err[16 + u] : err[24 + u]));
-        tf32x3::split_tf32((float)ev, h[u], lo[u]);
+      for (int u = 0; u < 8; u += 2) {
+        __half h0, l0, h1, l1;
+        const double e0 = l == 0 ? err[u] : (l == 1 ? err[8 + u] : (l == 2 ? err[16 + u] : err[24 + u]));
+        const double e1 = l == 0 ? err[u + 1] : (l == 1 ? err[9 + u] : (l == 2 ? err[17 + u] : err[25 + u]));
+        f16x3::split_f16((float)e0 * sks[8 * l + u] * se_row, h0, l0, sat);
+        f16x3::split_f16((float)e1 * sks[8 * l + u + 1] * se_row, h1, l1, sat);
+        hw[u >> 1] = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
+        lw[u >> 1] = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
       }
+      bad |= sat;
       const int64_t o = (int64_t)row * a.C + a.i + j0 + 8 * l;
-      float4* eh = reinterpret_cast<float4*>(a.Ehi + o);
-      float4* el = reinterpret_cast<float4*>(a.Elo + o);
-      eh[0] = make_float4(h[0], h[1], h[2], h[3]); eh[1] = make_float4(h[4], h[5], h[6], h[7]);
-      el[0] = make_float4(lo[0], lo[1], lo[2], lo[3]); el[1] = make_float4(lo[4], lo[5], lo[6], lo[7]);
+      *reinterpret_cast<uint4*>(a.Ehi + o) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+      *reinterpret_cast<uint4*>(a.Elo + o) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
       *reinterpret_cast<uint2*>(a.codes + o) = make_uint2(c0, c1);
     }
   }
@@ -285,33 +301,103 @@ __global__ void pack_kernel(const uint8_t* __restrict__ codes, int R, int C, int
   qweight[idx] = word;
 }
 
-// ---- U panel -> transposed tf32 hi / lo pair ------------------------------------------------------
-// Pt[c][r] = U[r][i2 + c] for r < rows, c < nb2 (row stride ldp): the right factor of the lazy
-// updates, transposed so the contraction index is contiguous, split so that hi + lo ~ U to 2^-22.
+// ---- power-of-two scales for the fp16 operand pairs ------------------------------------------------
+// largest power of two <= x (x > 0, finite); 1 for anything else
+__device__ __forceinline__ float pow2_floor(float x) {
+  if (!(x > 0.f) || !isfinite(x)) return 1.f;
+  int e;
+  frexpf(x, &e);                       // x = m 2^e, m in [0.5, 1)
+  e = max(-100, min(100, e - 1));
+  return ldexpf(1.f, e);
+}
+// power of two s with s * x in [2^(top-1), 2^top) (x > 0, finite); 1 for anything else
+__device__ __forceinline__ float pow2_scale_to(float x, int top) {
+  if (!(x > 0.f) || !isfinite(x)) return 1.f;
+  int e;
+  frexpf(x, &e);
+  e = max(-100, min(100, top - e));
+  return ldexpf(1.f, e);
+}
+// sK[k] = largest power of two <= U_kk; colmax[c] = 0
+__global__ void kscale_kernel(const float* __restrict__ U, int C, float* __restrict__ sK, uint32_t* __restrict__ colmax) {
+  int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= C) return;
+  sK[k] = pow2_floor(U[(int64_t)k * C + k]);
+  colmax[k] = 0u;
+}
+// colmax[c] = max over rows k <= c of |U[k][c]| / sK[k]   (bit pattern of a non-negative float: ordered as integers)
+__global__ void colmax_kernel(const float* __restrict__ U, int C, const float* __restrict__ sK, uint32_t* __restrict__ colmax) {
+  __shared__ float red[8][33];
+  const int c = blockIdx.x * 32 + threadIdx.x, r0 = blockIdx.y * 256;
+  if (r0 > blockIdx.x * 32 + 31) return;               // block wholly below the diagonal
+  float m = 0.f;
+  for (int r = r0 + threadIdx.y; r < min(C, r0 + 256); r += 8)
+    if (r <= c) m = fmaxf(m, fabsf(U[(int64_t)r * C + c]) / sK[r]);
+  red[threadIdx.y][threadIdx.x] = m;
+  __syncthreads();
+  if (threadIdx.y == 0) {
+#pragma unroll
+    for (int y = 1; y < 8; ++y) m = fmaxf(m, red[y][threadIdx.x]);
+    if (m > 0.f && isfinite(m)) atomicMax(colmax + c, __float_as_uint(m));
+  }
+}
+// sC[c] = power of two that brings the column's largest scaled entry just below 2^13; sCinv = 1 / sC
+__global__ void cscale_kernel(const uint32_t* __restrict__ colmax, int C, float* __restrict__ sC, float* __restrict__ sCinv) {
+  int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= C) return;
+  const float s = pow2_scale_to(__uint_as_float(colmax[c]), 13);
+  sC[c] = s; sCinv[c] = 1.f / s;
+}
+// sE[r] = power of two that brings the row's largest |weight| just below 2^11; sEinv = 1 / sE.  One warp per row.
+__global__ void rowscale_kernel(const __half* __restrict__ W, int R, int C, float* __restrict__ sE, float* __restrict__ sEinv) {
+  int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= R) return;
+  const uint4* p = reinterpret_cast<const uint4*>(W + (int64_t)row * C);
+  float mx = 0.f;
+  for (int i = lane; i < C / 8; i += 32) {
+    uint4 v = p[i];
+    const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      float2 f = __half22float2(h[k]);
+      mx = fmaxf(mx, fmaxf(fabsf(f.x), fabsf(f.y)));
+    }
+  }
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if (lane == 0) { const float s = pow2_scale_to(mx, 11); sE[row] = s; sEinv[row] = 1.f / s; }
+}
+
+// ---- U panel -> transposed, scaled fp16 hi / lo pair ------------------------------------------------
+// Pt[c][r] = U[r][i2 + c] / sK[r] * sC[i2 + c] for r < rows, c < nb2 (row stride ldp): the right factor of the
+// lazy updates, transposed so the contraction index is contiguous, split so that hi + lo ~ value to 2^-22.
 __global__ void split_panel_t_kernel(const float* __restrict__ U, int C, int i2, int rows,
-                                     float* __restrict__ Phi, float* __restrict__ Plo, int64_t ldp) {
+                                     const float* __restrict__ sK, const float* __restrict__ sC,
+                                     __half* __restrict__ Phi, __half* __restrict__ Plo, int64_t ldp) {
   __shared__ float t[32][33];
   const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
-  t[threadIdx.y][threadIdx.x] = U[(int64_t)(r0 + threadIdx.y) * C + i2 + c0 + threadIdx.x];
+  t[threadIdx.y][threadIdx.x] = U[(int64_t)(r0 + threadIdx.y) * C + i2 + c0 + threadIdx.x] / sK[r0 + threadIdx.y];
   __syncthreads();
-  float h, l;
-  tf32x3::split_tf32(t[threadIdx.x][threadIdx.y], h, l);
+  __half h, l;
+  bool sat = false;
+  f16x3::split_f16(t[threadIdx.x][threadIdx.y] * sC[i2 + c0 + threadIdx.y], h, l, sat);
   const int64_t o = (int64_t)(c0 + threadIdx.y) * ldp + r0 + threadIdx.x;
   Phi[o] = h; Plo[o] = l;
   (void)rows;
 }
 
 // ---- contraction epilogue (one thread: one row, 32 consecutive columns of a partial sum) --------
-// Wblk[row][nofs + col ..) -= partial, as fp64 reductions: partial sums of one tile may come from
-// several CTAs (one per super-chunk of the contraction).
+// Wblk[row][nofs + col ..) -= partial / (sE[row] sC[column]), as fp64 reductions: partial sums of one tile
+// come from several CTA pairs (one per super-chunk of the contraction).
 struct EpiSubWblk {
   double* Wblk; int64_t ldw; int nofs; int R, N;
+  const float* sEinv; const float* sCinv;     // sCinv already offset to the first column of this contraction
   __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
     if (row >= R || col0 >= N) return;
     double* p = Wblk + (int64_t)row * ldw + nofs + col0;
+    const double ir = -(double)sEinv[row];
 #pragma unroll
     for (int j = 0; j < 32; ++j)
-      asm volatile("red.global.add.f64 [%0], %1;" ::"l"(p + j), "d"(-(double)v[j]) : "memory");
+      asm volatile("red.global.add.f64 [%0], %1;" ::"l"(p + j), "d"((double)v[j] * ir * (double)sCinv[col0 + j]) : "memory");
   }
 };
 
@@ -333,11 +419,17 @@ extern "C" size_t gptq_quantize_workspace_bytes(int R, int C, int bits, int grou
   if (R <= 0 || C <= 0 || block <= 0 || !bits_ok(bits)) return 0;
   WsCarver w(nullptr);
   w.take<double>((size_t)R * outer_block(C, group_size, block));  // working weights of the outer block
-  w.take<float>((size_t)R * C);                                   // E (tf32 high parts), all columns
-  w.take<float>((size_t)R * C);                                   // E (tf32 remainders)
+  w.take<__half>((size_t)R * C);                                  // scaled E (fp16 high parts), all columns
+  w.take<__half>((size_t)R * C);                                  // scaled E (fp16 remainders)
   w.take<uint8_t>((size_t)R * C);                                 // unpacked codes
-  w.take<float>((size_t)C * outer_block(C, group_size, block));   // transposed panel of U, high parts
-  w.take<float>((size_t)C * outer_block(C, group_size, block));   // panel of U, remainders
+  w.take<__half>((size_t)C * outer_block(C, group_size, block));  // transposed scaled panel of U, high parts
+  w.take<__half>((size_t)C * outer_block(C, group_size, block));  // panel of U, remainders
+  w.take<float>((size_t)C);                                       // sK
+  w.take<float>((size_t)C);                                       // sC
+  w.take<float>((size_t)C);                                       // 1 / sC
+  w.take<uint32_t>((size_t)C);                                    // column maxima of the scaled U
+  w.take<float>((size_t)R);                                       // sE
+  w.take<float>((size_t)R);                                       // 1 / sE
   return w.off;
 }
 
@@ -366,11 +458,17 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   const int G = g > 0 ? C / g : 1;
   WsCarver w(ws);
   double* Wblk = w.take<double>((size_t)R * B2);
-  float* Ehi = w.take<float>((size_t)R * C);
-  float* Elo = w.take<float>((size_t)R * C);
+  __half* Ehi = w.take<__half>((size_t)R * C);
+  __half* Elo = w.take<__half>((size_t)R * C);
   uint8_t* codes = w.take<uint8_t>((size_t)R * C);
-  float* Phi = w.take<float>((size_t)C * B2);
-  float* Plo = w.take<float>((size_t)C * B2);
+  __half* Phi = w.take<__half>((size_t)C * B2);
+  __half* Plo = w.take<__half>((size_t)C * B2);
+  float* sK = w.take<float>((size_t)C);
+  float* sC = w.take<float>((size_t)C);
+  float* sCinv = w.take<float>((size_t)C);
+  uint32_t* colmax = w.take<uint32_t>((size_t)C);
+  float* sE = w.take<float>((size_t)R);
+  float* sEinv = w.take<float>((size_t)R);
   const int64_t ldw = B2;
   GridSpec gs{bits == GPTQ_BITS_TERNARY ? 2 : (1 << bits) - 1, (sym != 0 || bits == GPTQ_BITS_TERNARY) ? 1 : 0};
 
@@ -380,14 +478,26 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
     rowgrid_kernel<<<ceil_div(R, 8), 256, 0, s>>>(W, R, C, gs, scales, zeros);
     GPTQ_LAUNCH_CHECK();
   }
-  auto inblock_smem = [&](int B) { return (size_t)((size_t)B * kLDS + (size_t)kSB * B + kSB) * sizeof(double) + (size_t)kSB * kRPB * sizeof(float); };
+  // power-of-two scales of the fp16 operand pairs: per contraction index (from U's diagonal), per column of U, per row of W
+  kscale_kernel<<<ceil_div(C, 256), 256, 0, s>>>(U, C, sK, colmax);
+  GPTQ_LAUNCH_CHECK();
+  {
+    dim3 grid(C / 32, ceil_div(C, 256)), blk(32, 8);
+    colmax_kernel<<<grid, blk, 0, s>>>(U, C, sK, colmax);
+    GPTQ_LAUNCH_CHECK();
+  }
+  cscale_kernel<<<ceil_div(C, 256), 256, 0, s>>>(colmax, C, sC, sCinv);
+  GPTQ_LAUNCH_CHECK();
+  rowscale_kernel<<<ceil_div(R, 8), 256, 0, s>>>(W, R, C, sE, sEinv);
+  GPTQ_LAUNCH_CHECK();
+  auto inblock_smem = [&](int B) { return (size_t)((size_t)B * kLDS + (size_t)kSB * B + kSB) * sizeof(double) + (size_t)(kSB * kRPB + kSB) * sizeof(float); };
   GPTQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)inblock_smem(256)));
 
   for (int i2 = 0; i2 < C; i2 += B2) {
     const int nb2 = (C - i2 < B2) ? C - i2 : B2;
     {  // transposed tf32 hi/lo pair of U[0 : i2 + nb2, i2 : i2 + nb2] for the contractions of this outer block
       dim3 grid(nb2 / 32, (i2 + nb2) / 32), blk(32, 32);
-      split_panel_t_kernel<<<grid, blk, 0, s>>>(U, C, i2, i2 + nb2, Phi, Plo, (int64_t)C);
+      split_panel_t_kernel<<<grid, blk, 0, s>>>(U, C, i2, i2 + nb2, sK, sC, Phi, Plo, (int64_t)C);
       GPTQ_LAUNCH_CHECK();
     }
     // working weights of the outer block: original weights minus all updates from columns < i2
@@ -397,8 +507,8 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
       GPTQ_LAUNCH_CHECK();
     }
     if (i2 > 0) {
-      tf32x3::Operand A{Ehi, Elo, R, i2, C}, Bop{Phi, Plo, nb2, i2, C};
-      gptq_status_t st = tf32x3::launch<false, false>(A, Bop, R, nb2, EpiSubWblk{Wblk, ldw, 0, R, nb2}, dev_info, s);
+      f16x3::Operand A{Ehi, Elo, R, i2, C}, Bop{Phi, Plo, nb2, i2, C};
+      gptq_status_t st = f16x3::launch<false, false>(A, Bop, R, nb2, EpiSubWblk{Wblk, ldw, 0, R, nb2, sEinv, sCinv + i2}, dev_info, s);
       if (st != GPTQ_OK) return st;
     }
     for (int i = i2; i < i2 + nb2; i += block) {
@@ -408,15 +518,16 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
         GPTQ_LAUNCH_CHECK();
       }
       InblockArgs a{Wblk, ldw, i - i2, U, C, i, B, R, gs, g, (g > 0 && g <= B) ? 1 : 0,
-                    scales, zeros, G, Ehi, Elo, codes, loss, dev_info};
+                    scales, zeros, G, Ehi, Elo, sK, sE, codes, loss, dev_info};
       inblock_kernel<<<ceil_div(R, kRPB), kInblockThreads, inblock_smem(B), s>>>(a);
       GPTQ_LAUNCH_CHECK();
       // push this block's errors onto the remaining columns of the outer block
       const int rest = i2 + nb2 - (i + B);
       if (rest > 0) {
         const int64_t po = (int64_t)(i + B - i2) * C + i;     // U[i][i + B] inside the transposed panel
-        tf32x3::Operand A{Ehi + i, Elo + i, R, B, C}, Bop{Phi + po, Plo + po, rest, B, C};
-        gptq_status_t st = tf32x3::launch<false, false>(A, Bop, R, rest, EpiSubWblk{Wblk, ldw, i + B - i2, R, rest}, dev_info, s);
+        f16x3::Operand A{Ehi + i, Elo + i, R, B, C}, Bop{Phi + po, Plo + po, rest, B, C};
+        gptq_status_t st = f16x3::launch<false, false>(A, Bop, R, rest, EpiSubWblk{Wblk, ldw, i + B - i2, R, rest, sEinv, sCinv + i + B},
+                                                       dev_info, s);
         if (st != GPTQ_OK) return st;
       }
     }

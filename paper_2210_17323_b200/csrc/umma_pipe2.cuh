@@ -68,11 +68,7 @@ umma_pipe2_kernel(const __grid_constant__ typename Traits::Maps maps, const int 
         if (!itemf(idx, m0, n0, kb0, kb1)) continue;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1)) { report_error(dev_info, GPTQ_ERR_TIMEOUT, 21); ok = false; break; }
-#ifdef GPTQ_EXP_SKIP_B
-          if (rank == 0) mbar_arrive_expect_tx(&full[stage], STAGE_BYTES);
-#else
           if (rank == 0) mbar_arrive_expect_tx(&full[stage], 2 * STAGE_BYTES);   // bytes of both CTAs
-#endif
           Traits::load(tiles + (size_t)stage * STAGE_BYTES, maps, m0 + BM_CTA * (int)rank, n0 + (BN / 2) * (int)rank, kb,
                        &full[stage]);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
