@@ -162,6 +162,19 @@ gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U, int R, int
                                   uint32_t* qweight, float* scales, float* zeros, double* loss,
                                   void* ws, size_t ws_bytes, int* dev_info, void* stream);
 
+/* Which form of Algorithm 1's loops gptq_quantize_layer runs INSIDE an outer block of about 1024 columns (both are
+ * exact regroupings of the same updates, Section 3 Step 2; updates ACROSS outer blocks are one large tensor-core
+ * contraction per outer block either way):
+ *   1 (default)  row-stripe form: rows are independent (Section 2), so one CTA owns a stripe of rows and runs all
+ *                inner blocks of the outer block back to back in ONE launch -- the inner loop with one thread per
+ *                row, the block's lazy update for its rows with warp-level tensor-core instructions.  block <= 128;
+ *                a larger block falls back to form 0.
+ *   0            per inner block one in-block kernel and one small tcgen05 contraction (two launches per block).
+ * Process-wide, takes effect for calls made afterwards; returns the previous value (any other argument only
+ * queries).  Meant for side-by-side benchmarks; results of the two forms agree up to fp32-level rounding of the
+ * update sums. */
+int gptq_set_stage3_variant(int variant);
+
 /* ------------------------------------------------------------------ round-to-nearest baseline
  * RTN (Section 5, Baselines): every weight rounded to the nearest value of the solver's own
  * grid -- per-row (group_size <= 0) or per-group min-max taken from the ORIGINAL weights -- with

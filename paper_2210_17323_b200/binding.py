@@ -54,6 +54,8 @@ def _load():
     lib.gptq_quantize_layer.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_int, c.c_int, c.c_int,
                                         c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
                                         c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
+    lib.gptq_set_stage3_variant.restype = c.c_int
+    lib.gptq_set_stage3_variant.argtypes = [c.c_int]
     lib.gptq_solve_layer_host_workspace_bytes.restype = c.c_size_t
     lib.gptq_solve_layer_host_workspace_bytes.argtypes = [c.c_int, c.c_int, c.c_int64, c.c_int, c.c_int, c.c_int]
     lib.gptq_solve_layer_host.restype = c.c_int
@@ -199,6 +201,11 @@ def gptq_quantize_layer(W, U, bits, group_size=0, sym=False, block=128, ws=None,
         if st != OK:
             raise GptqError(st, "gptq_quantize_layer")
         return dict(qweight=qweight, scales=scales, zeros=zeros, loss=loss, dev_info=dev_info)
+
+
+def gptq_set_stage3_variant(variant: int) -> int:
+    """1: row-stripe kernel inside an outer block (default); 0: per-inner-block kernels.  Returns the previous value."""
+    return int(_lib.gptq_set_stage3_variant(int(variant)))
 
 
 def gptq_solve_layer_host_workspace_bytes(R, C, n_tokens, bits, group_size, block):

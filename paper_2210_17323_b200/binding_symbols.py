@@ -3,7 +3,7 @@ EXPORTS = (
     "gptq_status_string", "gptq_launch_count",
     "gptq_hessian_workspace_bytes", "gptq_hessian_accumulate",
     "gptq_prepare_hinv_workspace_bytes", "gptq_prepare_hinv", "gptq_prepare_hinv_static",
-    "gptq_quantize_workspace_bytes", "gptq_quantize_layer",
+    "gptq_quantize_workspace_bytes", "gptq_quantize_layer", "gptq_set_stage3_variant",
     "gptq_solve_layer_host_workspace_bytes", "gptq_solve_layer_host",
     "gptq_rtn_layer", "gptq_dequantize", "gptq_matvec",
 )

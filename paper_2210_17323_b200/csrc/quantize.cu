@@ -19,6 +19,8 @@
 //     sK[k] ~ U_kk (then E * sK = (w - q) / mantissa(U_kk) has the size of a weight), sE[r] ~ 2^11 / max|W[r][:]|,
 //     sC[c] ~ 2^13 / max_k |U[k][c] / sK[k]|.  An E' beyond fp16's range (an error thousands of times the
 //     row's largest weight) is saturated and reported as GPTQ_ERR_NONFINITE.
+#include <atomic>
+
 #include "common.cuh"
 #include "gemm_umma_f16.cuh"
 
@@ -89,12 +91,15 @@ __global__ void groupgrid_kernel(const double* __restrict__ Wblk, int64_t ldw, i
 }
 
 // ---- working weights of an outer block start as the original weights ---------------------------
+// stripe_major: the layout the row-stripe kernel wants (128-row stripes, each column of a stripe contiguous);
+// otherwise plain row-major [R][ldw].
 __global__ void wblk_from_w16_kernel(const __half* __restrict__ W, int R, int C, int i2, int nb,
-                                     double* __restrict__ Wblk, int64_t ldw) {
+                                     double* __restrict__ Wblk, int64_t ldw, int stripe_major) {
   int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)R * nb) return;
   int r = (int)(idx / nb), c = (int)(idx % nb);
-  Wblk[(int64_t)r * ldw + c] = (double)__half2float(W[(int64_t)r * C + i2 + c]);
+  const int64_t o = stripe_major ? ((int64_t)(r >> 7) * ldw + c) * 128 + (r & 127) : (int64_t)r * ldw + c;
+  Wblk[o] = (double)__half2float(W[(int64_t)r * C + i2 + c]);
 }
 
 // ---- the in-block loop (Algorithm 1, inner FOR) -------------------------------------------------
@@ -391,15 +396,38 @@ __global__ void split_panel_t_kernel(const float* __restrict__ U, int C, int i2,
 struct EpiSubWblk {
   double* Wblk; int64_t ldw; int nofs; int R, N;
   const float* sEinv; const float* sCinv;     // sCinv already offset to the first column of this contraction
+  int stripe_major;                           // layout of Wblk (see wblk_from_w16_kernel)
   __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
     if (row >= R || col0 >= N) return;
-    double* p = Wblk + (int64_t)row * ldw + nofs + col0;
     const double ir = -(double)sEinv[row];
+    double* p = stripe_major ? Wblk + ((int64_t)(row >> 7) * ldw + nofs + col0) * 128 + (row & 127)
+                             : Wblk + (int64_t)row * ldw + nofs + col0;
+    const int64_t step = stripe_major ? 128 : 1;
 #pragma unroll
     for (int j = 0; j < 32; ++j)
-      asm volatile("red.global.add.f64 [%0], %1;" ::"l"(p + j), "d"((double)v[j] * ir * (double)sCinv[col0 + j]) : "memory");
+      asm volatile("red.global.add.f64 [%0], %1;" ::"l"(p + j * step), "d"((double)v[j] * ir * (double)sCinv[col0 + j]) : "memory");
   }
 };
+
+#include "quantize_stripe.cuh"
+
+// Which form runs inside an outer block: 1 = row-stripe kernel (one launch per outer block), 0 = one in-block
+// kernel plus one small tensor-core contraction per inner block.  Process-wide; see gptq_set_stage3_variant.
+std::atomic<int> g_stage3_variant{1};
+
+gptq_status_t launch_stripe(const StripeArgs& a, const __half* Phi, const __half* Plo, cudaStream_t s) {
+  StripeMaps maps;
+  gptq_status_t st;
+  // Pt[c - i2][k]: rows = columns of the outer block, inner dimension = contraction index (rows of U so far)
+  if ((st = make_tmap_2d(&maps.p_hi, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, Phi, (uint64_t)(a.i2 + a.nb2), (uint64_t)a.nb2,
+                         (uint64_t)a.C * 2, 64, kStripeNT)) != GPTQ_OK) return st;
+  if ((st = make_tmap_2d(&maps.p_lo, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, Plo, (uint64_t)(a.i2 + a.nb2), (uint64_t)a.nb2,
+                         (uint64_t)a.C * 2, 64, kStripeNT)) != GPTQ_OK) return st;
+  GPTQ_CUDA_TRY(cudaFuncSetAttribute(stripe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stripe_smem(kStripeMaxB)));
+  stripe_kernel<<<ceil_div(a.R, kStripeRows), kStripeThreads, stripe_smem(a.B), s>>>(maps, a);
+  GPTQ_LAUNCH_CHECK();
+  return GPTQ_OK;
+}
 
 inline int field_bits(int bits) { return bits == GPTQ_BITS_TERNARY ? 2 : bits; }
 inline bool bits_ok(int bits) { return bits == 2 || bits == 3 || bits == 4 || bits == 8 || bits == GPTQ_BITS_TERNARY; }
@@ -418,7 +446,7 @@ extern "C" size_t gptq_quantize_workspace_bytes(int R, int C, int bits, int grou
   using namespace gptq;
   if (R <= 0 || C <= 0 || block <= 0 || !bits_ok(bits)) return 0;
   WsCarver w(nullptr);
-  w.take<double>((size_t)R * outer_block(C, group_size, block));  // working weights of the outer block
+  w.take<double>((size_t)ceil_div(R, 128) * 128 * outer_block(C, group_size, block));  // working weights of the outer block
   w.take<__half>((size_t)R * C);                                  // scaled E (fp16 high parts), all columns
   w.take<__half>((size_t)R * C);                                  // scaled E (fp16 remainders)
   w.take<uint8_t>((size_t)R * C);                                 // unpacked codes
@@ -457,7 +485,7 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   const int B2 = outer_block(C, g, block);
   const int G = g > 0 ? C / g : 1;
   WsCarver w(ws);
-  double* Wblk = w.take<double>((size_t)R * B2);
+  double* Wblk = w.take<double>((size_t)ceil_div(R, 128) * 128 * B2);
   __half* Ehi = w.take<__half>((size_t)R * C);
   __half* Elo = w.take<__half>((size_t)R * C);
   uint8_t* codes = w.take<uint8_t>((size_t)R * C);
@@ -493,6 +521,8 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   auto inblock_smem = [&](int B) { return (size_t)((size_t)B * kLDS + (size_t)kSB * B + kSB) * sizeof(double) + (size_t)(kSB * kRPB + kSB) * sizeof(float); };
   GPTQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)inblock_smem(256)));
 
+  // form of the loops inside an outer block (see gptq_set_stage3_variant)
+  const bool stripe = g_stage3_variant.load(std::memory_order_relaxed) == 1 && block <= kStripeMaxB && B2 <= kStripeMaxNb2;
   for (int i2 = 0; i2 < C; i2 += B2) {
     const int nb2 = (C - i2 < B2) ? C - i2 : B2;
     {  // transposed tf32 hi/lo pair of U[0 : i2 + nb2, i2 : i2 + nb2] for the contractions of this outer block
@@ -503,13 +533,22 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
     // working weights of the outer block: original weights minus all updates from columns < i2
     {
       int64_t total = (int64_t)R * nb2;
-      wblk_from_w16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(W, R, C, i2, nb2, Wblk, ldw);
+      wblk_from_w16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(W, R, C, i2, nb2, Wblk, ldw, stripe ? 1 : 0);
       GPTQ_LAUNCH_CHECK();
     }
     if (i2 > 0) {
       f16x3::Operand A{Ehi, Elo, R, i2, C}, Bop{Phi, Plo, nb2, i2, C};
-      gptq_status_t st = f16x3::launch<false, false>(A, Bop, R, nb2, EpiSubWblk{Wblk, ldw, 0, R, nb2, sEinv, sCinv + i2}, dev_info, s);
+      gptq_status_t st = f16x3::launch<false, false>(A, Bop, R, nb2, EpiSubWblk{Wblk, ldw, 0, R, nb2, sEinv, sCinv + i2, stripe ? 1 : 0},
+                                                     dev_info, s);
       if (st != GPTQ_OK) return st;
+    }
+    if (stripe) {
+      // row-stripe form: every inner block of this outer block in one launch
+      StripeArgs a{Wblk, ldw, nb2, U, C, i2, block, R, gs, g, scales, zeros, G, Ehi, Elo, Phi, Plo, (int64_t)C,
+                   sK, sE, sEinv, sCinv, codes, loss, dev_info};
+      gptq_status_t st = launch_stripe(a, Phi, Plo, s);
+      if (st != GPTQ_OK) return st;
+      continue;
     }
     for (int i = i2; i < i2 + nb2; i += block) {
       const int B = (i2 + nb2 - i < block) ? i2 + nb2 - i : block;
@@ -526,7 +565,7 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
       if (rest > 0) {
         const int64_t po = (int64_t)(i + B - i2) * C + i;     // U[i][i + B] inside the transposed panel
         f16x3::Operand A{Ehi + i, Elo + i, R, B, C}, Bop{Phi + po, Plo + po, rest, B, C};
-        gptq_status_t st = f16x3::launch<false, false>(A, Bop, R, rest, EpiSubWblk{Wblk, ldw, i + B - i2, R, rest, sEinv, sCinv + i + B},
+        gptq_status_t st = f16x3::launch<false, false>(A, Bop, R, rest, EpiSubWblk{Wblk, ldw, i + B - i2, R, rest, sEinv, sCinv + i + B, 0},
                                                        dev_info, s);
         if (st != GPTQ_OK) return st;
       }
@@ -540,3 +579,15 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   }
   return GPTQ_OK;
 }
+
+extern "C" int gptq_set_stage3_variant(int variant) {
+  if (variant != 0 && variant != 1) return gptq::g_stage3_variant.load();
+  return gptq::g_stage3_variant.exchange(variant);
+}
+
+#ifdef GPTQ_EXP_TIMING
+extern "C" int gptq_dbg_stripe_timing(unsigned long long* out32, int reset) {
+  if (reset) { unsigned long long z[32] = {}; return (int)cudaMemcpyToSymbol(gptq::g_stripe_dbg, z, sizeof(z)); }
+  return (int)cudaMemcpyFromSymbol(out32, gptq::g_stripe_dbg, 32 * sizeof(unsigned long long));
+}
+#endif

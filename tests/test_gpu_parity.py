@@ -144,6 +144,28 @@ def test_quantize_layer_matches_oracle(B, R, C, bits, group, sym, block):
     check_quantize_outputs(gpu, ref, W16, bits, C, H)
 
 
+@pytest.mark.parametrize("R,C,bits,group,sym,block", [CASES[0], CASES[1], CASES[4], CASES[5], CASES[8], CASES[11], CASES[12], CASES[14]])
+def test_quantize_layer_per_block_form_matches_oracle(B, R, C, bits, group, sym, block):
+    """The other form of the loops inside an outer block (one in-block kernel plus one small tensor-core contraction per
+    inner block instead of the row-stripe kernel): same parity bar, and its codes agree with the default form's."""
+    L = _layer(R, C, 2 * C + 64, cfg=8)
+    W16 = L.w()
+    H = O.hessian_accumulate(np.zeros((C, C)), L.x_bits())
+    U32 = O.cholesky_inverse_upper(O.dampen(H, 0.01)[0]).astype(np.float32)
+    ref = O.quantize_layer(W16, U32.astype(np.float64), bits, group, sym, block)
+    stripe = _run_quant(B, W16, U32, bits, group, sym, block)
+    prev = B.gptq_set_stage3_variant(0)
+    try:
+        assert prev == 1
+        gpu = _run_quant(B, W16, U32, bits, group, sym, block)
+    finally:
+        B.gptq_set_stage3_variant(prev)
+    check_quantize_outputs(gpu, ref, W16, bits, C, H)
+    a = O.unpack_codes(gpu["qweight"].view(np.uint32), bits, C)
+    b = O.unpack_codes(stripe["qweight"].view(np.uint32), bits, C)
+    assert (a == b).mean() >= 0.999
+
+
 def test_quantize_block_size_invariance_on_gpu(B):
     R, C = 128, 1024
     L = _layer(R, C, 3000, cfg=7)
