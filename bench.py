@@ -472,6 +472,93 @@ def run_gpu(args, wl):
     return 0
 
 
+def run_gpu_strong(args, wl):
+    """Strong scaling of the SAME layer set over the ranks (paper_2210_17323_b200/multi.py): every layer's calibration tokens
+    are sharded over the ranks, each rank accumulates its partial Hessian, ONE NCCL all-reduce of H per layer (a plain sum of
+    local buffers) gives every rank the full matrix, the factor is computed on every rank, and each rank quantizes its
+    stripe of rows.  Sequential schedule, host-issued launches.  value = the layer set's weights / the slowest rank's time."""
+    import torch
+    import torch.distributed as dist
+    from paper_2210_17323_b200 import binding as B, multi
+    from paper_2210_17323_b200.synth import device as D
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    state, ws_bytes = [], 256
+    for L in wl.layers:
+        tr = multi.token_shard(L.n_tokens, world, rank)
+        rows = multi.shard_units(L.R, world, rank)
+        Wfull = D.fill_w(L, device=dev)
+        st = dict(L=L, X=D.fill_x(L, tr.start, tr.stop, device=dev), W=Wfull[rows.start:rows.stop].contiguous(), rows=rows,
+                  H=torch.empty((L.C, L.C), dtype=torch.float32, device=dev),
+                  U=torch.empty((L.C, L.C), dtype=torch.float32, device=dev),
+                  info=torch.zeros(2, dtype=torch.int32, device=dev), out={})
+        del Wfull
+        ws_bytes = max(ws_bytes, B.gptq_hessian_workspace_bytes(L.C, len(tr)), B.gptq_prepare_hinv_workspace_bytes(L.C),
+                       *[B.gptq_quantize_workspace_bytes(max(1, len(rows)), L.C, g.bits, g.group_size, wl.block) for g in wl.grids])
+        state.append(st)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    comm_bytes = sum(st["L"].C ** 2 * 4 for st in state)
+
+    def step():
+        for st in state:
+            multi.solve_layer_sharded(
+                st["L"].n_tokens, st["L"].R, world, rank,
+                hessian_of_tokens=lambda tr, st=st: (st["H"].zero_(), B.gptq_hessian_accumulate(st["H"], st["X"], ws=ws))[1],
+                factor_of=lambda H, st=st: B.gptq_prepare_hinv(H, wl.damp, U=st["U"], ws=ws, dev_info=st["info"])[0],
+                quantize_rows=lambda rr, U, st=st: [st["out"].__setitem__(gi, B.gptq_quantize_layer(
+                    st["W"], U, g.bits, g.group_size, g.sym, wl.block, ws=ws)) for gi, g in enumerate(wl.grids)] if len(rr) else None)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    launches0 = B.gptq_launch_count()
+    step(); barrier()
+    launches_per_step = B.gptq_launch_count() - launches0
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    for st in state:
+        assert st["info"].tolist()[0] == 0, "prepare_hinv reported an error"
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0.record()
+    for _ in range(args.steps):
+        step()
+    t1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_per_step = multi.max_over_ranks(t0.elapsed_time(t1), dev) / args.steps
+    n_grids = len(wl.grids)
+    line = dict(metric=METRIC, value=wl.weights * n_grids / (ms_per_step * 1e-3), unit=UNIT, n_gpus=world, steps=args.steps,
+                warmup=args.warmup, ms_per_step=ms_per_step, higher_is_better=True, scaling="strong", vs_baseline=None,
+                dtype="bf16 x bf16 -> f32 (Hessian); f32 factor; f64 working weights + f32 update sums (quantize)",
+                data="synthetic",
+                config=dict(workload=wl.name, layers=[l.name for l in wl.layers],
+                            grids=[dict(bits=g.bits, group_size=g.group_size, sym=g.sym) for g in wl.grids],
+                            block=wl.block, damp=wl.damp, calib_tokens=wl.layers[0].n_tokens,
+                            cache="inputs larger than L2; no flush needed", launch="host-issued launches",
+                            parallelism=f"tokens of every Hessian and rows of every layer sharded x{world}; one all-reduce of H per "
+                                        f"layer ({comm_bytes} bytes per step), factor replicated"),
+                sec_per_layer=ms_per_step * 1e-3 / len(wl.layers), gpu_launches=int(launches_per_step * args.steps), clocks=clocks)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
 def run_e2e(args, wl, state, device_value):
     """Same metric end to end through the C ABI's host-buffer call: every step, for every layer (and grid),
     gptq_solve_layer_host streams X and W from pinned HOST memory to the device (copies overlapped with the
@@ -589,48 +676,20 @@ def run_inference(args, wl):
 
 
 def run_block(args, wl):
-    """Transformer-block pipeline on one GPU (Section 5, Setup: a block's layers are quantized from the same pass of
-    calibration inputs).  q, k and v read the same input, so they share ONE Hessian and ONE factor U; o, fc1 and fc2
-    have their own.  The Hessians run back to back on one stream; each input group's stage 2 follows on its own
-    stream, and every member layer's stage 3 on its own stream after that.  One grid (--grid) per run, as a real
+    """Transformer-block pipeline on one GPU (paper_2210_17323_b200/pipeline.py): q, k and v read the same input, so they
+    share ONE Hessian and ONE factor U; o, fc1 and fc2 have their own.  One grid (--grid) per run, as a real
     quantization run has.  Prints the block time and the solver-only time of a whole model of such blocks."""
     import torch
-    from paper_2210_17323_b200 import binding as B
+    from paper_2210_17323_b200 import binding as B, pipeline as P
     from paper_2210_17323_b200.synth import device as D
 
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     g = wl.grids[min(args.grid, len(wl.grids) - 1)]
-    groups = []                                   # (input layer, member layers)
-    for L in wl.layers:
-        shared = [gr for gr in groups if L.kind in ("k", "v") and gr[0].kind == "q" and gr[0].block_idx == L.block_idx
-                  and gr[0].C == L.C]
-        if shared:
-            shared[0][1].append(L)
-        else:
-            groups.append((L, [L]))
-    state = []
-    for Lx, members in groups:
-        gs = dict(Lx=Lx, X=D.fill_x(Lx, device=dev),
-                  H=torch.empty((Lx.C, Lx.C), dtype=torch.float32, device=dev),
-                  U=torch.empty((Lx.C, Lx.C), dtype=torch.float32, device=dev),
-                  info=torch.zeros(2, dtype=torch.int32, device=dev),
-                  ws=torch.empty(max(256, B.gptq_hessian_workspace_bytes(Lx.C, Lx.n_tokens),
-                                     B.gptq_prepare_hinv_workspace_bytes(Lx.C)), dtype=torch.uint8, device=dev),
-                  stream=torch.cuda.Stream(device=dev), members=[])
-        for L in members:
-            gs["members"].append(dict(L=L, W=D.fill_w(L, device=dev), out=None, stream=torch.cuda.Stream(device=dev),
-                                      ws=torch.empty(B.gptq_quantize_workspace_bytes(L.R, L.C, g.bits, g.group_size, wl.block),
-                                                     dtype=torch.uint8, device=dev)))
-        state.append(gs)
-    state.sort(key=lambda gs: -(gs["Lx"].C ** 2) * (gs["Lx"].n_tokens + gs["Lx"].C))
-    main = torch.cuda.Stream(device=dev)
+    groups = P.group_by_shared_input(wl.layers, lambda L: D.fill_x(L, device=dev), lambda L: D.fill_w(L, device=dev))
+    solver = P.BlockSolver(groups, g.bits, g.group_size, g.sym, wl.block, wl.damp)
+    main = solver.main
     torch.cuda.synchronize()
-
-    def fH(gs): gs["H"].zero_(); B.gptq_hessian_accumulate(gs["H"], gs["X"], ws=gs["ws"])
-    def fU(gs): B.gptq_prepare_hinv(gs["H"], wl.damp, U=gs["U"], ws=gs["ws"], dev_info=gs["info"])
-    def fQ(gs, m): m["out"] = B.gptq_quantize_layer(m["W"], gs["U"], g.bits, g.group_size, g.sym, wl.block, ws=m["ws"])
-
     graphs = {}
 
     def run(key, fn):
@@ -639,48 +698,27 @@ def run_block(args, wl):
         else:
             fn()
 
-    def step():
-        ends = []
-        for gi, gs in enumerate(state):
-            with torch.cuda.stream(main):
-                run(("H", gi), lambda: fH(gs))
-                h_done = torch.cuda.Event(); h_done.record(main)
-            with torch.cuda.stream(gs["stream"]):
-                gs["stream"].wait_event(h_done)
-                run(("U", gi), lambda: fU(gs))
-                u_done = torch.cuda.Event(); u_done.record(gs["stream"])
-            for mi, m in enumerate(gs["members"]):
-                with torch.cuda.stream(m["stream"]):
-                    m["stream"].wait_event(u_done)
-                    run(("Q", gi, mi), lambda: fQ(gs, m))
-                    e = torch.cuda.Event(); e.record(m["stream"]); ends.append(e)
-        for e in ends:
-            main.wait_event(e)
-
     launches0 = B.gptq_launch_count()
-    step()
+    solver.enqueue(run)
     torch.cuda.synchronize()
     launches_per_step = B.gptq_launch_count() - launches0
     if not args.no_graphs:
-        for gi, gs in enumerate(state):
-            for key, fn in ([(("H", gi), lambda: fH(gs)), (("U", gi), lambda: fU(gs))] +
-                            [(("Q", gi, mi), (lambda m=m: fQ(gs, m))) for mi, m in enumerate(gs["members"])]):
-                cg = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(cg):
-                    fn()
-                graphs[key] = cg
+        for key, fn in solver.stage_calls():
+            cg = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(cg):
+                fn()
+            graphs[key] = cg
     for _ in range(args.warmup):
-        step()
+        solver.enqueue(run)
     torch.cuda.synchronize()
-    for gs in state:
-        assert gs["info"].tolist()[0] == 0, "prepare_hinv reported an error"
+    solver.check()
     sampler = ClockSampler(0)
     sampler.start()
     t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     t0.record(main)
     for _ in range(args.steps):
-        step()
+        solver.enqueue(run)
     t1.record(main)
     torch.cuda.synchronize()
     clocks = sampler.stop()
@@ -693,8 +731,8 @@ def run_block(args, wl):
                 dtype="bf16 x bf16 -> f32 (Hessian); f32 factor; f64 working weights + f32 update sums (quantize)",
                 config=dict(workload=wl.name, mode="block pipeline: q, k, v share one Hessian and one factor",
                             grid=dict(bits=g.bits, group_size=g.group_size, sym=g.sym), block=wl.block, damp=wl.damp,
-                            input_groups=[[m["L"].name for m in gs["members"]] for gs in state],
-                            hessians_per_block=len(state) // blocks_here,
+                            input_groups=[[m["m"].name for m in st["members"]] for st in solver.state],
+                            hessians_per_block=len(solver.state) // blocks_here,
                             launch="CUDA graphs, one per stage" if graphs else "host-issued launches"),
                 sec_per_block=sec_per_block,
                 model_estimate=(dict(blocks=model_blocks, solver_seconds=model_blocks * sec_per_block,
@@ -719,6 +757,9 @@ def main():
                          "its Hessian is done; hessians-first: all Hessians, then all layers' stages 2-3 side by side; "
                          "sequential: one stream, layer after layer")
     ap.add_argument("--no-overlap", action="store_true", help="same as --schedule sequential")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="weak (default): every rank solves its own copy of the layer set; strong: the same layer set, tokens of "
+                         "every Hessian and rows of every layer sharded over the ranks with one all-reduce of H per layer")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-whole-layer-check", action="store_true",
@@ -744,6 +785,8 @@ def main():
         return run_inference(args, wl)
     if args.mode == "block":
         return run_block(args, wl)
+    if args.scaling == "strong":
+        return run_gpu_strong(args, wl)
     return run_gpu(args, wl)
 
 

@@ -54,6 +54,15 @@ typedef enum {
  * Quantization"); its codes 0, 1, 2 are stored in 2-bit fields. */
 #define GPTQ_BITS_TERNARY (-1)
 
+/* Bits of the `sym` argument of gptq_quantize_layer / gptq_rtn_layer / gptq_solve_layer_host (0 and 1 keep their
+ * old meaning).  GPTQ_GRID_FP16_SCALES: every scale is rounded to the nearest fp16 value when the grid is
+ * fixed -- before the zero-point is derived from it and before any weight is rounded on it -- so that a model stored
+ * with one FP16 scale per group (the storage Section 5, "Extreme Quantization", counts) dequantizes to exactly the
+ * values the solver compensated for.  The scale is still returned as fp32 (holding an fp16-representable value);
+ * a scale that fp16 would flush to 0 or overflow stays fp32. */
+#define GPTQ_GRID_SYMMETRIC 1
+#define GPTQ_GRID_FP16_SCALES 2
+
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* gptq_status_string(gptq_status_t status);
 
@@ -83,9 +92,9 @@ gptq_status_t gptq_hessian_accumulate(float* H, const void* X_bf16, int64_t n_to
  * lambda = damp * mean(diag H);  H~ = H + lambda I          (Section 3, Step 3)
  * U = Cholesky(H~^-1)^T: upper triangular, positive diagonal, U^T U = H~^-1
  *                                                          (Algorithm 1, line 3)
- *   H        [C x C] fp32, symmetric (only its upper triangle is read); left intact.
+ *   H        [C x C] fp32, symmetric (only its upper triangle is read); left intact unless U == H.
  *   U        [C x C] fp32, fully overwritten; the strict lower triangle is set to 0.
- *            U must not alias H.
+ *            U may be the same buffer as H (the factor then replaces the Hessian); partial overlap is not allowed.
  *   dev_info int[2]: [0] = GPTQ_OK or GPTQ_ERR_NOT_PD, [1] = index of the first
  *            non-positive pivot.  On NOT_PD the contents of U are unspecified
  *            but finite operations continue (no trap, no hang).
@@ -142,9 +151,9 @@ gptq_status_t gptq_prepare_hinv_static(const float* H, float damp, int C, float*
  *              `block` (g % block == 0 or block % g == 0).  Supported sizes: 4, 8, 16
  *              or any multiple of 32 (the paper uses 8, 32, 64, 128, 1024); anything
  *              else returns GPTQ_ERR_UNSUPPORTED.
- *   sym        0: asymmetric min-max grid (range widened to contain 0, integer
- *              zero-point).  non-zero: symmetric grid, zero = (maxq+1)/2.
- *              The ternary grid is always symmetric.
+ *   sym        bit mask: 0: asymmetric min-max grid (range widened to contain 0, integer
+ *              zero-point).  GPTQ_GRID_SYMMETRIC: symmetric grid, zero = (maxq+1)/2 (the ternary grid
+ *              is always symmetric).  GPTQ_GRID_FP16_SCALES: see above.  Other bits: GPTQ_ERR_INVALID_ARG.
  *   block      B of Algorithm 1: a multiple of 32 in [32, 256].  The result does
  *              not depend on it (Section 3, Step 2) up to rounding.
  *   qweight    [R x C*f/32] uint32, f = field width (bits; 2 for ternary): per

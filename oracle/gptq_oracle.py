@@ -82,14 +82,28 @@ def field_bits_of(bits: int) -> int:
     return 2 if bits == BITS_TERNARY else bits
 
 
-def find_params(v: np.ndarray, bits: int, sym: bool):
+def _storage_rounded(scale: np.ndarray, scale_fp16: bool) -> np.ndarray:
+    """The scale in the precision it is returned (and, with scale_fp16, stored) in, as float64 values.
+    fp32 always; with scale_fp16 additionally rounded to the nearest fp16 value (Section 5, Extreme Quantization,
+    counts one FP16 scale per group) unless that would be 0 or infinite, in which case the fp32 value stays."""
+    s32 = scale.astype(np.float32)
+    if not scale_fp16:
+        return s32.astype(np.float64)
+    with np.errstate(over="ignore"):
+        s16 = s32.astype(np.float16)
+    usable = np.isfinite(s16) & (s16 > 0)
+    return np.where(usable, s16.astype(np.float64), s32.astype(np.float64))
+
+
+def find_params(v: np.ndarray, bits: int, sym: bool, scale_fp16: bool = False):
     """Min-max grid of each row of v (Section 5, Setup: asymmetric uniform grid spanning the
     row's minimum and maximum; grouping applies the same to g consecutive weights).
     The range is widened to contain 0 so the zero-point is an integer code (Section 5,
     Extreme Quantization, counts a b-bit zero-point per group in its storage figures).  An
     all-zero row gets [-1, 1].  Symmetric / ternary: half-range a = max|v|,
     scale = 2a/maxq, zero = (maxq+1)//2.  The scale is rounded to fp32 -- the
-    precision it is returned in -- and used as that value.
+    precision it is returned in -- and used as that value; with scale_fp16 it is rounded to
+    fp16 instead (the stored model's precision), BEFORE the zero-point is derived from it.
     Returns (scale[R] float64 holding fp32 values, zero[R] float64 holding integers)."""
     maxq = maxq_of(bits)
     xmin = np.minimum(v.min(axis=1), 0.0)
@@ -99,10 +113,10 @@ def find_params(v: np.ndarray, bits: int, sym: bool):
     xmax = np.where(dead, 1.0, xmax)
     if sym or bits == BITS_TERNARY:
         a = np.maximum(np.abs(xmin), xmax)
-        scale = (2.0 * a / maxq).astype(np.float32).astype(np.float64)
+        scale = _storage_rounded(2.0 * a / maxq, scale_fp16)
         zero = np.full_like(scale, float((maxq + 1) // 2))
     else:
-        scale = ((xmax - xmin) / maxq).astype(np.float32).astype(np.float64)
+        scale = _storage_rounded((xmax - xmin) / maxq, scale_fp16)
         zero = np.rint(-xmin / scale)
     return scale, zero
 
@@ -115,10 +129,10 @@ def quant(w: np.ndarray, scale: np.ndarray, zero: np.ndarray, maxq: int):
 
 
 # --------------------------------------------------------------------------- stage 3
-def _fix_group_grid(W, j, g, bits, sym, scales, zeros):
+def _fix_group_grid(W, j, g, bits, sym, scales, zeros, scale_fp16=False):
     """Column j opens a group: its g columns, in the state the error feedback of all earlier
     columns has left them, decide the group's scale and zero-point (Section 5, grouping)."""
-    scales[:, j // g], zeros[:, j // g] = find_params(W[:, j:j + g], bits, sym)
+    scales[:, j // g], zeros[:, j // g] = find_params(W[:, j:j + g], bits, sym, scale_fp16)
 
 
 def _round_column_and_feed_back(W, U, j, stop, s, z, maxq):
@@ -139,7 +153,7 @@ def _push_block_errors(W, U, E, i, stop):
 
 
 def quantize_layer(W16: np.ndarray, U: np.ndarray, bits: int, group_size: int = 0,
-                   sym: bool = False, block: int = 128):
+                   sym: bool = False, block: int = 128, scale_fp16: bool = False):
     """Algorithm 1 with lazy batch updates of `block` columns.
 
     W16: (R x C) fp16 (promoted exactly to double); U: (C x C) upper factor.
@@ -165,13 +179,13 @@ def quantize_layer(W16: np.ndarray, U: np.ndarray, bits: int, group_size: int = 
     zeros = np.zeros((R, G))
     E_all = np.zeros((R, C))
     if not grouped:
-        scales[:, 0], zeros[:, 0] = find_params(W, bits, sym)
+        scales[:, 0], zeros[:, 0] = find_params(W, bits, sym, scale_fp16)
     for i in range(0, C, block):
         stop = min(i + block, C)
         E = np.zeros((R, stop - i))
         for j in range(i, stop):
             if grouped and j % g == 0:
-                _fix_group_grid(W, j, g, bits, sym, scales, zeros)
+                _fix_group_grid(W, j, g, bits, sym, scales, zeros, scale_fp16)
             codes[:, j], W_hat[:, j], E[:, j - i] = _round_column_and_feed_back(
                 W, U, j, stop, scales[:, j // g], zeros[:, j // g], maxq)
         _push_block_errors(W, U, E, i, stop)
@@ -180,7 +194,7 @@ def quantize_layer(W16: np.ndarray, U: np.ndarray, bits: int, group_size: int = 
     return dict(codes=codes, scales=scales, zeros=zeros, loss=loss, W_hat=W_hat, E=E_all)
 
 
-def rtn(W16: np.ndarray, bits: int, group_size: int = 0, sym: bool = False):
+def rtn(W16: np.ndarray, bits: int, group_size: int = 0, sym: bool = False, scale_fp16: bool = False):
     """Round-to-nearest on the same grid, no error feedback (Section 5, Baselines)."""
     W = np.asarray(W16, dtype=np.float64)
     R, C = W.shape
@@ -188,7 +202,7 @@ def rtn(W16: np.ndarray, bits: int, group_size: int = 0, sym: bool = False):
     codes = np.zeros((R, C), dtype=np.int32)
     What = np.zeros((R, C))
     for j0 in range(0, C, g):
-        s, z = find_params(W[:, j0:j0 + g], bits, sym)
+        s, z = find_params(W[:, j0:j0 + g], bits, sym, scale_fp16)
         q, What[:, j0:j0 + g] = quant(W[:, j0:j0 + g], s[:, None], z[:, None], maxq_of(bits))
         codes[:, j0:j0 + g] = q.astype(np.int32)
     return codes, What

@@ -179,7 +179,14 @@ def gptq_prepare_hinv_static(H, damp=0.01, U=None, dev_info=None, stream=None):
         return U, dev_info
 
 
-def gptq_quantize_layer(W, U, bits, group_size=0, sym=False, block=128, ws=None, dev_info=None, stream=None):
+GRID_SYMMETRIC, GRID_FP16_SCALES = 1, 2
+
+
+def _grid_flags(sym, scale_fp16):
+    return (GRID_SYMMETRIC if sym else 0) | (GRID_FP16_SCALES if scale_fp16 else 0)
+
+
+def gptq_quantize_layer(W, U, bits, group_size=0, sym=False, block=128, ws=None, dev_info=None, stream=None, scale_fp16=False):
     """Algorithm 1 on fp16 W (R x C) with U from gptq_prepare_hinv.
     Returns dict(qweight uint32 [R, C*f/32] (as int32 tensor), scales [R,G], zeros [R,G], loss double[1], dev_info)."""
     with _alloc_on(stream):
@@ -195,7 +202,7 @@ def gptq_quantize_layer(W, U, bits, group_size=0, sym=False, block=128, ws=None,
         loss = torch.zeros(1, dtype=torch.float64, device=dev)
         dev_info = torch.zeros(2, dtype=torch.int32, device=dev) if dev_info is None else dev_info
         ws = _ws(_lib.gptq_quantize_workspace_bytes(R, C, bits, group_size, block), dev, ws)
-        st = _lib.gptq_quantize_layer(W.data_ptr(), U.data_ptr(), R, C, bits, group_size, int(bool(sym)), block,
+        st = _lib.gptq_quantize_layer(W.data_ptr(), U.data_ptr(), R, C, bits, group_size, _grid_flags(sym, scale_fp16), block,
                                       qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), loss.data_ptr(),
                                       ws.data_ptr(), ws.numel(), dev_info.data_ptr(), _stream_ptr(stream))
         if st != OK:
@@ -243,7 +250,7 @@ def gptq_solve_layer_host(W_host, X_host, bits, group_size=0, sym=False, block=1
     return out
 
 
-def gptq_rtn_layer(W, bits, group_size=0, sym=False, stream=None):
+def gptq_rtn_layer(W, bits, group_size=0, sym=False, stream=None, scale_fp16=False):
     """Round-to-nearest on the solver's grid, no error feedback.  Returns dict(qweight, scales, zeros)."""
     with _alloc_on(stream):
         _check(W, torch.float16, "W")
@@ -252,7 +259,7 @@ def gptq_rtn_layer(W, bits, group_size=0, sym=False, stream=None):
         qweight = torch.empty((R, C * field_bits(bits) // 32), dtype=torch.int32, device=W.device)
         scales = torch.empty((R, G), dtype=torch.float32, device=W.device)
         zeros = torch.empty((R, G), dtype=torch.float32, device=W.device)
-        st = _lib.gptq_rtn_layer(W.data_ptr(), R, C, bits, group_size, int(bool(sym)), qweight.data_ptr(), scales.data_ptr(),
+        st = _lib.gptq_rtn_layer(W.data_ptr(), R, C, bits, group_size, _grid_flags(sym, scale_fp16), qweight.data_ptr(), scales.data_ptr(),
                                  zeros.data_ptr(), _stream_ptr(stream))
         if st != OK:
             raise GptqError(st, "gptq_rtn_layer")

@@ -38,7 +38,7 @@ __global__ void lambda_kernel(const float* __restrict__ H, int C, float damp, do
 }
 
 // U <- upper triangle of (H + lambda I); strict lower triangle <- 0.
-__global__ void init_upper_damped_kernel(const float* __restrict__ H, float* __restrict__ U, int C,
+__global__ void init_upper_damped_kernel(const float* H, float* U, int C,
                                          const double* __restrict__ lam) {
   int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   int64_t total = (int64_t)C * C / 4;
@@ -398,7 +398,9 @@ gptq_status_t launch_split_rect(const float* src, int64_t ld_src, int rows, int 
 extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, float* U,
                                            void* ws, size_t ws_bytes, int* dev_info, void* stream) {
   using namespace gptq;
-  if (!H || !U || !dev_info || C <= 0 || C % 32 != 0 || H == U || !(damp >= 0.f)) return GPTQ_ERR_INVALID_ARG;
+  if (!H || !U || !dev_info || C <= 0 || C % 32 != 0 || !(damp >= 0.f)) return GPTQ_ERR_INVALID_ARG;
+  // U == H is allowed: lambda is taken from H's diagonal first, then every element of U is written from the element
+  // of H at the same position by the same thread.
   if (!aligned_to(H, 16) || !aligned_to(U, 16)) return GPTQ_ERR_INVALID_ARG;
   if (!ws || !aligned_to(ws, kAlign) || ws_bytes < gptq_prepare_hinv_workspace_bytes(C)) return GPTQ_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -32,7 +32,15 @@ constexpr int kSB = 32;  // columns held in registers at a time by the in-block 
 struct GridSpec {
   int maxq;        // largest code
   int symmetric;   // symmetric (or ternary) grid
+  int f16scale;    // scales rounded to fp16 (the stored model's precision, Section 5) before anything uses them
 };
+
+// The scale in the precision it will be stored in: fp16 when asked for (unless that would be 0 or infinite).
+__device__ __forceinline__ float storage_rounded(float scale, int f16scale) {
+  if (!f16scale) return scale;
+  const float s16 = __half2float(__float2half_rn(scale));
+  return (s16 > 0.f && isfinite(s16)) ? s16 : scale;
+}
 
 // Min-max grid of a set of weights with minimum mn and maximum mx (Section 5, Setup).  The range
 // is widened to contain 0 so the zero-point is an integer code; an all-zero set gets [-1, 1].
@@ -42,10 +50,10 @@ __device__ __forceinline__ void find_params(double mn, double mx, GridSpec g, fl
   if (xmin == 0.0 && xmax == 0.0) { xmin = -1.0; xmax = 1.0; }
   if (g.symmetric) {
     double a = fmax(fabs(xmin), xmax);
-    scale = (float)(2.0 * a / (double)g.maxq);
+    scale = storage_rounded((float)(2.0 * a / (double)g.maxq), g.f16scale);
     zero = (float)((g.maxq + 1) / 2);
   } else {
-    scale = (float)((xmax - xmin) / (double)g.maxq);
+    scale = storage_rounded((float)((xmax - xmin) / (double)g.maxq), g.f16scale);
     zero = (float)rint(-xmin / (double)scale);
   }
 }
@@ -498,7 +506,9 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   float* sE = w.take<float>((size_t)R);
   float* sEinv = w.take<float>((size_t)R);
   const int64_t ldw = B2;
-  GridSpec gs{bits == GPTQ_BITS_TERNARY ? 2 : (1 << bits) - 1, (sym != 0 || bits == GPTQ_BITS_TERNARY) ? 1 : 0};
+  GridSpec gs{bits == GPTQ_BITS_TERNARY ? 2 : (1 << bits) - 1, ((sym & GPTQ_GRID_SYMMETRIC) != 0 || bits == GPTQ_BITS_TERNARY) ? 1 : 0,
+              (sym & GPTQ_GRID_FP16_SCALES) ? 1 : 0};
+  if (sym & ~(GPTQ_GRID_SYMMETRIC | GPTQ_GRID_FP16_SCALES)) return GPTQ_ERR_INVALID_ARG;
 
   GPTQ_CUDA_TRY(cudaMemsetAsync(dev_info, 0, 2 * sizeof(int), s));
   GPTQ_CUDA_TRY(cudaMemsetAsync(loss, 0, sizeof(double), s));

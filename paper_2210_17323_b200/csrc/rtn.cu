@@ -7,7 +7,13 @@
 namespace gptq {
 namespace {
 
-struct RtnGrid { int maxq; int symmetric; };
+struct RtnGrid { int maxq; int symmetric; int f16scale; };
+
+__device__ __forceinline__ float storage_rounded(float scale, int f16scale) {
+  if (!f16scale) return scale;
+  const float s16 = __half2float(__float2half_rn(scale));
+  return (s16 > 0.f && isfinite(s16)) ? s16 : scale;
+}
 
 // One warp per (row, group): min / max of the group -> scale (rounded to fp32), integer zero-point.
 __global__ void rtn_params_kernel(const __half* __restrict__ W, int R, int C, int g, int G, RtnGrid grid,
@@ -28,10 +34,10 @@ __global__ void rtn_params_kernel(const __half* __restrict__ W, int R, int C, in
     if (xmin == 0.0 && xmax == 0.0) { xmin = -1.0; xmax = 1.0; }
     float scale, zero;
     if (grid.symmetric) {
-      scale = (float)(2.0 * fmax(fabs(xmin), xmax) / (double)grid.maxq);
+      scale = storage_rounded((float)(2.0 * fmax(fabs(xmin), xmax) / (double)grid.maxq), grid.f16scale);
       zero = (float)((grid.maxq + 1) / 2);
     } else {
-      scale = (float)((xmax - xmin) / (double)grid.maxq);
+      scale = storage_rounded((float)((xmax - xmin) / (double)grid.maxq), grid.f16scale);
       zero = (float)rint(-xmin / (double)scale);
     }
     scales[wid] = scale; zeros[wid] = zero;
@@ -72,7 +78,9 @@ extern "C" gptq_status_t gptq_rtn_layer(const void* W_fp16, int R, int C, int bi
   const int g = group_size > 0 ? group_size : C;
   if (C % g != 0) return GPTQ_ERR_INVALID_ARG;
   const int G = C / g, f = bits == GPTQ_BITS_TERNARY ? 2 : bits;
-  RtnGrid grid{bits == GPTQ_BITS_TERNARY ? 2 : (1 << bits) - 1, (sym != 0 || bits == GPTQ_BITS_TERNARY) ? 1 : 0};
+  if (sym & ~(GPTQ_GRID_SYMMETRIC | GPTQ_GRID_FP16_SCALES)) return GPTQ_ERR_INVALID_ARG;
+  RtnGrid grid{bits == GPTQ_BITS_TERNARY ? 2 : (1 << bits) - 1, ((sym & GPTQ_GRID_SYMMETRIC) != 0 || bits == GPTQ_BITS_TERNARY) ? 1 : 0,
+               (sym & GPTQ_GRID_FP16_SCALES) ? 1 : 0};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const __half* W = static_cast<const __half*>(W_fp16);
   {

@@ -166,6 +166,47 @@ def test_quantize_layer_per_block_form_matches_oracle(B, R, C, bits, group, sym,
     assert (a == b).mean() >= 0.999
 
 
+@pytest.mark.parametrize("bits,group,sym", [(4, 0, False), (3, 128, False), (O.BITS_TERNARY, 8, False), (4, 64, True)])
+def test_quantize_and_rtn_with_fp16_scales(B, bits, group, sym):
+    """Scales rounded to fp16 when the grid is fixed (the stored model's scale precision, Section 5): solver and RTN
+    against the oracle run with the same option; returned scales are fp16-representable."""
+    R, C = 96, 1024
+    L = _layer(R, C, 2 * C + 64, cfg=5)
+    W16 = L.w()
+    H = O.hessian_accumulate(np.zeros((C, C)), L.x_bits())
+    U32 = O.cholesky_inverse_upper(O.dampen(H, 0.01)[0]).astype(np.float32)
+    ref = O.quantize_layer(W16, U32.astype(np.float64), bits, group, sym, 128, scale_fp16=True)
+    out = B.gptq_quantize_layer(torch.from_numpy(W16).cuda(), torch.from_numpy(U32).cuda(), bits, group, sym, 128, scale_fp16=True)
+    torch.cuda.synchronize()
+    assert out["dev_info"].tolist()[0] == 0
+    gpu = dict(qweight=out["qweight"].cpu().numpy(), scales=out["scales"].cpu().numpy(), zeros=out["zeros"].cpu().numpy(),
+               loss=out["loss"].item())
+    check_quantize_outputs(gpu, ref, W16, bits, C, H)
+    assert np.array_equal(gpu["scales"], gpu["scales"].astype(np.float16).astype(np.float32))
+    rt = B.gptq_rtn_layer(torch.from_numpy(W16).cuda(), bits, group, sym, scale_fp16=True)
+    codes_ref, _ = O.rtn(W16, bits, group, sym, scale_fp16=True)
+    assert np.array_equal(O.unpack_codes(rt["qweight"].cpu().numpy().view(np.uint32), bits, C), codes_ref)
+    # flag bits beyond the two defined ones are rejected
+    Wd = torch.from_numpy(W16).cuda()
+    st = B._lib.gptq_rtn_layer(Wd.data_ptr(), R, C, 4, 0, 4, rt["qweight"].data_ptr(), rt["scales"].data_ptr(),
+                               rt["zeros"].data_ptr(), None)
+    assert st == B.ERR_INVALID_ARG
+
+
+def test_prepare_hinv_in_place(B):
+    """U may be the same buffer as H: the factor replaces the Hessian."""
+    C = 1280
+    L = _layer(8, C, 3000, cfg=4)
+    H32 = O.hessian_accumulate(np.zeros((C, C)), L.x_bits()).astype(np.float32)
+    Uref = O.cholesky_inverse_upper(O.dampen(H32.astype(np.float64), 0.01)[0])
+    Hd = torch.from_numpy(H32).cuda()
+    U, info = B.gptq_prepare_hinv(Hd, 0.01, U=Hd)
+    torch.cuda.synchronize()
+    assert info.tolist() == [0, 0] and U.data_ptr() == Hd.data_ptr()
+    assert rel_fro(Hd.cpu().numpy(), Uref) <= TOL_U_FRO
+    assert np.array_equal(Hd.cpu().numpy(), np.triu(Hd.cpu().numpy()))
+
+
 def test_quantize_block_size_invariance_on_gpu(B):
     R, C = 128, 1024
     L = _layer(R, C, 3000, cfg=7)
@@ -409,3 +450,54 @@ def test_dequantize_and_matvec_match_oracle(B, bits, group, C):
     mag = np.repeat(scales, gsz, 1) * (codes + np.repeat(zeros, gsz, 1))
     bound = 4e-6 * (mag @ np.abs(x16.astype(np.float64))) + 1e-12
     assert (np.abs(y - yref) <= bound).all(), float(np.max(np.abs(y - yref) / bound))
+
+
+def test_block_pipeline_shares_hessian_and_factor_for_q_k_v(B, D):
+    """Section 5, Setup: a block's layers are quantized from one pass of calibration inputs.  q, k and v read the same
+    input, so the pipeline computes ONE Hessian and ONE factor for them; every member's outputs are bit-identical to
+    stages 2-3 run alone on the group's Hessian and agree with a fully separate solve of that layer; o / fc1 / fc2
+    keep their own inputs."""
+    from paper_2210_17323_b200 import pipeline as P
+    C, F, m = 512, 1280, 3000
+    layers = [WL.Layer(7, 0, k, C, C, m) for k in ("q", "k", "v", "o")] + [WL.Layer(7, 0, "fc1", F, C, m), WL.Layer(7, 0, "fc2", C, F, m)]
+    shared_x = D.fill_x(layers[0])                         # q's input is also k's and v's
+    groups = P.group_by_shared_input(layers, lambda L: shared_x if L.kind == "q" else D.fill_x(L), D.fill_w)
+    assert [[mm.name for mm in g.members] for g in groups] == [[layers[0].name, layers[1].name, layers[2].name], [layers[3].name],
+                                                               [layers[4].name], [layers[5].name]]
+    solver = P.BlockSolver(groups, 3, 128, False, 128, 0.01)
+    solver.enqueue()
+    torch.cuda.synchronize()
+    solver.check()
+    res = solver.results()
+    H_of = {mm["m"].name: st["H"] for st in solver.state for mm in st["members"]}
+    assert H_of[layers[0].name] is H_of[layers[1].name] is H_of[layers[2].name]          # one Hessian for q, k, v
+    for L in layers:
+        # (a) stages 2 and 3 alone from the group's Hessian: bit-identical (they are deterministic at these sizes), so the
+        #     pipeline handed the right factor and the right weights to every member
+        U, info = B.gptq_prepare_hinv(H_of[L.name], 0.01)
+        out = B.gptq_quantize_layer(D.fill_w(L), U, 3, 128, False, 128)
+        torch.cuda.synchronize()
+        assert info.tolist()[0] == 0
+        for key in ("qweight", "scales", "zeros"):
+            assert torch.equal(out[key], res[L.name][key]), (L.name, key)
+        # (b) a fully separate solve with its own Hessian of the same input: the Hessian kernel adds token ranges with
+        #     floating-point reductions whose order varies from run to run, so equality is up to that rounding
+        X = shared_x if L.kind in ("q", "k", "v") else D.fill_x(L)
+        H = torch.zeros((L.C, L.C), dtype=torch.float32, device="cuda")
+        B.gptq_hessian_accumulate(H, X)
+        assert rel_fro(H.cpu().numpy(), H_of[L.name].cpu().numpy()) <= 1e-6
+        U2, _ = B.gptq_prepare_hinv(H, 0.01)
+        out2 = B.gptq_quantize_layer(D.fill_w(L), U2, 3, 128, False, 128)
+        torch.cuda.synchronize()
+        a = O.unpack_codes(out2["qweight"].cpu().numpy().view(np.uint32), 3, L.C)
+        b = O.unpack_codes(res[L.name]["qweight"].cpu().numpy().view(np.uint32), 3, L.C)
+        assert (a == b).mean() >= 0.999 and np.abs(a - b).max() <= 1
+        assert rel_fro(out2["scales"].cpu().numpy(), res[L.name]["scales"].cpu().numpy()) <= 1e-5
+    # and one member against the oracle, end to end
+    L = layers[1]
+    bits_host = shared_x.view(torch.int16).cpu().numpy().view(np.uint16)
+    ref = O.solve_layer(L.w(), bits_host, 3, 128, False, 128, 0.01)
+    o = res[L.name]
+    gpu = dict(qweight=o["qweight"].cpu().numpy(), scales=o["scales"].cpu().numpy(), zeros=o["zeros"].cpu().numpy(),
+               loss=o["loss"].item())
+    check_quantize_outputs(gpu, ref, L.w(), 3, L.C, ref["H"])

@@ -37,6 +37,16 @@ def _worker(rank, world, port, out_dir):
         U = O.cholesky_inverse_upper(O.dampen(H, 0.01)[0])
         part = O.quantize_layer(L.w(rows=np.arange(rows.start, rows.stop)), U, 4, 0, False, 32)
         np.save(os.path.join(out_dir, f"codes{rank}.npy"), part["codes"])
+        # strong scaling of a whole layer: token-sharded Hessian + one all-reduce, factor on every rank, row stripes
+        L2 = WL.Layer(7, 1, "k", 21, 32, 257)
+        Xi = np.round(O.bf16_bits_to_f64(L2.x_bits()) * 4).clip(-64, 64)         # small integers: sums are exact in any order
+        rows2, out2, H2, _ = multi.solve_layer_sharded(
+            L2.n_tokens, L2.R, world, rank,
+            hessian_of_tokens=lambda tr: torch.from_numpy(2.0 * Xi[tr.start:tr.stop].T @ Xi[tr.start:tr.stop]),
+            factor_of=lambda H: O.cholesky_inverse_upper(O.dampen(H.numpy(), 0.01)[0]),
+            quantize_rows=lambda rr, U: O.quantize_layer(L2.w(rows=np.arange(rr.start, rr.stop)), U, 3, 16, False, 16))
+        assert np.array_equal(H2.numpy(), 2.0 * Xi.T @ Xi)                          # every rank holds the full Hessian
+        np.save(os.path.join(out_dir, f"strong{rank}.npy"), out2["codes"])
         # timing reduction: the job's time is the slowest rank's; throughput sums
         assert multi.max_over_ranks(10.0 + rank) == 10.0 + world - 1
         assert multi.sum_over_ranks(float(len(rows))) == float(L.R)
@@ -54,6 +64,12 @@ def test_two_ranks_shard_rows_and_reduce_timing(tmp_path):
     full = O.quantize_layer(L.w(), U, 4, 0, False, 32)
     joined = np.concatenate([np.load(tmp_path / f"codes{r}.npy") for r in range(world)])
     assert np.array_equal(joined, full["codes"])
+    L2 = WL.Layer(7, 1, "k", 21, 32, 257)
+    Xi = np.round(O.bf16_bits_to_f64(L2.x_bits()) * 4).clip(-64, 64)
+    U2 = O.cholesky_inverse_upper(O.dampen(2.0 * Xi.T @ Xi, 0.01)[0])
+    full2 = O.quantize_layer(L2.w(), U2, 3, 16, False, 16)
+    joined2 = np.concatenate([np.load(tmp_path / f"strong{r}.npy") for r in range(world)])
+    assert np.array_equal(joined2, full2["codes"])
 
 
 def test_shard_units_is_a_partition():

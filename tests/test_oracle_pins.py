@@ -354,6 +354,46 @@ def test_group_grid_is_taken_from_current_weights(bits, group, block):
     assert differs >= 0.9 * R * (C // group - 1)
 
 
+# ------------------------------------------------------------------ fp16 scale storage (Section 5, Extreme Quantization)
+@pytest.mark.parametrize("bits,group", [(4, 0), (3, 16), (2, 32), (O.BITS_TERNARY, 8)])
+def test_fp16_scale_option(bits, group):
+    """Section 5 counts one FP16 scale per group in the stored model.  With scale_fp16 the grid is built on the
+    fp16-rounded scale: the returned scale is the fp16 value nearest to the unrounded one, the zero-point is derived
+    from THAT scale, every code is the nearest level of THAT grid (diagonal H: no feedback, so codes are plain
+    nearest-level choices), and scale * (code - zero) needs no rounding in fp32, so the fp16-scale model
+    dequantizes to exactly the values the solver compensated for."""
+    r = RNG(41)
+    R, C = 16, 64
+    W = (r.normal(size=(R, C)) * 0.02).astype(np.float16)
+    Wd = W.astype(np.float64)
+    g = group if group > 0 else C
+    maxq = O.maxq_of(bits)
+    U = O.cholesky_inverse_upper(np.diag(np.exp(r.normal(size=C))))
+    out = O.quantize_layer(W, U, bits, group, False, block=16, scale_fp16=True)
+    plain = O.quantize_layer(W, U, bits, group, False, block=16)
+    s16 = out["scales"]
+    assert np.array_equal(s16, s16.astype(np.float16).astype(np.float64))          # fp16-representable
+    if bits != O.BITS_TERNARY:        # (a ternary scale is max|w| of fp16 weights: already an fp16 value)
+        assert not np.array_equal(s16, plain["scales"])                            # and it did change something
+    for gi in range(C // g):
+        seg = Wd[:, gi * g:(gi + 1) * g]
+        lo, hi = np.minimum(seg.min(1), 0), np.maximum(seg.max(1), 0)
+        exact = (2 * np.maximum(-lo, hi) if bits == O.BITS_TERNARY else (hi - lo)) / maxq
+        for rr in range(R):
+            s = np.float16(s16[rr, gi])
+            for nb in (np.nextafter(s, np.float16(0)), np.nextafter(s, np.float16(np.inf))):
+                assert abs(float(s) - exact[rr]) <= abs(float(nb) - exact[rr]) * (1 + 1e-7)   # nearest fp16 value
+            z = out["zeros"][rr, gi]
+            if bits != O.BITS_TERNARY:
+                assert z == np.rint(-lo[rr] / float(s))                            # zero-point from the ROUNDED scale
+            for c in range(gi * g, (gi + 1) * g):
+                d = np.abs(np.array(_grid_values(float(s), z, maxq)) - Wd[rr, c])
+                assert d[out["codes"][rr, c]] == d.min()
+    prod32 = (np.repeat(s16, g, 1).astype(np.float32) * (out["codes"] - np.repeat(out["zeros"], g, 1)).astype(np.float32))
+    assert np.array_equal(prod32.astype(np.float64), out["W_hat"])                 # exact in fp32
+    assert np.array_equal(O.rtn(W, bits, group, False, scale_fp16=True)[0], out["codes"])
+
+
 # ------------------------------------------------------------------ P8: packed layout
 def _golden_pack_vectors():
     path = os.path.join(os.path.dirname(__file__), "golden", "pack_vectors.txt")
