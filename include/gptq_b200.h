@@ -70,6 +70,13 @@ const char* gptq_status_string(gptq_status_t status);
  * launched in the calling process so far.  Host-side counter; thread-safe. */
 uint64_t gptq_launch_count(void);
 
+/* Test hook (no counterpart in the paper).  Every wait inside the tensor-core kernels is bounded: when it runs out the
+ * kernel records GPTQ_ERR_TIMEOUT in dev_info, every role leaves through its own bounded wait, tensor memory is freed and
+ * the kernel returns -- it never hangs or traps.  This call lets a test see that path: it sets the limit of the waits
+ * (nanoseconds; 0 restores the default of 4 s) and the index of one work item whose operand loads the producer leaves
+ * out (-1: none), for kernels of the current device launched afterwards.  Synchronises the device.  Restore with (0, -1). */
+gptq_status_t gptq_debug_wait_test(uint64_t wait_limit_ns, int skip_loads_of_item);
+
 /* ------------------------------------------------------------------ stage 1
  * H += 2 * sum_t x_t x_t^T                     (Section 2: H_F = 2 X_F X_F^T;
  *                                               Algorithm 1 caption: 2 X X^T)

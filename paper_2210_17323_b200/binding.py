@@ -38,6 +38,8 @@ def _load():
     lib.gptq_status_string.argtypes = [c.c_int]
     lib.gptq_launch_count.restype = c.c_uint64
     lib.gptq_launch_count.argtypes = []
+    lib.gptq_debug_wait_test.restype = c.c_int
+    lib.gptq_debug_wait_test.argtypes = [c.c_uint64, c.c_int]
     lib.gptq_hessian_workspace_bytes.restype = c.c_size_t
     lib.gptq_hessian_workspace_bytes.argtypes = [c.c_int, c.c_int64]
     lib.gptq_hessian_accumulate.restype = c.c_int
@@ -80,6 +82,13 @@ def status_string(status) -> str:
 
 def gptq_launch_count() -> int:
     return int(_lib.gptq_launch_count())
+
+
+def gptq_debug_wait_test(wait_limit_ns=0, skip_loads_of_item=-1):
+    """Test hook: limit of the kernels' bounded waits and one work item whose loads are left out; (0, -1) restores."""
+    st = _lib.gptq_debug_wait_test(int(wait_limit_ns), int(skip_loads_of_item))
+    if st != OK:
+        raise GptqError(st, "gptq_debug_wait_test")
 
 
 def _stream_ptr(stream):

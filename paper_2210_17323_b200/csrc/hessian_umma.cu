@@ -255,4 +255,6 @@ gptq_status_t hessian_umma(float* H, const __nv_bfloat16* X, int64_t n_tokens, i
   return GPTQ_OK;
 }
 
+cudaError_t hessian_set_wait_test_knobs(unsigned long long limit_ns, int skip_item) { return set_wait_test_knobs(limit_ns, skip_item); }
+
 }  // namespace gptq

@@ -624,3 +624,7 @@ extern "C" gptq_status_t gptq_prepare_hinv_static(const float* H, float damp, in
   // temporary are all written by this call before they are read, so stale contents are harmless.
   return gptq_prepare_hinv(H, damp, C, U, scratch, kStaticScratchBytes, dev_info, stream);
 }
+
+namespace gptq {
+cudaError_t hinv_set_wait_test_knobs(unsigned long long limit_ns, int skip_item) { return set_wait_test_knobs(limit_ns, skip_item); }
+}  // namespace gptq

@@ -590,6 +590,10 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   return GPTQ_OK;
 }
 
+namespace gptq {
+cudaError_t quantize_set_wait_test_knobs(unsigned long long limit_ns, int skip_item) { return set_wait_test_knobs(limit_ns, skip_item); }
+}  // namespace gptq
+
 extern "C" int gptq_set_stage3_variant(int variant) {
   if (variant != 0 && variant != 1) return gptq::g_stage3_variant.load();
   return gptq::g_stage3_variant.exchange(variant);

@@ -45,14 +45,19 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 constexpr uint64_t kWaitLimitNs = 4000000000ull;  // 4 s: far beyond any legitimate wait in these kernels
+// Test knobs (one copy per translation unit, set through gptq_debug_wait_test): the limit of every bounded wait, and the
+// index of one work item whose operand loads the producer leaves out, so that the waits downstream of it run out.
+static __device__ unsigned long long g_wait_limit_ns = kWaitLimitNs;
+static __device__ int g_skip_loads_of_item = -1;
 
 // Waits for the phase with the given parity; false if the limit ran out.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
+  const uint64_t limit = g_wait_limit_ns;
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 0x3FF) == 0 && global_timer_ns() - t0 > kWaitLimitNs) return false;
+    if ((++spins & 0x3FF) == 0 && global_timer_ns() - t0 > limit) return false;
   }
   return true;
 }
@@ -155,6 +160,13 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 }  // namespace umma
 
 int device_sm_count();
+
+// Host side of the test knobs above, for the translation unit that includes this header.
+static inline cudaError_t set_wait_test_knobs(unsigned long long limit_ns, int skip_item) {
+  cudaError_t e = cudaMemcpyToSymbol(umma::g_wait_limit_ns, &limit_ns, sizeof(limit_ns));
+  if (e != cudaSuccess) return e;
+  return cudaMemcpyToSymbol(umma::g_skip_loads_of_item, &skip_item, sizeof(skip_item));
+}
 
 // Host: encodes a 2-D tiled tensor map (row-major matrix, `inner` contiguous elements per row)
 // with 128-byte swizzle.  The driver entry point is looked up at run time, so the library does

@@ -75,7 +75,8 @@ umma_pipe_kernel(const __grid_constant__ typename Traits::Maps maps, const int n
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1)) { report_error(dev_info, GPTQ_ERR_TIMEOUT, 1); ok = false; break; }
           mbar_arrive_expect_tx(&full[stage], STAGE_BYTES);
-          Traits::load(tiles + (size_t)stage * STAGE_BYTES, maps, m0, n0, kb, &full[stage]);
+          if (idx != g_skip_loads_of_item)      // (test knob: an item whose loads never come, see umma.cuh)
+            Traits::load(tiles + (size_t)stage * STAGE_BYTES, maps, m0, n0, kb, &full[stage]);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
       }

@@ -69,8 +69,9 @@ umma_pipe2_kernel(const __grid_constant__ typename Traits::Maps maps, const int 
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1)) { report_error(dev_info, GPTQ_ERR_TIMEOUT, 21); ok = false; break; }
           if (rank == 0) mbar_arrive_expect_tx(&full[stage], 2 * STAGE_BYTES);   // bytes of both CTAs
-          Traits::load(tiles + (size_t)stage * STAGE_BYTES, maps, m0 + BM_CTA * (int)rank, n0 + (BN / 2) * (int)rank, kb,
-                       &full[stage]);
+          if (idx != g_skip_loads_of_item)      // (test knob: an item whose loads never come, see umma.cuh)
+            Traits::load(tiles + (size_t)stage * STAGE_BYTES, maps, m0 + BM_CTA * (int)rank, n0 + (BN / 2) * (int)rank, kb,
+                         &full[stage]);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
       }

@@ -501,3 +501,28 @@ def test_block_pipeline_shares_hessian_and_factor_for_q_k_v(B, D):
     gpu = dict(qweight=o["qweight"].cpu().numpy(), scales=o["scales"].cpu().numpy(), zeros=o["zeros"].cpu().numpy(),
                loss=o["loss"].item())
     check_quantize_outputs(gpu, ref, L.w(), 3, L.C, ref["H"])
+
+
+def test_bounded_waits_report_timeout_and_the_gpu_stays_usable(B, D):
+    """Every wait in the tensor-core kernels is bounded.  With the limit lowered to 20 ms and the loads of one work item
+    left out (a barrier that nothing completes), the Hessian kernel must come back by itself with GPTQ_ERR_TIMEOUT in
+    dev_info -- every role leaving through its own bounded wait, tensor memory freed -- and the next, normal call on the
+    same context must work and give the right Hessian."""
+    L = _layer(8, 768, 4096, cfg=3)
+    X = D.fill_x(L)
+    H = torch.zeros((L.C, L.C), dtype=torch.float32, device="cuda")
+    info = torch.zeros(2, dtype=torch.int32, device="cuda")
+    B.gptq_debug_wait_test(20_000_000, 0)
+    try:
+        B.gptq_hessian_accumulate(H, X, dev_info=info)
+        torch.cuda.synchronize()
+        st, where = info.tolist()
+        assert st == B.ERR_TIMEOUT and where in (21, 22, 23, 24), (st, where)
+    finally:
+        B.gptq_debug_wait_test(0, -1)
+    H.zero_()
+    B.gptq_hessian_accumulate(H, X, dev_info=info)
+    torch.cuda.synchronize()
+    assert info.tolist() == [0, 0]
+    Href = O.hessian_accumulate(np.zeros((L.C, L.C)), L.x_bits())
+    assert rel_fro(H.cpu().numpy(), Href) <= TOL_H_FRO
