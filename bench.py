@@ -559,6 +559,62 @@ def run_gpu_strong(args, wl):
     return 0
 
 
+def run_block_sweep(args, wl):
+    """Stage 3 across block sizes and forms (config 4 asks for this sweep to profile the lazy update): one layer, one
+    Hessian and factor, then gptq_quantize_layer timed for B in {32, 64, 128, 256} x {row-stripe, per-inner-block} x grids."""
+    import torch
+    from paper_2210_17323_b200 import binding as B
+    from paper_2210_17323_b200.synth import device as D
+
+    torch.cuda.set_device(0)
+    L = wl.layers[0] if not args.layer else wl.layers[0]
+    X = D.fill_x(L)
+    H = torch.zeros((L.C, L.C), dtype=torch.float32, device="cuda")
+    B.gptq_hessian_accumulate(H, X)
+    del X
+    U, info = B.gptq_prepare_hinv(H, wl.damp)
+    W = D.fill_w(L)
+    torch.cuda.synchronize()
+    assert info.tolist()[0] == 0
+    peaks = _peaks()
+    rows = []
+    for g in wl.grids:
+        base = None
+        for blk in (32, 64, 128, 256):
+            if g.group_size > 0 and (g.group_size % blk and blk % g.group_size):
+                continue
+            for variant in (1, 0):
+                B.gptq_set_stage3_variant(variant)
+                ws = torch.empty(B.gptq_quantize_workspace_bytes(L.R, L.C, g.bits, g.group_size, blk), dtype=torch.uint8, device="cuda")
+                out = None
+                ts = []
+                for it in range(max(2, args.warmup) + max(3, args.steps)):
+                    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    out = B.gptq_quantize_layer(W, U, g.bits, g.group_size, g.sym, blk, ws=ws)
+                    e1.record(); torch.cuda.synchronize()
+                    if it >= max(2, args.warmup):
+                        ts.append(e0.elapsed_time(e1))
+                ms = statistics.median(ts)
+                if base is None:
+                    base = out["qweight"].clone()
+                same = float((out["qweight"] == base).float().mean().item())
+                useful = L.R * (L.C * L.C - L.C * blk) / (ms * 1e-3) / 1e12
+                rows.append(dict(bits=g.bits, group_size=g.group_size, block=blk,
+                                 form="row-stripe" if (variant == 1 and blk <= 128) else "per-inner-block", ms=ms,
+                                 useful_tflops=useful, executed_tflops=3 * useful,
+                                 frac_of_bf16_sustained=3 * useful / peaks["bf16_sustained"],
+                                 packed_words_identical_to_first=same, loss=out["loss"].item()))
+    B.gptq_set_stage3_variant(1)
+    line = dict(metric="gptq_stage3_ms_by_block_size", unit="ms", value=min(r["ms"] for r in rows), n_gpus=1, higher_is_better=False,
+                data="synthetic", dtype="f64 working weights; fp16-pair (3 products) f32 update sums",
+                config=dict(workload=wl.name, layer=L.name, note="executed flops = 3 x useful R (C^2 - C B); peak = bf16 sustained "
+                            f"({peaks['source']}): the update contractions are kind::f16 tensor-core instructions"),
+                sweep=rows)
+    print(json.dumps(line))
+    return 0
+
+
 def run_e2e(args, wl, state, device_value):
     """Same metric end to end through the C ABI's host-buffer call: every step, for every layer (and grid),
     gptq_solve_layer_host streams X and W from pinned HOST memory to the device (copies overlapped with the
@@ -769,6 +825,13 @@ def main():
                          "packed matvec / dequantize kernels; block: Transformer-block pipeline in which q, k, v share "
                          "one Hessian and one factor")
     ap.add_argument("--grid", type=int, default=0, help="--mode block: index of the workload's grid to run")
+    ap.add_argument("--block", type=int, default=None, help="block size B of Algorithm 1 (default: the workload's, 128)")
+    ap.add_argument("--stage3-variant", type=int, default=1, choices=[0, 1],
+                    help="form of the loops inside an outer block: 1 row-stripe kernel (default), 0 one in-block kernel plus one "
+                         "small contraction per inner block")
+    ap.add_argument("--block-sweep", action="store_true",
+                    help="--mode sweep helper: time stage 3 of the workload's largest-Hessian layer for B in {32, 64, 128, 256} "
+                         "and both forms, on one Hessian and factor")
     ap.add_argument("--layer", default=None, metavar="RxCxTOKENS",
                     help="profile one layer of this shape (grid, block and damp of --workload) instead of the "
                          "whole layer set -- a small case of the same kernels for profiler captures")
@@ -779,8 +842,16 @@ def main():
         R, C, T = (int(v) for v in args.layer.lower().split("x"))
         wl = WL.Workload(wl.config_id, f"{wl.name}-single-{R}x{C}x{T}", (WL.Layer(wl.config_id, 0, "q", R, C, T),),
                          wl.grids, wl.block, wl.damp)
+    if args.block:
+        import dataclasses
+        wl = dataclasses.replace(wl, block=args.block)
     if args.impl == "reference":
         return run_reference(args, wl)
+    if args.block_sweep:
+        return run_block_sweep(args, wl)
+    if args.stage3_variant != 1:
+        from paper_2210_17323_b200 import binding as _B
+        _B.gptq_set_stage3_variant(args.stage3_variant)
     if args.mode == "inference":
         return run_inference(args, wl)
     if args.mode == "block":

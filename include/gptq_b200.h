@@ -104,7 +104,10 @@ gptq_status_t gptq_hessian_accumulate(float* H, const void* X_bf16, int64_t n_to
  *            U may be the same buffer as H (the factor then replaces the Hessian); partial overlap is not allowed.
  *   dev_info int[2]: [0] = GPTQ_OK or GPTQ_ERR_NOT_PD, [1] = index of the first
  *            non-positive pivot.  On NOT_PD the contents of U are unspecified
- *            but finite operations continue (no trap, no hang).
+ *            but finite operations continue (no trap, no hang).  GPTQ_ERR_NONFINITE: an entry of
+ *            the factor or of its inverse left the range of the scaled fp16 operand pairs the
+ *            tensor-core contractions use for C > 1024 (a Hessian so ill-conditioned that entries of
+ *            the inverse factor exceed ~100 times their row's diagonal entry); [1] = a row index.
  * Computed as the inverse of the upper factor of H~ = U~ U~^T, which equals
  * Cholesky(H~^-1)^T by uniqueness of the Cholesky factor.
  * Streams: for C > 1024 part of the work is enqueued on two internal streams (created once

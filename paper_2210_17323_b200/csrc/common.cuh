@@ -51,6 +51,22 @@ __device__ __forceinline__ void report_error(int* dev_info, int status, int deta
   if (dev_info && atomicCAS(dev_info, 0, status) == 0) dev_info[1] = detail;
 }
 
+// largest power of two <= x (x > 0, finite); 1 for anything else
+__device__ __forceinline__ float pow2_floor(float x) {
+  if (!(x > 0.f) || !isfinite(x)) return 1.f;
+  int e;
+  frexpf(x, &e);                       // x = m 2^e, m in [0.5, 1)
+  e = max(-100, min(100, e - 1));
+  return ldexpf(1.f, e);
+}
+// power of two s with s * x in [2^(top-1), 2^top) (x > 0, finite); 1 for anything else
+__device__ __forceinline__ float pow2_scale_to(float x, int top) {
+  if (!(x > 0.f) || !isfinite(x)) return 1.f;
+  int e;
+  frexpf(x, &e);
+  e = max(-100, min(100, top - e));
+  return ldexpf(1.f, e);
+}
 __device__ __forceinline__ int ceil_div_d(int a, int b) { return (a + b - 1) / b; }
 inline int ceil_div(int64_t a, int64_t b) { return static_cast<int>((a + b - 1) / b); }
 

@@ -90,7 +90,8 @@ struct Operand {
 
 // acc = A * B^T over K = A.cols = B.cols; epi must accumulate (it is called once per super-chunk).
 template <bool kTriLeft, bool kUpperOut, class EpiF>
-gptq_status_t launch(const Operand& A, const Operand& B, int M, int N, EpiF epi, int* dev_info, cudaStream_t stream) {
+gptq_status_t launch(const Operand& A, const Operand& B, int M, int N, EpiF epi, int* dev_info, cudaStream_t stream,
+                     int reserve_sms = 0) {
   const int64_t K = A.cols;
   if (M <= 0 || N <= 0 || K <= 0) return GPTQ_OK;
   Traits::Maps maps;
@@ -105,7 +106,8 @@ gptq_status_t launch(const Operand& A, const Operand& B, int M, int N, EpiF epi,
   if ((st = mk(&maps.b_lo, B.lo, B)) != GPTQ_OK) return st;
   TileItems<kTriLeft, kUpperOut> items{(M + BM - 1) / BM, (N + BN - 1) / BN, (int)((K + BK - 1) / BK), kSuperK / BK};
   const int n_sc = (items.kb_total + items.sc_kb - 1) / items.sc_kb;
-  return pipe2::launch_pipe2<Traits>(maps, (int64_t)items.tiles_m * items.tiles_n * n_sc, items, epi, dev_info, stream);
+  return pipe2::launch_pipe2<Traits>(maps, (int64_t)items.tiles_m * items.tiles_n * n_sc, items, epi, dev_info, stream,
+                                     reserve_sms);
 }
 
 // ---- splitting a (pre-scaled) fp32 value into an fp16 hi / lo pair --------------------------------

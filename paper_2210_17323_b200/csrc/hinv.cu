@@ -8,13 +8,14 @@
 // Two-level blocking.  128 x 128 diagonal blocks are factored and inverted in fp64 (registers) by
 // one CTA; products inside a 1024-column outer panel are small fp32 CUDA-core GEMMs
 // (gemm_small.cuh); everything that reaches across outer panels (almost all of the flops for
-// large C) is a left-looking fp32-accurate tensor-core contraction (3xTF32, tcgen05) over tf32
-// hi / lo copies of the factor that are written as each panel is finalised.  The launches of one
+// large C) is a left-looking fp32-accurate tensor-core contraction over fp16 hi / lo copies of the
+// factor (three kind::f16 products per term, gemm_umma_f16.cuh) that are written as each panel is
+// finalised.  fp16's narrow exponent range is met with exact power-of-two scalings (below).  The launches of one
 // call go to three streams (dependency chain, wide contractions, diagonal-block inverses): see
 // gptq_prepare_hinv below.
 #include "common.cuh"
 #include "gemm_small.cuh"
-#include "gemm_umma.cuh"
+#include "gemm_umma_f16.cuh"
 
 #include <mutex>
 
@@ -194,20 +195,74 @@ struct SubUpperOfsF32 {   // p[m][nofs + n] -= acc where that element is on or a
   }
 };
 
-// ---- tensor-core (3xTF32) epilogues: one thread, one row, 32 consecutive columns of a partial sum
+// ---- power-of-two scalings of the fp16 operand pairs ------------------------------------------------
+// With d_i = sqrt(H~_ii) (the norm of row i of the factor U~, H~ = U~ U~^T) and r_i the power of two with
+// r_i d_i in [0.5, 1), every operand is brought into fp16's range by exact scalings that the epilogues undo:
+//   rows of the factor          F'[i][k]  = U~[i][k] * r_i 2^12                          (|.| < 2^12: an entry is at most its row's norm)
+//   Schur-complement blocks     A'[i][j]  = A[i][j] * r_i 2^12 * r_j                     (|A_ij| <= d_i d_j)
+//   inverse of a diagonal block V'[j'][j] = V[j'][j] / r_j * g_j'                        (g_j' from the row's actual maximum, < 2^15)
+//   its transpose (phase 2)     VT'[j'][j] = V[j][j'] * gam_j'                           (gam_j' from the column's actual maximum, < 2^15)
+//   T = V^T U~^T (phase 2)      T'[j'][i] = T[j'][i] * r_i * gam_j' 2^-5                 (|.| < 2^15 by Cauchy-Schwarz)
+//   rows of the inverse         U'[i][k]  = U[i][k] / r_k * u_i                          (u_i brings the diagonal entry to ~2^9; saturated and
+//                                                                                         reported if an entry still leaves the range)
+// r_i 2^12 is called rs_i below.
+__global__ void factor_scales_kernel(const float* __restrict__ U, int C, float* __restrict__ r, float* __restrict__ rinv,
+                                     float* __restrict__ rs, float* __restrict__ rsinv) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= C) return;
+  const float ri = pow2_scale_to(sqrtf(U[(int64_t)i * C + i]), 0);
+  r[i] = ri; rinv[i] = 1.f / ri; rs[i] = ri * 4096.f; rsinv[i] = 1.f / (ri * 4096.f);
+}
+// One CTA per row / column index b of the w x w block V at D (leading dimension ld):
+//   g[b]   brings max_j |V[b][j]| / r[j] just below 2^15,  ginv = 1 / g
+//   gam[b] brings max_j |V[j][b]|        just below 2^15,  gam2inv = 2^5 / gam
+__global__ void panel_scales_kernel(const float* __restrict__ D, int64_t ld, int w, const float* __restrict__ rinv,
+                                    float* __restrict__ g, float* __restrict__ ginv, float* __restrict__ gam, float* __restrict__ gam2inv) {
+  __shared__ float red[2][32];
+  const int b = blockIdx.x;
+  float mr = 0.f, mc = 0.f;
+  for (int j = threadIdx.x; j < w; j += blockDim.x) {
+    mr = fmaxf(mr, fabsf(D[(int64_t)b * ld + j]) * rinv[j]);
+    mc = fmaxf(mc, fabsf(D[(int64_t)j * ld + b]));
+  }
+  for (int o = 16; o > 0; o >>= 1) { mr = fmaxf(mr, __shfl_xor_sync(0xffffffffu, mr, o)); mc = fmaxf(mc, __shfl_xor_sync(0xffffffffu, mc, o)); }
+  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = mr; red[1][threadIdx.x >> 5] = mc; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int k = 1; k < (int)(blockDim.x >> 5); ++k) { mr = fmaxf(mr, red[0][k]); mc = fmaxf(mc, red[1][k]); }
+    const float gg = pow2_scale_to(mr, 15), cc = pow2_scale_to(mc, 15);
+    g[b] = gg; ginv[b] = 1.f / gg; gam[b] = cc; gam2inv[b] = 32.f / cc;
+  }
+}
+// u[i] brings the diagonal entry of row i of the inverse, U_ii / r_i, to about 2^9;  uinv = 1 / u
+__global__ void inverse_row_scales_kernel(const float* __restrict__ U, int C, const float* __restrict__ rinv,
+                                          float* __restrict__ u, float* __restrict__ uinv) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= C) return;
+  const float ui = pow2_scale_to(fabsf(U[(int64_t)i * C + i]) * rinv[i], 9);
+  u[i] = ui; uinv[i] = 1.f / ui;
+}
+
+// ---- tensor-core epilogues: one thread, one row, 32 consecutive columns of a partial sum ---------------
+// Every epilogue multiplies the partial sum by sa[row] * sb[col] (powers of two: the operands' scalings undone).
 // dst[row][cofs + col] -= partial for elements on or above the diagonal (fp32 reductions).
 struct EpiSubUpperRed {
   float* p; int64_t ld; int cofs; int M, N;
+  const float* sa; const float* sb;
   __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
     if (row >= M || col0 >= N) return;
     float* d = p + (int64_t)row * ld + cofs + col0;
+    const float a = -sa[row];
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
       const int c = cofs + col0 + 4 * g;            // global column of the group's first element
-      if (c >= row) umma::red_add_v4(d + 4 * g, -v[4 * g], -v[4 * g + 1], -v[4 * g + 2], -v[4 * g + 3]);
+      const float4 b = *reinterpret_cast<const float4*>(sb + col0 + 4 * g);
+      const float x0 = v[4 * g] * a * b.x, x1 = v[4 * g + 1] * a * b.y, x2 = v[4 * g + 2] * a * b.z, x3 = v[4 * g + 3] * a * b.w;
+      if (c >= row) umma::red_add_v4(d + 4 * g, x0, x1, x2, x3);
       else if (c + 3 >= row) {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) if (c + u >= row) atomicAdd(d + 4 * g + u, -v[4 * g + u]);
+        if (c + 1 >= row) atomicAdd(d + 4 * g + 1, x1);
+        if (c + 2 >= row) atomicAdd(d + 4 * g + 2, x2);
+        atomicAdd(d + 4 * g + 3, x3);
       }
     }
   }
@@ -215,87 +270,112 @@ struct EpiSubUpperRed {
 // dst[row][col] -= partial over the whole rectangle (fp32 reductions).
 struct EpiSubRed {
   float* p; int64_t ld; int M, N;
+  const float* sa; const float* sb;
   __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
     if (row >= M || col0 >= N) return;
     float* d = p + (int64_t)row * ld + col0;
-#pragma unroll
-    for (int g = 0; g < 8; ++g) umma::red_add_v4(d + 4 * g, -v[4 * g], -v[4 * g + 1], -v[4 * g + 2], -v[4 * g + 3]);
-  }
-};
-// Stores the result as a tf32 hi / lo pair.  Only valid when the contraction is a single
-// super-chunk (K <= tf32x3::kSuperK), so that the partial sum IS the result.
-struct EpiStoreSplit {
-  float* hi; float* lo; int64_t ld; int M, N;
-  __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
-    if (row >= M || col0 >= N) return;
-    float4* h = reinterpret_cast<float4*>(hi + (int64_t)row * ld + col0);
-    float4* l = reinterpret_cast<float4*>(lo + (int64_t)row * ld + col0);
+    const float a = -sa[row];
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
-      float4 a, b;
-      tf32x3::split_tf32(v[4 * g], a.x, b.x); tf32x3::split_tf32(v[4 * g + 1], a.y, b.y);
-      tf32x3::split_tf32(v[4 * g + 2], a.z, b.z); tf32x3::split_tf32(v[4 * g + 3], a.w, b.w);
-      h[g] = a; l[g] = b;
+      const float4 b = *reinterpret_cast<const float4*>(sb + col0 + 4 * g);
+      umma::red_add_v4(d + 4 * g, v[4 * g] * a * b.x, v[4 * g + 1] * a * b.y, v[4 * g + 2] * a * b.z, v[4 * g + 3] * a * b.w);
     }
   }
 };
+// Stores partial * factor as an fp16 hi / lo pair.  Only valid when the contraction is a single super-chunk
+// (K <= f16x3::kSuperK), so that the partial sum IS the result.
+struct EpiStoreSplit {
+  __half* hi; __half* lo; int64_t ld; int M, N; float factor; int* dev_info;
+  __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
+    if (row >= M || col0 >= N) return;
+    uint4* h = reinterpret_cast<uint4*>(hi + (int64_t)row * ld + col0);
+    uint4* l = reinterpret_cast<uint4*>(lo + (int64_t)row * ld + col0);
+    bool sat = false;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      uint32_t hw[4], lw[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        __half h0, l0, h1, l1;
+        f16x3::split_f16(v[8 * g + 2 * u] * factor, h0, l0, sat);
+        f16x3::split_f16(v[8 * g + 2 * u + 1] * factor, h1, l1, sat);
+        hw[u] = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
+        lw[u] = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
+      }
+      h[g] = make_uint4(hw[0], hw[1], hw[2], hw[3]); l[g] = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+    }
+    if (sat) report_error(dev_info, GPTQ_ERR_NONFINITE, row);
+  }
+};
 
-// Stores the result as fp32 into the factor AND as a tf32 hi / lo pair into its split copies (same
-// offsets, leading dimension ldf).  Single super-chunk contractions only, like EpiStoreSplit.
+// Stores partial * sa[row] * sb[col] as fp32 into the factor AND partial * sb[col] (= that value * rs[row], the scaling of
+// the factor's rows) as an fp16 hi / lo pair into its split copies (same offsets, leading dimension ldf).
+// Single super-chunk contractions only, like EpiStoreSplit.
 struct EpiStoreF32AndSplit {
-  float* u; int64_t ldu; float* hi; float* lo; int64_t ldf; int M, N;
+  float* u; int64_t ldu; __half* hi; __half* lo; int64_t ldf; int M, N;
+  const float* sa; const float* sb; int* dev_info;
   __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
     if (row >= M || col0 >= N) return;
     float4* d = reinterpret_cast<float4*>(u + (int64_t)row * ldu + col0);
-    float4* h = reinterpret_cast<float4*>(hi + (int64_t)row * ldf + col0);
-    float4* l = reinterpret_cast<float4*>(lo + (int64_t)row * ldf + col0);
+    uint4* h = reinterpret_cast<uint4*>(hi + (int64_t)row * ldf + col0);
+    uint4* l = reinterpret_cast<uint4*>(lo + (int64_t)row * ldf + col0);
+    const float a = sa[row];
+    bool sat = false;
 #pragma unroll
-    for (int g = 0; g < 8; ++g) {
-      float4 a, b;
-      tf32x3::split_tf32(v[4 * g], a.x, b.x); tf32x3::split_tf32(v[4 * g + 1], a.y, b.y);
-      tf32x3::split_tf32(v[4 * g + 2], a.z, b.z); tf32x3::split_tf32(v[4 * g + 3], a.w, b.w);
-      d[g] = make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-      h[g] = a; l[g] = b;
+    for (int g = 0; g < 4; ++g) {
+      uint32_t hw[4], lw[4];
+      float x[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) x[e] = v[8 * g + e] * sb[col0 + 8 * g + e];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        __half h0, l0, h1, l1;
+        f16x3::split_f16(x[2 * e], h0, l0, sat);
+        f16x3::split_f16(x[2 * e + 1], h1, l1, sat);
+        hw[e] = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
+        lw[e] = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
+      }
+      d[2 * g] = make_float4(x[0] * a, x[1] * a, x[2] * a, x[3] * a);
+      d[2 * g + 1] = make_float4(x[4] * a, x[5] * a, x[6] * a, x[7] * a);
+      h[g] = make_uint4(hw[0], hw[1], hw[2], hw[3]); l[g] = make_uint4(lw[0], lw[1], lw[2], lw[3]);
     }
+    if (sat) report_error(dev_info, GPTQ_ERR_NONFINITE, row);
   }
 };
 
-// dst{hi,lo}[r][c] = split(src[r][c]) for r < rows, c < w (w a multiple of 4; both 16-byte aligned).
-__global__ void split_rect_kernel(const float* __restrict__ src, int64_t ld_src, int rows, int w,
-                                  float* __restrict__ dhi, float* __restrict__ dlo, int64_t ld_dst) {
+// dst{hi,lo}[r][c] = split(src[r][c] * sr[r] * sc[c]) for r < rows, c < w (w a multiple of 4; 16-byte aligned rows).
+__global__ void split_scaled_kernel(const float* __restrict__ src, int64_t ld_src, int rows, int w,
+                                    const float* __restrict__ sr, const float* __restrict__ sc,
+                                    __half* __restrict__ dhi, __half* __restrict__ dlo, int64_t ld_dst, int* dev_info) {
   const int q = w / 4;
   int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)rows * q) return;
   const int r = (int)(idx / q), c = (int)(idx % q) * 4;
-  float4 v = *reinterpret_cast<const float4*>(src + (int64_t)r * ld_src + c), h, l;
-  tf32x3::split_tf32(v.x, h.x, l.x); tf32x3::split_tf32(v.y, h.y, l.y);
-  tf32x3::split_tf32(v.z, h.z, l.z); tf32x3::split_tf32(v.w, h.w, l.w);
-  *reinterpret_cast<float4*>(dhi + (int64_t)r * ld_dst + c) = h;
-  *reinterpret_cast<float4*>(dlo + (int64_t)r * ld_dst + c) = l;
+  const float4 v = *reinterpret_cast<const float4*>(src + (int64_t)r * ld_src + c);
+  const float4 b = *reinterpret_cast<const float4*>(sc + c);
+  const float a = sr[r];
+  __half h[4], l[4];
+  bool sat = false;
+  f16x3::split_f16(v.x * a * b.x, h[0], l[0], sat); f16x3::split_f16(v.y * a * b.y, h[1], l[1], sat);
+  f16x3::split_f16(v.z * a * b.z, h[2], l[2], sat); f16x3::split_f16(v.w * a * b.w, h[3], l[3], sat);
+  *reinterpret_cast<uint2*>(dhi + (int64_t)r * ld_dst + c) =
+      make_uint2((uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16),
+                 (uint32_t)__half_as_ushort(h[2]) | ((uint32_t)__half_as_ushort(h[3]) << 16));
+  *reinterpret_cast<uint2*>(dlo + (int64_t)r * ld_dst + c) =
+      make_uint2((uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16),
+                 (uint32_t)__half_as_ushort(l[2]) | ((uint32_t)__half_as_ushort(l[3]) << 16));
+  if (sat) report_error(dev_info, GPTQ_ERR_NONFINITE, r);
 }
-// F{hi,lo}[r][c0 + c] = split(U[r][c0 + c]) for r < rows, c < w.
-__global__ void split_block_kernel(const float* __restrict__ U, int C, int c0, int w, int rows,
-                                   float* __restrict__ Fhi, float* __restrict__ Flo) {
-  const int q = w / 4;
-  int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (int64_t)rows * q) return;
-  const int r = (int)(idx / q), c = (int)(idx % q) * 4;
-  const int64_t o = (int64_t)r * C + c0 + c;
-  float4 v = *reinterpret_cast<const float4*>(U + o), h, l;
-  tf32x3::split_tf32(v.x, h.x, l.x); tf32x3::split_tf32(v.y, h.y, l.y);
-  tf32x3::split_tf32(v.z, h.z, l.z); tf32x3::split_tf32(v.w, h.w, l.w);
-  *reinterpret_cast<float4*>(Fhi + o) = h;
-  *reinterpret_cast<float4*>(Flo + o) = l;
-}
-// VT{hi,lo}[c][r] = split(U[j0 + r][j0 + c]) for r, c < w  (transpose of a diagonal block, ld = ldv).
-__global__ void split_diag_t_kernel(const float* __restrict__ U, int C, int j0,
-                                    float* __restrict__ Vhi, float* __restrict__ Vlo, int ldv) {
+// VT{hi,lo}[c][r] = split(U[j0 + r][j0 + c] * gam[c]) for r, c < w  (transpose of a diagonal block, ld = ldv).
+__global__ void split_diag_t_kernel(const float* __restrict__ U, int C, int j0, const float* __restrict__ gam,
+                                    __half* __restrict__ Vhi, __half* __restrict__ Vlo, int ldv) {
   __shared__ float t[32][33];
   const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
   t[threadIdx.y][threadIdx.x] = U[(int64_t)(j0 + r0 + threadIdx.y) * C + j0 + c0 + threadIdx.x];
   __syncthreads();
-  float h, l;
-  tf32x3::split_tf32(t[threadIdx.x][threadIdx.y], h, l);
+  __half h, l;
+  bool sat = false;
+  f16x3::split_f16(t[threadIdx.x][threadIdx.y] * gam[c0 + threadIdx.y], h, l, sat);
   const int64_t o = (int64_t)(c0 + threadIdx.y) * ldv + r0 + threadIdx.x;
   Vhi[o] = h; Vlo[o] = l;
 }
@@ -303,8 +383,10 @@ __global__ void split_diag_t_kernel(const float* __restrict__ U, int C, int j0,
 constexpr int kNB2 = 1024;   // outer panel width: contractions over everything outside it run on the tensor cores
 
 struct HinvWs {
-  double* lam; float* Dinv; float* T; float* Fhi; float* Flo; float* VThi; float* VTlo; float* TThi; float* TTlo;
-  float* Vhi[2]; float* Vlo[2]; float* TAhi; float* TAlo;
+  double* lam; float* Dinv; float* T; __half* Fhi; __half* Flo; __half* VThi; __half* VTlo; __half* TThi; __half* TTlo;
+  __half* Vhi[2]; __half* Vlo[2]; __half* TAhi; __half* TAlo;
+  float* r; float* rinv; float* rs; float* rsinv; float* u; float* uinv;      // [C] each
+  float* g[2]; float* ginv[2]; float* gam; float* gam2inv;                     // [kNB2] each
   size_t bytes;
 };
 HinvWs carve_hinv(void* ws, int C) {
@@ -314,18 +396,23 @@ HinvWs carve_hinv(void* ws, int C) {
   o.Dinv = w.take<float>((size_t)ceil_div(C, kNB) * kNB * kNB);   // inverses of the 128 x 128 diagonal blocks
   o.T = w.take<float>((size_t)C * kNB);                           // panel temporary (CUDA-core path)
   const bool outer = C > kNB2;
-  o.Fhi = w.take<float>(outer ? (size_t)C * C : 0);               // tf32 hi / lo of the factor as it is finalised
-  o.Flo = w.take<float>(outer ? (size_t)C * C : 0);
-  o.VThi = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);        // transposed inverse of an outer diagonal block
-  o.VTlo = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);
-  o.TThi = w.take<float>(outer ? (size_t)kNB2 * C : 0);           // (U~[0:j0, J] V_JJ)^T
-  o.TTlo = w.take<float>(outer ? (size_t)kNB2 * C : 0);
+  o.Fhi = w.take<__half>(outer ? (size_t)C * C : 0);              // scaled fp16 hi / lo of the factor as it is finalised
+  o.Flo = w.take<__half>(outer ? (size_t)C * C : 0);
+  o.VThi = w.take<__half>(outer ? (size_t)kNB2 * kNB2 : 0);       // transposed inverse of an outer diagonal block
+  o.VTlo = w.take<__half>(outer ? (size_t)kNB2 * kNB2 : 0);
+  o.TThi = w.take<__half>(outer ? (size_t)kNB2 * C : 0);          // (U~[0:j0, J] V_JJ)^T
+  o.TTlo = w.take<__half>(outer ? (size_t)kNB2 * C : 0);
   for (int i = 0; i < 2; ++i) {                                   // inverse of an outer diagonal block, two in flight
-    o.Vhi[i] = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);
-    o.Vlo[i] = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);
+    o.Vhi[i] = w.take<__half>(outer ? (size_t)kNB2 * kNB2 : 0);
+    o.Vlo[i] = w.take<__half>(outer ? (size_t)kNB2 * kNB2 : 0);
   }
-  o.TAhi = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);        // split copy of the row block above a diagonal block
-  o.TAlo = w.take<float>(outer ? (size_t)kNB2 * kNB2 : 0);
+  o.TAhi = w.take<__half>(outer ? (size_t)kNB2 * kNB2 : 0);       // split copy of the row block above a diagonal block
+  o.TAlo = w.take<__half>(outer ? (size_t)kNB2 * kNB2 : 0);
+  const size_t nc = outer ? (size_t)C : 0, np = outer ? (size_t)kNB2 : 0;
+  o.r = w.take<float>(nc); o.rinv = w.take<float>(nc); o.rs = w.take<float>(nc); o.rsinv = w.take<float>(nc);
+  o.u = w.take<float>(nc); o.uinv = w.take<float>(nc);
+  for (int i = 0; i < 2; ++i) { o.g[i] = w.take<float>(np); o.ginv[i] = w.take<float>(np); }
+  o.gam = w.take<float>(np); o.gam2inv = w.take<float>(np);
   o.bytes = w.off;
   return o;
 }
@@ -384,11 +471,11 @@ gptq_status_t get_async(HinvAsync** out) {
   return GPTQ_OK;
 }
 
-gptq_status_t launch_split_rect(const float* src, int64_t ld_src, int rows, int w, float* dhi, float* dlo,
-                                int64_t ld_dst, cudaStream_t s) {
+gptq_status_t launch_split_scaled(const float* src, int64_t ld_src, int rows, int w, const float* sr, const float* sc,
+                                  __half* dhi, __half* dlo, int64_t ld_dst, int* dev_info, cudaStream_t s) {
   if (rows <= 0 || w <= 0) return GPTQ_OK;
   const int64_t total = (int64_t)rows * (w / 4);
-  split_rect_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(src, ld_src, rows, w, dhi, dlo, ld_dst);
+  split_scaled_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(src, ld_src, rows, w, sr, sc, dhi, dlo, ld_dst, dev_info);
   GPTQ_LAUNCH_CHECK();
   return GPTQ_OK;
 }
@@ -429,6 +516,9 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
     GPTQ_LAUNCH_CHECK();
   }
   if (outer) {
+    // scalings of the fp16 operand pairs that follow from the damped diagonal alone
+    factor_scales_kernel<<<ceil_div(C, 256), 256, 0, s>>>(U, C, w.r, w.rinv, w.rs, w.rsinv);
+    GPTQ_LAUNCH_CHECK();
     GPTQ_CUDA_TRY(cudaEventRecord(as->fork, s));
     GPTQ_CUDA_TRY(cudaStreamWaitEvent(sb, as->fork, 0));
     GPTQ_CUDA_TRY(cudaStreamWaitEvent(ss, as->fork, 0));
@@ -453,14 +543,14 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
     if (K > 0) {
       if (J + 2 < n_outer) GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, as->b2[J + 2], 0));
       // C1
-      tf32x3::Operand A{w.Fhi + (int64_t)j0 * C + rows_p, w.Flo + (int64_t)j0 * C + rows_p, wj, K, C};
-      st = tf32x3::launch<false, true>(A, A, wj, wj, EpiSubUpperRed{D, C, 0, wj, wj}, dev_info, s);
+      f16x3::Operand A{w.Fhi + (int64_t)j0 * C + rows_p, w.Flo + (int64_t)j0 * C + rows_p, wj, K, C};
+      st = f16x3::launch<false, true>(A, A, wj, wj, EpiSubUpperRed{D, C, 0, wj, wj, w.rsinv + j0, w.rsinv + j0}, dev_info, s);
       if (st != GPTQ_OK) return st;
       if (j0 > 0) {
         // B1
         GPTQ_CUDA_TRY(cudaStreamWaitEvent(sb, as->c4[J + 1], 0));
-        tf32x3::Operand A1{w.Fhi + rows_p, w.Flo + rows_p, j0, K, C};
-        st = tf32x3::launch<false, false>(A1, A, j0, wj, EpiSubRed{U + j0, C, j0, wj}, dev_info, sb, reserve);
+        f16x3::Operand A1{w.Fhi + rows_p, w.Flo + rows_p, j0, K, C};
+        st = f16x3::launch<false, false>(A1, A, j0, wj, EpiSubRed{U + j0, C, j0, wj, w.rsinv, w.rsinv + j0}, dev_info, sb, reserve);
         if (st != GPTQ_OK) return st;
         GPTQ_CUDA_TRY(cudaEventRecord(as->b1[J], sb));
       }
@@ -504,18 +594,23 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
       GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, as->side_done, 0));
     }
     if (!outer || j0 == 0) continue;
-    float* Vhi = w.Vhi[J & 1]; float* Vlo = w.Vlo[J & 1];
-    if ((st = launch_split_rect(D, C, wj, wj, Vhi, Vlo, kNB2, s)) != GPTQ_OK) return st;
+    __half* Vhi = w.Vhi[J & 1]; __half* Vlo = w.Vlo[J & 1];
+    float* gJ = w.g[J & 1]; float* ginvJ = w.ginv[J & 1];
+    // V' = V / r (columns) * g (rows, from the rows' actual maxima); gam of this panel is recomputed in phase 2
+    panel_scales_kernel<<<wj, 256, 0, s>>>(D, C, wj, w.rinv + j0, gJ, ginvJ, w.gam, w.gam2inv);
+    GPTQ_LAUNCH_CHECK();
+    if ((st = launch_split_scaled(D, C, wj, wj, gJ, w.rinv + j0, Vhi, Vlo, kNB2, dev_info, s)) != GPTQ_OK) return st;
     GPTQ_CUDA_TRY(cudaEventRecord(as->c3[J], s));
-    tf32x3::Operand V{Vhi, Vlo, wj, wj, kNB2};
+    f16x3::Operand V{Vhi, Vlo, wj, wj, kNB2};
     const int r1 = j0 - kNB2;                       // first row of row block J-1
     // B2 (rows above row block J-1)
     if (r1 > 0) {
       GPTQ_CUDA_TRY(cudaStreamWaitEvent(sb, as->c3[J], 0));
-      if ((st = launch_split_rect(U + j0, C, r1, wj, w.TThi, w.TTlo, kNB2, sb)) != GPTQ_OK) return st;
-      tf32x3::Operand A2{w.TThi, w.TTlo, r1, wj, kNB2};
-      st = tf32x3::launch<false, false>(A2, V, r1, wj,
-                                        EpiStoreF32AndSplit{U + j0, C, w.Fhi + j0, w.Flo + j0, C, r1, wj}, dev_info, sb, reserve);
+      if ((st = launch_split_scaled(U + j0, C, r1, wj, w.rs, w.r + j0, w.TThi, w.TTlo, kNB2, dev_info, sb)) != GPTQ_OK) return st;
+      f16x3::Operand A2{w.TThi, w.TTlo, r1, wj, kNB2};
+      st = f16x3::launch<false, false>(A2, V, r1, wj,
+                                       EpiStoreF32AndSplit{U + j0, C, w.Fhi + j0, w.Flo + j0, C, r1, wj, w.rsinv, ginvJ, dev_info},
+                                       dev_info, sb, reserve);
       if (st != GPTQ_OK) return st;
     }
     GPTQ_CUDA_TRY(cudaEventRecord(as->b2[J], sb));
@@ -523,10 +618,11 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
     if (K > 0) GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, as->b1[J], 0));
     {
       const int64_t o = (int64_t)r1 * C + j0;
-      if ((st = launch_split_rect(U + o, C, kNB2, wj, w.TAhi, w.TAlo, kNB2, s)) != GPTQ_OK) return st;
-      tf32x3::Operand A4{w.TAhi, w.TAlo, kNB2, wj, kNB2};
-      st = tf32x3::launch<false, false>(A4, V, kNB2, wj,
-                                        EpiStoreF32AndSplit{U + o, C, w.Fhi + o, w.Flo + o, C, kNB2, wj}, dev_info, s);
+      if ((st = launch_split_scaled(U + o, C, kNB2, wj, w.rs + r1, w.r + j0, w.TAhi, w.TAlo, kNB2, dev_info, s)) != GPTQ_OK) return st;
+      f16x3::Operand A4{w.TAhi, w.TAlo, kNB2, wj, kNB2};
+      st = f16x3::launch<false, false>(A4, V, kNB2, wj,
+                                       EpiStoreF32AndSplit{U + o, C, w.Fhi + o, w.Flo + o, C, kNB2, wj, w.rsinv + r1, ginvJ, dev_info},
+                                       dev_info, s);
       if (st != GPTQ_OK) return st;
     }
     GPTQ_CUDA_TRY(cudaEventRecord(as->c4[J], s));
@@ -548,32 +644,34 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
   // rows above them: U[0:j0, J] = -U[0:j0, 0:j0] * (U~[0:j0, J] * V_JJ).
   for (int J = 1; J < n_outer; ++J) {
     const int j0 = J * kNB2, wj = (C - j0 < kNB2) ? C - j0 : kNB2, rows_p = j0 + wj;
-    if (J == 1) {                                   // split copy of the first panel of the inverse
-      int64_t total = (int64_t)kNB2 * (kNB2 / 4);
-      split_block_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(U, C, 0, kNB2, kNB2, w.Fhi, w.Flo);
+    if (J == 1) {                                   // row scales of the inverse; split copy of its first panel
+      inverse_row_scales_kernel<<<ceil_div(C, 256), 256, 0, s>>>(U, C, w.rinv, w.u, w.uinv);
       GPTQ_LAUNCH_CHECK();
+      if ((st = launch_split_scaled(U, C, kNB2, kNB2, w.u, w.rinv, w.Fhi, w.Flo, C, dev_info, s)) != GPTQ_OK) return st;
     }
+    panel_scales_kernel<<<wj, 256, 0, s>>>(U + (int64_t)j0 * C + j0, C, wj, w.rinv + j0, w.g[0], w.ginv[0], w.gam, w.gam2inv);
+    GPTQ_LAUNCH_CHECK();
     dim3 grid(ceil_div(wj, 32), ceil_div(wj, 32)), blk(32, 32);
-    split_diag_t_kernel<<<grid, blk, 0, s>>>(U, C, j0, w.VThi, w.VTlo, kNB2);
+    split_diag_t_kernel<<<grid, blk, 0, s>>>(U, C, j0, w.gam, w.VThi, w.VTlo, kNB2);
     GPTQ_LAUNCH_CHECK();
     // TT = V_JJ^T * U~[0:j0, J]^T   (wj x j0), written as a hi / lo pair (single super-chunk: K = wj)
     {
-      tf32x3::Operand A{w.VThi, w.VTlo, wj, wj, kNB2};
-      tf32x3::Operand B{w.Fhi + j0, w.Flo + j0, j0, wj, C};
-      st = tf32x3::launch<false, false>(A, B, wj, j0, EpiStoreSplit{w.TThi, w.TTlo, C, wj, j0}, dev_info, s);
+      f16x3::Operand A{w.VThi, w.VTlo, wj, wj, kNB2};
+      f16x3::Operand B{w.Fhi + j0, w.Flo + j0, j0, wj, C};
+      // partial = gam_j' rs_i T; stored as T r_i gam_j' 2^-5 = partial 2^-17
+      st = f16x3::launch<false, false>(A, B, wj, j0, EpiStoreSplit{w.TThi, w.TTlo, C, wj, j0, 1.f / 131072.f, dev_info}, dev_info, s);
       if (st != GPTQ_OK) return st;
     }
     GPTQ_CUDA_TRY(cudaMemset2DAsync(U + j0, (size_t)C * 4, 0, (size_t)wj * 4, j0, s));
     {
-      tf32x3::Operand A{w.Fhi, w.Flo, j0, j0, C};
-      tf32x3::Operand B{w.TThi, w.TTlo, wj, j0, C};
-      st = tf32x3::launch<true, false>(A, B, j0, wj, EpiSubRed{U + j0, C, j0, wj}, dev_info, s);
+      f16x3::Operand A{w.Fhi, w.Flo, j0, j0, C};
+      f16x3::Operand B{w.TThi, w.TTlo, wj, j0, C};
+      // partial = u_i gam_j' 2^-5 (sum_k U[i][k] T[j'][k])
+      st = f16x3::launch<true, false>(A, B, j0, wj, EpiSubRed{U + j0, C, j0, wj, w.uinv, w.gam2inv}, dev_info, s);
       if (st != GPTQ_OK) return st;
     }
     if (J + 1 < n_outer) {
-      int64_t total = (int64_t)rows_p * (wj / 4);
-      split_block_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(U, C, j0, wj, rows_p, w.Fhi, w.Flo);
-      GPTQ_LAUNCH_CHECK();
+      if ((st = launch_split_scaled(U + j0, C, rows_p, wj, w.u, w.rinv + j0, w.Fhi + j0, w.Flo + j0, C, dev_info, s)) != GPTQ_OK) return st;
     }
   }
   return GPTQ_OK;

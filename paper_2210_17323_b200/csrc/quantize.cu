@@ -315,22 +315,6 @@ __global__ void pack_kernel(const uint8_t* __restrict__ codes, int R, int C, int
 }
 
 // ---- power-of-two scales for the fp16 operand pairs ------------------------------------------------
-// largest power of two <= x (x > 0, finite); 1 for anything else
-__device__ __forceinline__ float pow2_floor(float x) {
-  if (!(x > 0.f) || !isfinite(x)) return 1.f;
-  int e;
-  frexpf(x, &e);                       // x = m 2^e, m in [0.5, 1)
-  e = max(-100, min(100, e - 1));
-  return ldexpf(1.f, e);
-}
-// power of two s with s * x in [2^(top-1), 2^top) (x > 0, finite); 1 for anything else
-__device__ __forceinline__ float pow2_scale_to(float x, int top) {
-  if (!(x > 0.f) || !isfinite(x)) return 1.f;
-  int e;
-  frexpf(x, &e);
-  e = max(-100, min(100, top - e));
-  return ldexpf(1.f, e);
-}
 // sK[k] = largest power of two <= U_kk; colmax[c] = 0
 __global__ void kscale_kernel(const float* __restrict__ U, int C, float* __restrict__ sK, uint32_t* __restrict__ colmax) {
   int k = blockIdx.x * blockDim.x + threadIdx.x;

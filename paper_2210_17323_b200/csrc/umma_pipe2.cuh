@@ -147,11 +147,12 @@ umma_pipe2_kernel(const __grid_constant__ typename Traits::Maps maps, const int 
 
 template <class Traits, class ItemF, class EpiF>
 gptq_status_t launch_pipe2(const typename Traits::Maps& maps, int64_t n_items, ItemF itemf, EpiF epi, int* dev_info,
-                           cudaStream_t stream) {
+                           cudaStream_t stream, int reserve_sms = 0) {
   if (n_items <= 0) return GPTQ_OK;
   if (n_items > 0x7FFFFFFF) return GPTQ_ERR_UNSUPPORTED;
   constexpr size_t smem = (size_t)Traits::STAGES * Traits::STAGE_BYTES + 1024 + 256;
-  const int pairs_max = device_sm_count() / 2;
+  int pairs_max = (device_sm_count() - reserve_sms) / 2;     // SMs left free for kernels running beside this one
+  if (pairs_max < 1) pairs_max = 1;
   const int pairs = (int)(n_items < pairs_max ? n_items : pairs_max);
   auto kern = umma_pipe2_kernel<Traits, ItemF, EpiF>;
   GPTQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
