@@ -411,15 +411,15 @@ def run_gpu(args, wl):
                                  "captures of 4096- and 16384-channel launches (2.4 x and 10.9 x), interpolated in C",
                     peak_source=f"bf16 sustained, {peaks['source']}")
     else:
-        ach = upd_flops / (tot["quantize_ms"] * 1e-3) / 1e12
-        pk = peaks["bf16_sustained"] / 2.0
-        roof = dict(kernel="quantize_layer (lazy update contraction)", bound="tensor", achieved=ach, peak=pk,
-                    unit="TFLOP/s", frac=ach / pk, traffic=None,
-                    peak_source=f"tf32 = bf16 sustained / 2 (nominal ratio), {peaks['source']}")
+        ach = 3 * upd_flops / (tot["quantize_ms"] * 1e-3) / 1e12
+        pk = peaks["bf16_sustained"]
+        roof = dict(kernel="quantize_layer (lazy update contraction, fp16 pairs: executed flops = 3 x useful)", bound="tensor",
+                    achieved=ach, peak=pk, unit="TFLOP/s", frac=ach / pk, traffic=None,
+                    peak_source=f"bf16 sustained (kind::f16 runs at the bf16 rate), {peaks['source']}")
 
     # every stage against the roofline that bounds it (CUDA events around the stage's launches; in the overlapped
     # schedules the stages of different layers run side by side, so these are in-context rates)
-    tf32_peak = peaks["bf16_sustained"] / 2.0
+    f16_peak = peaks["bf16_sustained"]           # kind::f16 instructions run at the bf16 rate
     fac_flops = sum(2.0 * L.C ** 3 / 3.0 for L in layers)
     hess_ach = hess_flops / (tot["hessian_ms"] * 1e-3) / 1e12
     fac_ach = fac_flops / (tot["hinv_ms"] * 1e-3) / 1e12
@@ -427,20 +427,20 @@ def run_gpu(args, wl):
     stage_rooflines = [
         dict(stage="hessian_accumulate", bound="tensor", dtype="bf16", achieved=hess_ach, peak=peaks["bf16_sustained"],
              unit="TFLOP/s", frac=hess_ach / peaks["bf16_sustained"], flops="algorithmic C (C + 1) m"),
-        dict(stage="prepare_hinv", bound="tensor", dtype="tf32 x3", achieved=fac_ach, executed=3 * fac_ach, peak=tf32_peak,
-             unit="TFLOP/s", frac=3 * fac_ach / tf32_peak, useful_frac=fac_ach / tf32_peak,
-             flops="useful 2 C^3 / 3; executed = 3 x (hi*hi + hi*lo + lo*hi); the serial 128 x 128 diagonal-block chain is inside this time"),
-        dict(stage="quantize_layer", bound="tensor", dtype="tf32 x3", achieved=upd_ach, executed=3 * upd_ach, peak=tf32_peak,
-             unit="TFLOP/s", frac=3 * upd_ach / tf32_peak, useful_frac=upd_ach / tf32_peak,
-             flops="useful R (C^2 - C B) per grid (lazy updates); the in-block kernels, packing and grids are inside this time"),
+        dict(stage="prepare_hinv", bound="tensor", dtype="fp16 pairs, 3 products per term", achieved=fac_ach, executed=3 * fac_ach,
+             peak=f16_peak, unit="TFLOP/s", frac=3 * fac_ach / f16_peak, useful_frac=fac_ach / f16_peak,
+             flops="useful 2 C^3 / 3; executed = 3 x (hi*hi + hi*lo + lo*hi); the serial 128 x 128 diagonal-block chain and the "
+                   "CUDA-core work inside an outer panel are inside this time"),
+        dict(stage="quantize_layer", bound="tensor", dtype="fp16 pairs, 3 products per term", achieved=upd_ach, executed=3 * upd_ach,
+             peak=f16_peak, unit="TFLOP/s", frac=3 * upd_ach / f16_peak, useful_frac=upd_ach / f16_peak,
+             flops="useful R (C^2 - C B) per grid (lazy updates); the column chains, packing and grids are inside this time"),
     ]
     for r in stage_rooflines:
-        r["peak_source"] = (f"bf16 sustained, {peaks['source']}" if r["dtype"] == "bf16"
-                            else f"tf32 = bf16 sustained / 2 (nominal ratio), {peaks['source']}")
+        r["peak_source"] = f"bf16 sustained, {peaks['source']}"
 
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
-                dtype="bf16 x bf16 -> f32 (Hessian); f32 factor; f64 working weights + f32 update sums (quantize)",
+                dtype="bf16 x bf16 -> f32 (Hessian); f32 factor (fp16-pair contractions, f64 diagonal blocks); f64 working weights + f32 update sums (quantize)",
                 data="synthetic",
                 config=dict(workload=wl.name, layers=[l.name for l in wl.layers],
                             grids=[dict(bits=g.bits, group_size=g.group_size, sym=g.sym) for g in wl.grids],
@@ -543,7 +543,7 @@ def run_gpu_strong(args, wl):
     n_grids = len(wl.grids)
     line = dict(metric=METRIC, value=wl.weights * n_grids / (ms_per_step * 1e-3), unit=UNIT, n_gpus=world, steps=args.steps,
                 warmup=args.warmup, ms_per_step=ms_per_step, higher_is_better=True, scaling="strong", vs_baseline=None,
-                dtype="bf16 x bf16 -> f32 (Hessian); f32 factor; f64 working weights + f32 update sums (quantize)",
+                dtype="bf16 x bf16 -> f32 (Hessian); f32 factor (fp16-pair contractions, f64 diagonal blocks); f64 working weights + f32 update sums (quantize)",
                 data="synthetic",
                 config=dict(workload=wl.name, layers=[l.name for l in wl.layers],
                             grids=[dict(bits=g.bits, group_size=g.group_size, sym=g.sym) for g in wl.grids],
@@ -624,23 +624,26 @@ def run_e2e(args, wl, state, device_value):
 
     host = []
     need = 256
+    grids = [(g.bits, g.group_size, g.sym) for g in wl.grids]
+    import ctypes
     for st in state:
         L = st["L"]
-        host.append(dict(L=L, X=st["X"].cpu().pin_memory(), W=st["W"].cpu().pin_memory(), out={}))
-        for g in wl.grids:
-            need = max(need, B.gptq_solve_layer_host_workspace_bytes(L.R, L.C, L.n_tokens, g.bits, g.group_size, wl.block))
+        host.append(dict(L=L, X=st["X"].cpu().pin_memory(), W=st["W"].cpu().pin_memory(), outs=None))
+        ng = len(grids)
+        need = max(need, B._lib.gptq_solve_layer_host_grids_workspace_bytes(
+            L.R, L.C, L.n_tokens, ng, (ctypes.c_int * ng)(*[g[0] for g in grids]), (ctypes.c_int * ng)(*[g[1] for g in grids]), wl.block))
     for st in state:                       # device copies are not needed any more: the call has its own staging
         st["X"] = st["H"] = st["U"] = st["ws"] = None
     torch.cuda.empty_cache()
     # Two calls in flight (two host threads, each with its own stream and device workspace): while one layer is being
-    # factored and quantized, the next layer's activations are already crossing PCIe.
-    n_workers = 2 if need * 2 < 100e9 and len(host) * len(wl.grids) > 1 else 1
+    # factored and quantized, the next layer's activations are already crossing PCIe.  Every call solves ALL grids of its
+    # layer, so a layer's activations cross once per step.
+    n_workers = 2 if need * 2 < 120e9 and len(host) > 1 else 1
     dev = torch.cuda.current_device()
     workers = [dict(ws=torch.empty(need, dtype=torch.uint8, device="cuda"), stream=torch.cuda.Stream()) for _ in range(n_workers)]
     torch.cuda.synchronize()
-    h2d = sum((h["X"].numel() * 2 + h["W"].numel() * 2) * len(wl.grids) for h in host)
-    tasks = sorted(((h, gi, g) for h in host for gi, g in enumerate(wl.grids)),
-                   key=lambda t: -(t[0]["L"].C ** 2) * (t[0]["L"].n_tokens + t[0]["L"].C))
+    h2d = sum(h["X"].numel() * 2 + h["W"].numel() * 2 for h in host)
+    tasks = sorted(host, key=lambda h: -(h["L"].C ** 2) * (h["L"].n_tokens + h["L"].C))
     import queue
 
     def step():
@@ -654,13 +657,12 @@ def run_e2e(args, wl, state, device_value):
             try:
                 while True:
                     try:
-                        h, gi, g = q.get_nowait()
+                        h = q.get_nowait()
                     except queue.Empty:
                         return
-                    o = B.gptq_solve_layer_host(h["W"], h["X"], g.bits, g.group_size, g.sym, wl.block, wl.damp,
-                                                out=h["out"].get(gi), dev_ws=wk["ws"], stream=wk["stream"])
-                    h["out"][gi] = o
-                    assert o["info"].tolist()[0] == 0, o["info"].tolist()
+                    h["outs"] = B.gptq_solve_layer_host_grids(h["W"], h["X"], grids, wl.block, wl.damp, outs=h["outs"],
+                                                              dev_ws=wk["ws"], stream=wk["stream"])
+                    assert h["outs"][0]["info"].tolist()[0] == 0, h["outs"][0]["info"].tolist()
             except Exception as e:          # surfaced after the join
                 errors.append(e)
 
@@ -671,7 +673,8 @@ def run_e2e(args, wl, state, device_value):
             t.join()
         if errors:
             raise errors[0]
-        return sum(t.numel() * t.element_size() for h in host for o in h["out"].values() for t in o.values())
+        return sum(o[k].numel() * o[k].element_size() for h in host for o in h["outs"] for k in ("qweight", "scales", "zeros")) + \
+            sum(8 * len(h["outs"]) + 8 for h in host)
 
     steps = max(1, min(args.steps, 5))      # each step moves every layer's activations across PCIe again (seconds)
     d2h = step()
@@ -681,8 +684,8 @@ def run_e2e(args, wl, state, device_value):
     dt = (time.perf_counter() - t0) / steps
     return dict(value=wl.weights * len(wl.grids) / dt, unit=UNIT, h2d_bytes_per_step=int(h2d),
                 d2h_bytes_per_step=int(d2h), ms_per_step=dt * 1e3, steps=steps,
-                api=f"gptq_solve_layer_host (pinned host buffers; X streamed in 512 MiB chunks on a copy stream); "
-                    f"{n_workers} call(s) in flight from {n_workers} host thread(s)")
+                api=f"gptq_solve_layer_host_grids (pinned host buffers; per layer X streamed once in 512 MiB chunks on a copy stream, "
+                    f"all {len(grids)} grid(s) solved from one Hessian and factor); {n_workers} call(s) in flight from {n_workers} host thread(s)")
 
 
 def run_inference(args, wl):
@@ -784,7 +787,7 @@ def run_block(args, wl):
     sec_per_block = ms * 1e-3 / blocks_here
     line = dict(metric=METRIC, value=wl.weights / (ms * 1e-3), unit=UNIT, n_gpus=1, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, data="synthetic",
-                dtype="bf16 x bf16 -> f32 (Hessian); f32 factor; f64 working weights + f32 update sums (quantize)",
+                dtype="bf16 x bf16 -> f32 (Hessian); f32 factor (fp16-pair contractions, f64 diagonal blocks); f64 working weights + f32 update sums (quantize)",
                 config=dict(workload=wl.name, mode="block pipeline: q, k, v share one Hessian and one factor",
                             grid=dict(bits=g.bits, group_size=g.group_size, sym=g.sym), block=wl.block, damp=wl.damp,
                             input_groups=[[m["m"].name for m in st["members"]] for st in solver.state],

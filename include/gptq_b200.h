@@ -247,6 +247,22 @@ gptq_status_t gptq_solve_layer_host(const void* W_fp16_host, const void* X_bf16_
                                     double* loss_host, int* info_host, void* dev_ws, size_t dev_ws_bytes,
                                     void* stream);
 
+/* The same for SEVERAL grids of one layer (e.g. the 4-bit and the 3-bit model of the paper's tables from one calibration
+ * pass): the activations cross to the device ONCE, one Hessian and one factor serve every grid (Algorithm 1's H^-1 does
+ * not depend on the grid), and stage 3 runs and is copied back grid after grid.
+ *   n_grids >= 1; bits / group_size / sym: host arrays of n_grids entries (as in gptq_quantize_layer);
+ *   qweight_host / scales_host / zeros_host: host arrays of n_grids host pointers, each shaped for its grid;
+ *   loss_host double[n_grids]; info_host int[2]: first non-OK device status of any stage or grid.
+ * Everything else as gptq_solve_layer_host. */
+size_t gptq_solve_layer_host_grids_workspace_bytes(int R, int C, int64_t n_tokens, int n_grids, const int* bits,
+                                                   const int* group_size, int block);
+gptq_status_t gptq_solve_layer_host_grids(const void* W_fp16_host, const void* X_bf16_host, int64_t n_tokens,
+                                          int R, int C, float damp, int n_grids, const int* bits,
+                                          const int* group_size, const int* sym, int block,
+                                          uint32_t* const* qweight_host, float* const* scales_host,
+                                          float* const* zeros_host, double* loss_host, int* info_host,
+                                          void* dev_ws, size_t dev_ws_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

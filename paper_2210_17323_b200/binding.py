@@ -64,6 +64,12 @@ def _load():
     lib.gptq_solve_layer_host.argtypes = [c.c_void_p, c.c_void_p, c.c_int64, c.c_int, c.c_int, c.c_float, c.c_int, c.c_int,
                                           c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
                                           c.c_void_p, c.c_size_t, c.c_void_p]
+    lib.gptq_solve_layer_host_grids_workspace_bytes.restype = c.c_size_t
+    lib.gptq_solve_layer_host_grids_workspace_bytes.argtypes = [c.c_int, c.c_int, c.c_int64, c.c_int, c.c_void_p, c.c_void_p, c.c_int]
+    lib.gptq_solve_layer_host_grids.restype = c.c_int
+    lib.gptq_solve_layer_host_grids.argtypes = [c.c_void_p, c.c_void_p, c.c_int64, c.c_int, c.c_int, c.c_float, c.c_int, c.c_void_p,
+                                                c.c_void_p, c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+                                                c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p]
     lib.gptq_rtn_layer.restype = c.c_int
     lib.gptq_rtn_layer.argtypes = [c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
     lib.gptq_dequantize.restype = c.c_int
@@ -257,6 +263,47 @@ def gptq_solve_layer_host(W_host, X_host, bits, group_size=0, sym=False, block=1
     if st != OK:
         raise GptqError(st, "gptq_solve_layer_host")
     return out
+
+
+def gptq_solve_layer_host_grids(W_host, X_host, grids, block=128, damp=0.01, outs=None, dev_ws=None, stream=None):
+    """Stages 1-3 for one layer and SEVERAL grids with HOST inputs and outputs: X crosses to the device once, one Hessian
+    and one factor serve every grid.  grids: sequence of (bits, group_size, sym) or (bits, group_size, sym, scale_fp16).
+    Returns a list of dicts like gptq_solve_layer_host's (pass `outs` to reuse pinned result buffers); the list's first
+    dict also carries 'info' (int32[2]).  Synchronises the stream."""
+    for t, dt, name in ((W_host, torch.float16, "W_host"), (X_host, torch.bfloat16, "X_host")):
+        if not (isinstance(t, torch.Tensor) and not t.is_cuda and t.is_contiguous() and t.dtype == dt):
+            raise TypeError(f"{name}: expected a contiguous CPU tensor of {dt}")
+    R, C = W_host.shape
+    n = X_host.shape[0]
+    ng = len(grids)
+    c = ctypes
+    bits = (c.c_int * ng)(*[g[0] for g in grids])
+    group = (c.c_int * ng)(*[g[1] for g in grids])
+    sym = (c.c_int * ng)(*[_grid_flags(g[2], g[3] if len(g) > 3 else False) for g in grids])
+    if outs is None:
+        outs = []
+        for g in grids:
+            G = C // g[1] if g[1] > 0 else 1
+            outs.append(dict(qweight=torch.empty((R, C * field_bits(g[0]) // 32), dtype=torch.int32).pin_memory(),
+                             scales=torch.empty((R, G), dtype=torch.float32).pin_memory(),
+                             zeros=torch.empty((R, G), dtype=torch.float32).pin_memory()))
+        outs[0]["loss_all"] = torch.zeros(ng, dtype=torch.float64).pin_memory()
+        outs[0]["info"] = torch.zeros(2, dtype=torch.int32).pin_memory()
+    qp = (c.c_void_p * ng)(*[o["qweight"].data_ptr() for o in outs])
+    sp = (c.c_void_p * ng)(*[o["scales"].data_ptr() for o in outs])
+    zp = (c.c_void_p * ng)(*[o["zeros"].data_ptr() for o in outs])
+    need = _lib.gptq_solve_layer_host_grids_workspace_bytes(R, C, n, ng, bits, group, block)
+    if need == 0:
+        raise GptqError(ERR_UNSUPPORTED, "gptq_solve_layer_host_grids_workspace_bytes")
+    dev_ws = _ws(need, torch.device("cuda", torch.cuda.current_device()), dev_ws)
+    st = _lib.gptq_solve_layer_host_grids(W_host.data_ptr(), X_host.data_ptr(), n, R, C, float(damp), ng, bits, group, sym, block,
+                                          qp, sp, zp, outs[0]["loss_all"].data_ptr(), outs[0]["info"].data_ptr(),
+                                          dev_ws.data_ptr(), dev_ws.numel(), _stream_ptr(stream))
+    if st != OK:
+        raise GptqError(st, "gptq_solve_layer_host_grids")
+    for i, o in enumerate(outs):
+        o["loss"] = outs[0]["loss_all"][i:i + 1]
+    return outs
 
 
 def gptq_rtn_layer(W, bits, group_size=0, sym=False, stream=None, scale_fp16=False):

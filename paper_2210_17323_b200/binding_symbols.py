@@ -5,5 +5,6 @@ EXPORTS = (
     "gptq_prepare_hinv_workspace_bytes", "gptq_prepare_hinv", "gptq_prepare_hinv_static",
     "gptq_quantize_workspace_bytes", "gptq_quantize_layer", "gptq_set_stage3_variant",
     "gptq_solve_layer_host_workspace_bytes", "gptq_solve_layer_host",
+    "gptq_solve_layer_host_grids_workspace_bytes", "gptq_solve_layer_host_grids",
     "gptq_rtn_layer", "gptq_dequantize", "gptq_matvec",
 )

@@ -19,7 +19,7 @@ struct HostWs {
 
 inline int field_bits_h(int bits) { return bits == GPTQ_BITS_TERNARY ? 2 : bits; }
 
-HostWs carve_host(void* ws, int R, int C, int64_t n_tokens, int bits, int group_size, int block) {
+HostWs carve_host(void* ws, int R, int C, int64_t n_tokens, int n_grids, const int* bits_v, const int* group_v, int block) {
   WsCarver w(ws);
   HostWs o;
   int64_t ct = kChunkBytes / ((int64_t)C * 2);
@@ -32,14 +32,22 @@ HostWs carve_host(void* ws, int R, int C, int64_t n_tokens, int bits, int group_
   o.W = w.take<__half>((size_t)R * C);
   o.X[0] = w.take<__nv_bfloat16>((size_t)ct * C);
   o.X[1] = w.take<__nv_bfloat16>((size_t)ct * C);
-  const int G = group_size > 0 ? C / group_size : 1;
-  o.qweight = w.take<uint32_t>((size_t)R * (C * field_bits_h(bits) / 32));
+  // one set of output buffers, sized for the widest grid, reused grid after grid
+  int G = 1, f = 2;
+  size_t s3 = 0;
+  for (int i = 0; i < n_grids; ++i) {
+    const int Gi = group_v[i] > 0 ? C / group_v[i] : 1;
+    if (Gi > G) G = Gi;
+    if (field_bits_h(bits_v[i]) > f) f = field_bits_h(bits_v[i]);
+    const size_t q = gptq_quantize_workspace_bytes(R, C, bits_v[i], group_v[i], block);
+    if (q > s3) s3 = q;
+  }
+  o.qweight = w.take<uint32_t>((size_t)R * (C * f / 32));
   o.scales = w.take<float>((size_t)R * G);
   o.zeros = w.take<float>((size_t)R * G);
   o.loss = w.take<double>(1);
   o.info = w.take<int>(8);
-  size_t s1 = gptq_hessian_workspace_bytes(C, ct), s2 = gptq_prepare_hinv_workspace_bytes(C),
-         s3 = gptq_quantize_workspace_bytes(R, C, bits, group_size, block);
+  size_t s1 = gptq_hessian_workspace_bytes(C, ct), s2 = gptq_prepare_hinv_workspace_bytes(C);
   o.stage_ws_bytes = s1 > s2 ? (s1 > s3 ? s1 : s3) : (s2 > s3 ? s2 : s3);
   if (o.stage_ws_bytes < kAlign) o.stage_ws_bytes = kAlign;
   o.stage_ws = w.take<unsigned char>(o.stage_ws_bytes);
@@ -69,17 +77,25 @@ struct StreamGuard {
 extern "C" size_t gptq_solve_layer_host_workspace_bytes(int R, int C, int64_t n_tokens, int bits, int group_size,
                                                         int block) {
   using namespace gptq;
-  if (R <= 0 || C <= 0 || C % 32 != 0 || n_tokens < 0 || block <= 0) return 0;
-  if (gptq_quantize_workspace_bytes(R, C, bits, group_size, block) == 0) return 0;
-  return carve_host(nullptr, R, C, n_tokens, bits, group_size, block).bytes;
+  return gptq_solve_layer_host_grids_workspace_bytes(R, C, n_tokens, 1, &bits, &group_size, block);
+}
+
+extern "C" size_t gptq_solve_layer_host_grids_workspace_bytes(int R, int C, int64_t n_tokens, int n_grids, const int* bits,
+                                                              const int* group_size, int block) {
+  using namespace gptq;
+  if (R <= 0 || C <= 0 || C % 32 != 0 || n_tokens < 0 || block <= 0 || n_grids <= 0 || !bits || !group_size) return 0;
+  for (int i = 0; i < n_grids; ++i)
+    if (gptq_quantize_workspace_bytes(R, C, bits[i], group_size[i], block) == 0) return 0;
+  return carve_host(nullptr, R, C, n_tokens, n_grids, bits, group_size, block).bytes;
 }
 
 namespace gptq {
 namespace {
 gptq_status_t solve_layer_host_enqueue(const HostWs& w, StreamGuard& g, cudaStream_t s, const void* W_fp16_host,
-                                       const void* X_bf16_host, int64_t n_tokens, int R, int C, float damp, int bits,
-                                       int group_size, int sym, int block, uint32_t* qweight_host, float* scales_host,
-                                       float* zeros_host, double* loss_host, int* info8_host);
+                                       const void* X_bf16_host, int64_t n_tokens, int R, int C, float damp, int n_grids,
+                                       const int* bits, const int* group_size, const int* sym, int block,
+                                       uint32_t* const* qweight_host, float* const* scales_host, float* const* zeros_host,
+                                       double* loss_host, int* info8_host);
 }  // namespace
 }  // namespace gptq
 
@@ -88,14 +104,26 @@ extern "C" gptq_status_t gptq_solve_layer_host(const void* W_fp16_host, const vo
                                                uint32_t* qweight_host, float* scales_host, float* zeros_host,
                                                double* loss_host, int* info_host, void* dev_ws, size_t dev_ws_bytes,
                                                void* stream) {
+  return gptq_solve_layer_host_grids(W_fp16_host, X_bf16_host, n_tokens, R, C, damp, 1, &bits, &group_size, &sym, block,
+                                     &qweight_host, &scales_host, &zeros_host, loss_host, info_host, dev_ws, dev_ws_bytes, stream);
+}
+
+extern "C" gptq_status_t gptq_solve_layer_host_grids(const void* W_fp16_host, const void* X_bf16_host, int64_t n_tokens,
+                                                     int R, int C, float damp, int n_grids, const int* bits,
+                                                     const int* group_size, const int* sym, int block,
+                                                     uint32_t* const* qweight_host, float* const* scales_host,
+                                                     float* const* zeros_host, double* loss_host, int* info_host,
+                                                     void* dev_ws, size_t dev_ws_bytes, void* stream) {
   using namespace gptq;
   if (!W_fp16_host || !X_bf16_host || !qweight_host || !scales_host || !zeros_host || !loss_host || !info_host ||
-      R <= 0 || C <= 0 || C % 32 != 0 || n_tokens <= 0)
+      !bits || !group_size || !sym || n_grids <= 0 || R <= 0 || C <= 0 || C % 32 != 0 || n_tokens <= 0)
     return GPTQ_ERR_INVALID_ARG;
-  const size_t need = gptq_solve_layer_host_workspace_bytes(R, C, n_tokens, bits, group_size, block);
+  for (int i = 0; i < n_grids; ++i)
+    if (!qweight_host[i] || !scales_host[i] || !zeros_host[i]) return GPTQ_ERR_INVALID_ARG;
+  const size_t need = gptq_solve_layer_host_grids_workspace_bytes(R, C, n_tokens, n_grids, bits, group_size, block);
   if (need == 0) return GPTQ_ERR_UNSUPPORTED;
   if (!dev_ws || !aligned_to(dev_ws, kAlign) || dev_ws_bytes < need) return GPTQ_ERR_WORKSPACE;
-  HostWs w = carve_host(dev_ws, R, C, n_tokens, bits, group_size, block);
+  HostWs w = carve_host(dev_ws, R, C, n_tokens, n_grids, bits, group_size, block);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   StreamGuard g;
   GPTQ_CUDA_TRY(cudaStreamCreateWithFlags(&g.s, cudaStreamNonBlocking));
@@ -106,7 +134,7 @@ extern "C" gptq_status_t gptq_solve_layer_host(const void* W_fp16_host, const vo
   GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&g.w_done, cudaEventDisableTiming));
 
   int info[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  gptq_status_t st = solve_layer_host_enqueue(w, g, s, W_fp16_host, X_bf16_host, n_tokens, R, C, damp, bits, group_size,
+  gptq_status_t st = solve_layer_host_enqueue(w, g, s, W_fp16_host, X_bf16_host, n_tokens, R, C, damp, n_grids, bits, group_size,
                                               sym, block, qweight_host, scales_host, zeros_host, loss_host, info);
   // Whatever happened, nothing of this call may still be in flight when it returns: the caller may free the host
   // buffers the copy stream reads, and the guard destroys that stream and its events.
@@ -122,9 +150,10 @@ extern "C" gptq_status_t gptq_solve_layer_host(const void* W_fp16_host, const vo
 namespace gptq {
 namespace {
 gptq_status_t solve_layer_host_enqueue(const HostWs& w, StreamGuard& g, cudaStream_t s, const void* W_fp16_host,
-                                       const void* X_bf16_host, int64_t n_tokens, int R, int C, float damp, int bits,
-                                       int group_size, int sym, int block, uint32_t* qweight_host, float* scales_host,
-                                       float* zeros_host, double* loss_host, int* info8_host) {
+                                       const void* X_bf16_host, int64_t n_tokens, int R, int C, float damp, int n_grids,
+                                       const int* bits, const int* group_size, const int* sym, int block,
+                                       uint32_t* const* qweight_host, float* const* scales_host, float* const* zeros_host,
+                                       double* loss_host, int* info8_host) {
   GPTQ_CUDA_TRY(cudaMemsetAsync(w.H, 0, (size_t)C * C * sizeof(float), s));
   GPTQ_CUDA_TRY(cudaMemsetAsync(w.info, 0, 8 * sizeof(int), s));
   const __nv_bfloat16* Xh = static_cast<const __nv_bfloat16*>(X_bf16_host);
@@ -151,14 +180,20 @@ gptq_status_t solve_layer_host_enqueue(const HostWs& w, StreamGuard& g, cudaStre
   GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, g.w_done, 0));
   st = gptq_prepare_hinv(w.H, damp, C, w.U, w.stage_ws, w.stage_ws_bytes, w.info + 2, s);
   if (st != GPTQ_OK) return st;
-  st = gptq_quantize_layer(w.W, w.U, R, C, bits, group_size, sym, block, w.qweight, w.scales, w.zeros, w.loss,
-                           w.stage_ws, w.stage_ws_bytes, w.info + 4, s);
-  if (st != GPTQ_OK) return st;
-  const int G = group_size > 0 ? C / group_size : 1;
-  GPTQ_CUDA_TRY(cudaMemcpyAsync(qweight_host, w.qweight, (size_t)R * (C * field_bits_h(bits) / 32) * 4, cudaMemcpyDeviceToHost, s));
-  GPTQ_CUDA_TRY(cudaMemcpyAsync(scales_host, w.scales, (size_t)R * G * 4, cudaMemcpyDeviceToHost, s));
-  GPTQ_CUDA_TRY(cudaMemcpyAsync(zeros_host, w.zeros, (size_t)R * G * 4, cudaMemcpyDeviceToHost, s));
-  GPTQ_CUDA_TRY(cudaMemcpyAsync(loss_host, w.loss, sizeof(double), cudaMemcpyDeviceToHost, s));
+  // one Hessian and one factor serve every grid: quantize and copy back grid after grid (the device output buffers are
+  // reused, the stream keeps a grid's copies ahead of the next grid's kernels)
+  for (int gi = 0; gi < n_grids; ++gi) {
+    st = gptq_quantize_layer(w.W, w.U, R, C, bits[gi], group_size[gi], sym[gi], block, w.qweight, w.scales, w.zeros, w.loss,
+                             w.stage_ws, w.stage_ws_bytes, w.info + 6, s);
+    if (st != GPTQ_OK) return st;
+    fold_info_kernel<<<1, 1, 0, s>>>(w.info + 4, w.info + 6);
+    GPTQ_LAUNCH_CHECK();
+    const int G = group_size[gi] > 0 ? C / group_size[gi] : 1;
+    GPTQ_CUDA_TRY(cudaMemcpyAsync(qweight_host[gi], w.qweight, (size_t)R * (C * field_bits_h(bits[gi]) / 32) * 4, cudaMemcpyDeviceToHost, s));
+    GPTQ_CUDA_TRY(cudaMemcpyAsync(scales_host[gi], w.scales, (size_t)R * G * 4, cudaMemcpyDeviceToHost, s));
+    GPTQ_CUDA_TRY(cudaMemcpyAsync(zeros_host[gi], w.zeros, (size_t)R * G * 4, cudaMemcpyDeviceToHost, s));
+    GPTQ_CUDA_TRY(cudaMemcpyAsync(loss_host + gi, w.loss, sizeof(double), cudaMemcpyDeviceToHost, s));
+  }
   GPTQ_CUDA_TRY(cudaMemcpyAsync(info8_host, w.info, 8 * sizeof(int), cudaMemcpyDeviceToHost, s));
   return GPTQ_OK;
 }

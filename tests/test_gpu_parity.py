@@ -526,3 +526,27 @@ def test_bounded_waits_report_timeout_and_the_gpu_stays_usable(B, D):
     assert info.tolist() == [0, 0]
     Href = O.hessian_accumulate(np.zeros((L.C, L.C)), L.x_bits())
     assert rel_fro(H.cpu().numpy(), Href) <= TOL_H_FRO
+
+
+def test_solve_layer_from_host_buffers_several_grids(B):
+    """One host-buffer call for several grids of a layer (activations cross once, one Hessian and factor): every grid's
+    result matches the oracle, and equals the single-grid call's for the grid they share."""
+    L = _layer(96, 1280, 5000, cfg=5, kind="v")
+    bits_host, W16 = L.x_bits(), L.w()
+    Xh = torch.from_numpy(bits_host.view(np.int16)).view(torch.bfloat16).pin_memory()
+    Wh = torch.from_numpy(W16).pin_memory()
+    grids = [(4, 0, False), (3, 128, False), (B.BITS_TERNARY, 32, False)]
+    outs = None
+    for _ in range(2):                      # twice: the second call reuses the result buffers
+        outs = B.gptq_solve_layer_host_grids(Wh, Xh, grids, 128, 0.01, outs=outs)
+    assert outs[0]["info"].tolist() == [0, 0]
+    H = O.hessian_accumulate(np.zeros((L.C, L.C)), bits_host)
+    U = O.cholesky_inverse_upper(O.dampen(H, 0.01)[0])
+    for (bits, group, sym), o in zip(grids, outs):
+        ref = O.quantize_layer(W16, U, bits, group, sym, 128)
+        gpu = dict(qweight=o["qweight"].numpy(), scales=o["scales"].numpy(), zeros=o["zeros"].numpy(), loss=o["loss"].item())
+        check_quantize_outputs(gpu, ref, W16, bits, L.C, H)
+    single = B.gptq_solve_layer_host(Wh, Xh, 3, 128, False, 128, 0.01)
+    a = O.unpack_codes(single["qweight"].numpy().view(np.uint32), 3, L.C)
+    b = O.unpack_codes(outs[1]["qweight"].numpy().view(np.uint32), 3, L.C)
+    assert (a == b).mean() >= 0.999
