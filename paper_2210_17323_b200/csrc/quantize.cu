@@ -109,6 +109,18 @@ __global__ void wblk_from_w16_kernel(const __half* __restrict__ W, int R, int C,
   const int64_t o = stripe_major ? ((int64_t)(r >> 7) * ldw + c) * 128 + (r & 127) : (int64_t)r * ldw + c;
   Wblk[o] = (double)__half2float(W[(int64_t)r * C + i2 + c]);
 }
+// The same for the stripe-major layout through a 32 x 32 shared-memory tile, so that both the reads (along a row of W)
+// and the writes (along a column of a stripe) are coalesced.  grid (nb / 32, ceil(R / 32)), block (32, 32).
+__global__ void wblk_stripe_major_kernel(const __half* __restrict__ W, int R, int C, int i2,
+                                         double* __restrict__ Wblk, int64_t ldw) {
+  __shared__ float t[32][33];
+  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+  const int r = r0 + threadIdx.y;
+  t[threadIdx.y][threadIdx.x] = r < R ? __half2float(W[(int64_t)r * C + i2 + c0 + threadIdx.x]) : 0.f;
+  __syncthreads();
+  const int rr = r0 + threadIdx.x, cc = c0 + threadIdx.y;      // row fastest: 32 consecutive doubles of one stripe column
+  if (rr < R) Wblk[((int64_t)(rr >> 7) * ldw + cc) * 128 + (rr & 127)] = (double)t[threadIdx.x][threadIdx.y];
+}
 
 // ---- the in-block loop (Algorithm 1, inner FOR) -------------------------------------------------
 struct InblockArgs {
@@ -526,8 +538,13 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
     }
     // working weights of the outer block: original weights minus all updates from columns < i2
     {
-      int64_t total = (int64_t)R * nb2;
-      wblk_from_w16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(W, R, C, i2, nb2, Wblk, ldw, stripe ? 1 : 0);
+      if (stripe) {
+        dim3 grid(nb2 / 32, ceil_div(R, 32)), blk(32, 32);
+        wblk_stripe_major_kernel<<<grid, blk, 0, s>>>(W, R, C, i2, Wblk, ldw);
+      } else {
+        int64_t total = (int64_t)R * nb2;
+        wblk_from_w16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(W, R, C, i2, nb2, Wblk, ldw, 0);
+      }
       GPTQ_LAUNCH_CHECK();
     }
     if (i2 > 0) {
