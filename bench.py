@@ -323,6 +323,18 @@ def run_gpu(args, wl):
             last = h_done[list(layer_order)[-1]]
             for li in layer_order:
                 chain(li, last)
+        elif args.schedule == "small-first":
+            # cheap layers first: their Hessians back to back, their chains side by side; the most expensive layer's Hessian
+            # starts when those chains have drained (a persistent Hessian launch would starve them), and its own chain
+            # then has the GPU to itself
+            asc = list(layer_order)[::-1]
+            for li in asc[:-1]:
+                hessian(li)
+                chain(li, h_done[li])
+            for e in done:
+                main.wait_event(e)
+            hessian(asc[-1])
+            chain(asc[-1], h_done[asc[-1]])
         else:
             for li in layer_order:
                 hessian(li)
@@ -451,6 +463,9 @@ def run_gpu(args, wl):
                                                    "stream as soon as its Hessian is done; stage_ms are in-context times that overlap",
                                       "hessians-first": "hessians-first: all Hessians on one stream, then every layer's stages 2-3 side by "
                                                         "side on its own stream; stage 2-3 times overlap one another",
+                                      "small-first": "small-first: the cheaper layers' Hessians back to back with their stages 2-3 side by side on "
+                                                     "their own streams; the most expensive layer's Hessian starts when those have drained and "
+                                                     "its stages 2-3 then run alone; stage 2-3 times of the cheaper layers overlap one another",
                                       "sequential": "sequential: one stream, layer after layer"}[args.schedule],
                             parallelism=f"layer-set replica per GPU x{world}"),
                 sec_per_layer=ms_per_step * 1e-3 / len(layers),
@@ -601,7 +616,7 @@ def run_block_sweep(args, wl):
                 same = float((out["qweight"] == base).float().mean().item())
                 useful = L.R * (L.C * L.C - L.C * blk) / (ms * 1e-3) / 1e12
                 rows.append(dict(bits=g.bits, group_size=g.group_size, block=blk,
-                                 form="row-stripe" if (variant == 1 and blk <= 128) else "per-inner-block", ms=ms,
+                                 form="row-stripe" if variant == 1 else "per-inner-block", ms=ms,
                                  useful_tflops=useful, executed_tflops=3 * useful,
                                  frac_of_bf16_sustained=3 * useful / peaks["bf16_sustained"],
                                  packed_words_identical_to_first=same, loss=out["loss"].item()))
@@ -811,7 +826,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-graphs", action="store_true", help="issue every kernel launch from the host instead of replaying CUDA graphs")
-    ap.add_argument("--schedule", default="pipelined", choices=["pipelined", "hessians-first", "sequential"],
+    ap.add_argument("--schedule", default="pipelined", choices=["pipelined", "hessians-first", "small-first", "sequential"],
                     help="pipelined: Hessians back to back on one stream, each layer's stages 2-3 on its own stream as soon as "
                          "its Hessian is done; hessians-first: all Hessians, then all layers' stages 2-3 side by side; "
                          "sequential: one stream, layer after layer")

@@ -186,8 +186,8 @@ gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U, int R, int
  * contraction per outer block either way):
  *   1 (default)  row-stripe form: rows are independent (Section 2), so one CTA owns a stripe of rows and runs all
  *                inner blocks of the outer block back to back in ONE launch -- the inner loop with one thread per
- *                row, the block's lazy update for its rows with warp-level tensor-core instructions.  block <= 128;
- *                a larger block falls back to form 0.
+ *                row, the pushes of its errors with tcgen05 tensor-core instructions on the stripe's 128 rows.  A block
+ *                of 256 columns runs there as two 128-column inner blocks (the same updates, regrouped).
  *   0            per inner block one in-block kernel and one small tcgen05 contraction (two launches per block).
  * Process-wide, takes effect for calls made afterwards; returns the previous value (any other argument only
  * queries).  Meant for side-by-side benchmarks; results of the two forms agree up to fp32-level rounding of the

@@ -528,7 +528,11 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   GPTQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)inblock_smem(256)));
 
   // form of the loops inside an outer block (see gptq_set_stage3_variant)
-  const bool stripe = g_stage3_variant.load(std::memory_order_relaxed) == 1 && block <= kStripeMaxB && B2 <= kStripeMaxNb2;
+  // A block wider than the row-stripe kernel's 128 columns (256) is run there as 128-column inner blocks: the same updates
+  // in the same column order, regrouped (Section 3, Step 2) -- groups still nest with 128 whenever they nest with 256.
+  const bool stripe = g_stage3_variant.load(std::memory_order_relaxed) == 1 && B2 <= kStripeMaxNb2 &&
+                      (block <= kStripeMaxB || block % kStripeMaxB == 0);
+  const int stripe_block = block <= kStripeMaxB ? block : kStripeMaxB;
   for (int i2 = 0; i2 < C; i2 += B2) {
     const int nb2 = (C - i2 < B2) ? C - i2 : B2;
     {  // transposed tf32 hi/lo pair of U[0 : i2 + nb2, i2 : i2 + nb2] for the contractions of this outer block
@@ -555,7 +559,7 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
     }
     if (stripe) {
       // row-stripe form: every inner block of this outer block in one launch
-      StripeArgs a{Wblk, ldw, nb2, U, C, i2, block, R, gs, g, scales, zeros, G, Ehi, Elo, Phi, Plo, (int64_t)C,
+      StripeArgs a{Wblk, ldw, nb2, U, C, i2, stripe_block, R, gs, g, scales, zeros, G, Ehi, Elo, Phi, Plo, (int64_t)C,
                    sK, sE, sEinv, sCinv, codes, loss, dev_info};
       gptq_status_t st = launch_stripe(a, Phi, Plo, s);
       if (st != GPTQ_OK) return st;
