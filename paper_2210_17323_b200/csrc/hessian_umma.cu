@@ -82,9 +82,10 @@ struct HessPairTraits {
   static constexpr int B_BYTES = 2 * BOX_BYTES;           // 16 KB: this CTA's 128 of the 256 columns
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 32 KB per CTA
   static constexpr int CHUNK_KB = 8;
-  struct Maps { CUtensorMap x; };
+  static constexpr int EPI_SMEM = 8 * 4096;               // one 32 x 32 fp32 staging tile per epilogue warp
+  struct Maps { CUtensorMap x; CUtensorMap h; };          // X (bf16, 64 x 64 boxes), H (fp32, 32 x 32 boxes)
 
-  static __device__ __forceinline__ void prefetch(const Maps& m) { umma::prefetch_tmap(&m.x); }
+  static __device__ __forceinline__ void prefetch(const Maps& m) { umma::prefetch_tmap(&m.x); umma::prefetch_tmap(&m.h); }
   static __device__ __forceinline__ void load(uint8_t* s, const Maps& m, int m0, int n0, int kb, uint64_t* bar) {
     const int y = kb * BK;
 #pragma unroll
@@ -104,25 +105,30 @@ struct HessPairTraits {
   }
 };
 
-// 256 x 256 tiles on or above the diagonal, in bands of `band` tile rows, column by column inside a band.  ONLY valid
-// tiles are enumerated: every work item then has the same length, the CTA pairs stay in step, and the ~74 tiles in
-// flight at any time form a compact window of the tile grid whose operand strips are fetched from DRAM once and
-// shared through L2.  (With below-diagonal tiles enumerated and skipped, the pairs drifted apart by whole windows
-// and X was read 30 times at 16384 channels.)  Token ranges (super-chunks) are the outer loop: consecutive windows
-// of a band then reuse the band's row strips of that token range from L2.
+// 256 x 256 tiles on or above the diagonal.  ONLY valid tiles are enumerated.  Order of the work items, which the
+// dynamic item feed hands out in sequence so that the ~74 pairs always work on neighbouring items:
+//   bands of `band` tile rows; inside a band the valid tiles column by column, cut into windows of `wt` tiles;
+//   inside a window every token range (super-chunk) in turn; inside a token range the window's tiles.
+// At any time the pairs therefore share the ~band + wt / band operand strips of one window over one or two token
+// ranges (a few tens of MB, fetched from DRAM once and then read from L2), and the window's tiles of H stay in L2
+// from one token range to the next, so that H goes to DRAM once per window and not once per token range.
 struct HessPairItems {
-  int tiles, n_enum, sc_kb, total_kb, band;
+  int tiles, n_enum, sc_kb, total_kb, band, wt, nsc;
   // valid tiles of band s: rows r0 .. r0+rows-1, columns r0 .. tiles-1, row <= column
   static __host__ __device__ __forceinline__ int band_count(int tiles, int band, int s) {
     const int r0 = s * band, rows = tiles - r0 < band ? tiles - r0 : band;
     return rows * (rows + 1) / 2 + rows * (tiles - r0 - rows);
   }
   __device__ __forceinline__ bool operator()(int idx, int& m0, int& n0, int& kb0, int& kb1) const {
-    const int sc = idx / n_enum;
-    int t = idx % n_enum, mi = 0, nj = 0;
+    int mi = 0, nj = 0, sc = 0;
     for (int s = 0; s * band < tiles; ++s) {
       const int cnt = band_count(tiles, band, s);
-      if (t < cnt) {
+      if (idx < cnt * nsc) {
+        const int per_window = wt * nsc;
+        const int j = idx / per_window, local = idx - j * per_window;
+        const int n_w = cnt - j * wt < wt ? cnt - j * wt : wt;          // tiles in this window (the last one may be short)
+        sc = local / n_w;
+        const int t = j * wt + local - sc * n_w;
         const int r0 = s * band, rows = tiles - r0 < band ? tiles - r0 : band, tri = rows * (rows + 1) / 2;
         if (t < tri) {                     // diagonal part: column c (0-based inside the band) has c + 1 valid rows
           int c = 0;
@@ -134,7 +140,7 @@ struct HessPairItems {
         }
         break;
       }
-      t -= cnt;
+      idx -= cnt * nsc;
     }
     m0 = mi * 256; n0 = nj * 256;
     kb0 = sc * sc_kb;
@@ -154,6 +160,32 @@ struct EpiAddTwiceUpper {
       const int col = col0 + 4 * g;
       if (col < C && col + 3 >= row)
         umma::red_add_v4(hrow + col, 2.f * v[4 * g], 2.f * v[4 * g + 1], 2.f * v[4 * g + 2], 2.f * v[4 * g + 3]);
+    }
+  }
+};
+
+// H[row0 .. +32)[col0 .. +32) += 2 * sums, one TMA reduction per warp and block: the lanes write their rows into a
+// 128-byte-swizzled staging tile and one lane sends it off.  Blocks wholly below the diagonal are left out; the parts
+// of diagonal blocks below it receive sums that the mirror pass overwrites.  The columns and rows beyond C are dropped
+// by the TMA unit.
+struct EpiAddTwiceTile {
+  static constexpr bool kTile = true;
+  int C;
+  __device__ __forceinline__ void tile(const HessPairTraits::Maps& maps, uint8_t* buf, int row0, int col0,
+                                       const float (&v)[32], int lane) const {
+    if (row0 >= C || col0 >= C || col0 + 31 < row0) return;          // (warp-uniform)
+    if (lane == 0) umma::bulk_group_wait_read_all();                  // the previous reduction has read the staging tile
+    __syncwarp();
+    const uint32_t base = umma::smem_u32(buf) + (uint32_t)lane * 128u;
+#pragma unroll
+    for (int g = 0; g < 8; ++g)
+      asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(base + (uint32_t)((g ^ (lane & 7)) << 4)),
+                   "f"(2.f * v[4 * g]), "f"(2.f * v[4 * g + 1]), "f"(2.f * v[4 * g + 2]), "f"(2.f * v[4 * g + 3]) : "memory");
+    umma::fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) {
+      umma::tma_reduce_add_2d(&maps.h, col0, row0, buf);
+      umma::bulk_group_commit();
     }
   }
 };
@@ -219,21 +251,24 @@ gptq_status_t hessian_umma(float* H, const __nv_bfloat16* X, int64_t n_tokens, i
   if (st != GPTQ_OK) return st;
   const int sms = device_sm_count();
   const int total_kb = ceil_div(n_tokens, BK);
-  // tokens per super-chunk: 16384 (256 blocks) while a super-chunk's slice of X still shares L2 with the
-  // reductions into H, 8192 beyond that; shorter when there are too few tiles to fill the GPU
-  int ck = C <= 8192 ? 256 : 128;
+  int ck = C <= 8192 ? 256 : 128;       // one-CTA path: tokens per work item / 64
   if (C >= 512) {
-    // two-CTA tiles of 256 x 256
-    HessPairTraits::Maps maps{tmap};
+    // two-CTA tiles of 256 x 256, dynamic item feed
+    HessPairTraits::Maps maps;
+    maps.x = tmap;
+    st = make_tmap_2d(&maps.h, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, H, (uint64_t)C, (uint64_t)C, (uint64_t)C * 4, 32, 32);
+    if (st != GPTQ_OK) return st;
     HessPairItems it;
     it.tiles = ceil_div(C, 256);
-    it.band = 16;                          // measured: 16-24 tile rows per band beat 4, 8, 32 and more at 12288-49152 channels
+    it.band = 8;
+    it.wt = 144;
     it.n_enum = it.tiles * (it.tiles + 1) / 2;
-    const int n_valid = it.n_enum;
-    while (ck > 8 && (int64_t)n_valid * ceil_div(total_kb, ck) < sms) ck >>= 1;
-    it.total_kb = total_kb; it.sc_kb = ck;
-    st = pipe2::launch_pipe2<HessPairTraits>(maps, (int64_t)it.n_enum * ceil_div(total_kb, ck), it, EpiAddTwiceUpper{H, C},
-                                             dev_info, stream);
+    ck = 128;                             // 8192 tokens per item
+    while (ck > 8 && (int64_t)it.n_enum * ceil_div(total_kb, ck) < sms) ck >>= 1;
+    while ((int64_t)it.n_enum * ceil_div(total_kb, ck) > 0x3FFFFFFF) ck <<= 1;     // (the grid has one cluster per item)
+    it.total_kb = total_kb; it.sc_kb = ck; it.nsc = ceil_div(total_kb, ck);
+    const int64_t n_items = (int64_t)it.n_enum * it.nsc;
+    st = pipe2::launch_pipe2_dynamic<HessPairTraits>(maps, n_items, it, EpiAddTwiceTile{C}, dev_info, stream);
   } else {
     HessTraits::Maps maps{tmap};
     HessItems it;
@@ -258,3 +293,4 @@ gptq_status_t hessian_umma(float* H, const __nv_bfloat16* X, int64_t n_tokens, i
 cudaError_t hessian_set_wait_test_knobs(unsigned long long limit_ns, int skip_item) { return set_wait_test_knobs(limit_ns, skip_item); }
 
 }  // namespace gptq
+

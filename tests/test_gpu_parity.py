@@ -517,7 +517,7 @@ def test_bounded_waits_report_timeout_and_the_gpu_stays_usable(B, D):
         B.gptq_hessian_accumulate(H, X, dev_info=info)
         torch.cuda.synchronize()
         st, where = info.tolist()
-        assert st == B.ERR_TIMEOUT and where in (21, 22, 23, 24), (st, where)
+        assert st == B.ERR_TIMEOUT and 21 <= where <= 27, (st, where)   # whichever role's wait ran out first
     finally:
         B.gptq_debug_wait_test(0, -1)
     H.zero_()
