@@ -4,7 +4,7 @@
 //   acc[m][n] = sum_k A[m][k] * B[n][k]  ~  Ahi*Bhi + Ahi*Blo + Alo*Bhi     (hi = fp16(x), lo = fp16(x - hi))
 //
 // An fp16 number carries 11 significant bits like a tf32 number, so hi + lo holds 22 bits and the
-// dropped lo*lo term is of relative size 2^-22 -- the same accuracy as the 3xTF32 form (gemm_umma.cuh)
+// dropped lo*lo term is of relative size 2^-22 -- the accuracy of three tf32 products of tf32 pairs
 // -- while kind::f16 instructions run at twice the tf32 rate and the operands take half the bytes.
 // Products of two fp16 values are exact in the fp32 accumulator.  The price is fp16's narrow exponent
 // range: callers must scale their operands by powers of two (exact) so that the entries that matter
@@ -12,7 +12,7 @@
 // largest one lose relative precision gracefully (absolute error <= 2^-25 in scaled units); values
 // beyond the range must be saturated by whoever writes the operands.
 //
-// Operand layouts as in gemm_umma.cuh: both row-major with K contiguous (A is [M][K], B is [N][K]).
+// Operand layouts: both row-major with K contiguous (A is [M][K], B is [N][K]).
 // TMA boxes of 64 fp16 x 128 rows with 128-byte swizzle are the canonical K-major tiles.  Per CTA and
 // 64-wide K block: its 128 rows of A (hi, lo) and its 128 of the tile's 256 rows of B (hi, lo) = 64 KB;
 // twelve MMAs (four 16-wide K steps x three products) per K block go into one TMEM accumulator, which is
@@ -20,6 +20,8 @@
 // why; draining after every block costs 7 % of a whole 175B-shaped step for an error that is already at the
 // 1e-6 level of the factor either way: probe residual of U at 49152 columns 1.1e-6 against 1.8e-6).
 #pragma once
+#include <cstring>
+
 #include "umma_pipe2.cuh"
 
 namespace gptq {
@@ -33,7 +35,8 @@ struct Traits {
   static constexpr int OP_BYTES = 128 * BK * 2;            // 16 KB: 128 rows x 64 fp16 (one of hi / lo, A or B half)
   static constexpr int STAGE_BYTES = 4 * OP_BYTES;         // 64 KB per CTA
   static constexpr int CHUNK_KB = 2;                       // 24 MMAs per TMEM accumulation
-  struct Maps { CUtensorMap a_hi, a_lo, b_hi, b_lo; };
+  static constexpr int EPI_SMEM = 8 * 4096;                // staging for epilogues that leave through TMA reductions
+  struct Maps { CUtensorMap a_hi, a_lo, b_hi, b_lo, out; };  // out: the output, for those epilogues only
 
   static __device__ __forceinline__ void prefetch(const Maps& m) {
     umma::prefetch_tmap(&m.a_hi); umma::prefetch_tmap(&m.a_lo); umma::prefetch_tmap(&m.b_hi); umma::prefetch_tmap(&m.b_lo);
@@ -93,10 +96,13 @@ struct Operand {
 // acc = A * B^T over K = A.cols = B.cols; epi must accumulate (it is called once per super-chunk).
 template <bool kTriLeft, bool kUpperOut, class EpiF>
 gptq_status_t launch(const Operand& A, const Operand& B, int M, int N, EpiF epi, int* dev_info, cudaStream_t stream,
-                     int reserve_sms = 0) {
+                     int reserve_sms = 0, const CUtensorMap* out_map = nullptr) {
   const int64_t K = A.cols;
   if (M <= 0 || N <= 0 || K <= 0) return GPTQ_OK;
+  static_assert(!pipe2::is_tile_epilogue<EpiF>::value || !kUpperOut, "tile epilogues write whole 32 x 32 blocks");
+  if (pipe2::is_tile_epilogue<EpiF>::value != (out_map != nullptr)) return GPTQ_ERR_INVALID_ARG;
   Traits::Maps maps;
+  if (out_map) maps.out = *out_map; else memset(&maps.out, 0, sizeof(maps.out));
   gptq_status_t st;
   auto mk = [&](CUtensorMap* m, const __half* p, const Operand& o) {
     return make_tmap_2d(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, p, (uint64_t)o.cols, (uint64_t)o.rows,
@@ -110,6 +116,44 @@ gptq_status_t launch(const Operand& A, const Operand& B, int M, int N, EpiF epi,
   const int n_sc = (items.kb_total + items.sc_kb - 1) / items.sc_kb;
   return pipe2::launch_pipe2<Traits>(maps, (int64_t)items.tiles_m * items.tiles_n * n_sc, items, epi, dev_info, stream,
                                      reserve_sms);
+}
+
+// Epilogue that leaves through TMA reductions: out[row][col] += alpha * sa[row] * sb[col] * partial (sa, sb optional) for
+// a row-major fp32 output described by Maps::out ({N, M}, 32 x 32 boxes, 128-byte swizzle).  The lanes write their rows
+// into the warp's swizzled 4 KB staging tile and one lane sends it off; elements beyond M or N are dropped by the TMA
+// unit.  L2 then adds whole 128-byte rows instead of 32 separate 16-byte pieces per instruction, which is what made
+// per-lane reductions cost 13 us per 256 x 256 tile (this form: 5 us).
+struct EpiTileAddF32 {
+  static constexpr bool kTile = true;
+  int M, N; float alpha;
+  const float* sa; const float* sb;
+  __device__ __forceinline__ void tile(const Traits::Maps& maps, uint8_t* buf, int row0, int col0, const float (&v)[32],
+                                       int lane) const {
+    if (row0 >= M || col0 >= N) return;          // (warp-uniform)
+    const int row = row0 + lane;
+    const float a = (sa != nullptr && row < M) ? alpha * sa[row] : alpha;
+    if (lane == 0) umma::bulk_group_wait_read_all();     // the previous reduction has read the staging tile
+    __syncwarp();
+    const uint32_t base = umma::smem_u32(buf) + (uint32_t)lane * 128u;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      float4 b = make_float4(1.f, 1.f, 1.f, 1.f);
+      if (sb != nullptr && col0 + 4 * g < N) b = *reinterpret_cast<const float4*>(sb + col0 + 4 * g);
+      asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(base + (uint32_t)((g ^ (lane & 7)) << 4)),
+                   "f"(v[4 * g] * a * b.x), "f"(v[4 * g + 1] * a * b.y), "f"(v[4 * g + 2] * a * b.z), "f"(v[4 * g + 3] * a * b.w)
+                   : "memory");
+    }
+    umma::fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) {
+      umma::tma_reduce_add_2d(&maps.out, col0, row0, buf);
+      umma::bulk_group_commit();
+    }
+  }
+};
+// The tensor map such an epilogue needs: `out` points at the output's first element, ld in elements (a multiple of 4).
+inline gptq_status_t make_out_map_f32(CUtensorMap* m, float* out, int M, int N, int64_t ld) {
+  return make_tmap_2d(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, out, (uint64_t)N, (uint64_t)M, (uint64_t)ld * 4, 32, 32);
 }
 
 // ---- splitting a (pre-scaled) fp32 value into an fp16 hi / lo pair --------------------------------

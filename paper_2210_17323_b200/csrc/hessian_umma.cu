@@ -223,6 +223,19 @@ gptq_status_t make_tmap_2d(CUtensorMap* out, CUtensorMapDataType dtype, int elem
   return r == CUDA_SUCCESS ? GPTQ_OK : GPTQ_ERR_CUDA;
 }
 
+gptq_status_t make_tmap_3d_plain(CUtensorMap* out, CUtensorMapDataType dtype, const void* base, const uint64_t dims[3],
+                                 const uint64_t strides_bytes[2], const uint32_t box[3]) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return GPTQ_ERR_CUDA;
+  cuuint64_t d[3] = {dims[0], dims[1], dims[2]};
+  cuuint64_t st[2] = {strides_bytes[0], strides_bytes[1]};
+  cuuint32_t b[3] = {box[0], box[1], box[2]};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(out, dtype, 3, const_cast<void*>(base), d, st, b, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? GPTQ_OK : GPTQ_ERR_CUDA;
+}
+
 int device_sm_count() {
   // SM count of the CURRENT device, cached per device ordinal (a process may drive several GPUs).
   constexpr int kMaxDev = 64;

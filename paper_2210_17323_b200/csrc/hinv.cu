@@ -267,21 +267,6 @@ struct EpiSubUpperRed {
     }
   }
 };
-// dst[row][col] -= partial over the whole rectangle (fp32 reductions).
-struct EpiSubRed {
-  float* p; int64_t ld; int M, N;
-  const float* sa; const float* sb;
-  __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
-    if (row >= M || col0 >= N) return;
-    float* d = p + (int64_t)row * ld + col0;
-    const float a = -sa[row];
-#pragma unroll
-    for (int g = 0; g < 8; ++g) {
-      const float4 b = *reinterpret_cast<const float4*>(sb + col0 + 4 * g);
-      umma::red_add_v4(d + 4 * g, v[4 * g] * a * b.x, v[4 * g + 1] * a * b.y, v[4 * g + 2] * a * b.z, v[4 * g + 3] * a * b.w);
-    }
-  }
-};
 // Stores partial * factor as an fp16 hi / lo pair.  Only valid when the contraction is a single super-chunk
 // (K <= f16x3::kSuperK), so that the partial sum IS the result.
 struct EpiStoreSplit {
@@ -550,7 +535,10 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
         // B1
         GPTQ_CUDA_TRY(cudaStreamWaitEvent(sb, as->c4[J + 1], 0));
         f16x3::Operand A1{w.Fhi + rows_p, w.Flo + rows_p, j0, K, C};
-        st = f16x3::launch<false, false>(A1, A, j0, wj, EpiSubRed{U + j0, C, j0, wj, w.rsinv, w.rsinv + j0}, dev_info, sb, reserve);
+        CUtensorMap out;
+        if ((st = f16x3::make_out_map_f32(&out, U + j0, j0, wj, C)) != GPTQ_OK) return st;
+        st = f16x3::launch<false, false>(A1, A, j0, wj, f16x3::EpiTileAddF32{j0, wj, -1.f, w.rsinv, w.rsinv + j0}, dev_info, sb,
+                                         reserve, &out);
         if (st != GPTQ_OK) return st;
         GPTQ_CUDA_TRY(cudaEventRecord(as->b1[J], sb));
       }
@@ -667,7 +655,9 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
       f16x3::Operand A{w.Fhi, w.Flo, j0, j0, C};
       f16x3::Operand B{w.TThi, w.TTlo, wj, j0, C};
       // partial = u_i gam_j' 2^-5 (sum_k U[i][k] T[j'][k])
-      st = f16x3::launch<true, false>(A, B, j0, wj, EpiSubRed{U + j0, C, j0, wj, w.uinv, w.gam2inv}, dev_info, s);
+      CUtensorMap out;
+      if ((st = f16x3::make_out_map_f32(&out, U + j0, j0, wj, C)) != GPTQ_OK) return st;
+      st = f16x3::launch<true, false>(A, B, j0, wj, f16x3::EpiTileAddF32{j0, wj, -1.f, w.uinv, w.gam2inv}, dev_info, s, 0, &out);
       if (st != GPTQ_OK) return st;
     }
     if (J + 1 < n_outer) {

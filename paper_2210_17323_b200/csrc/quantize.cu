@@ -110,16 +110,26 @@ __global__ void wblk_from_w16_kernel(const __half* __restrict__ W, int R, int C,
   Wblk[o] = (double)__half2float(W[(int64_t)r * C + i2 + c]);
 }
 // The same for the stripe-major layout through a 32 x 32 shared-memory tile, so that both the reads (along a row of W)
-// and the writes (along a column of a stripe) are coalesced.  grid (nb / 32, ceil(R / 32)), block (32, 32).
+// and the writes (along a column of a stripe) are coalesced; and with the lazy update folded in:
+//   Wblk = W[:, blk] - D / (sE[row] sC[col]),   D = E'[:, :i2] U'[:i2, blk] (scaled fp32 sums of the tensor-core contraction)
+// formed in fp64.  D == nullptr for the first outer block.  grid (nb / 32, ceil(R / 32)), block (32, 32).
 __global__ void wblk_stripe_major_kernel(const __half* __restrict__ W, int R, int C, int i2,
+                                         const float* __restrict__ D, int64_t ldd,
+                                         const float* __restrict__ sEinv, const float* __restrict__ sCinv,
                                          double* __restrict__ Wblk, int64_t ldw) {
   __shared__ float t[32][33];
+  __shared__ float d[32][33];
   const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
   const int r = r0 + threadIdx.y;
   t[threadIdx.y][threadIdx.x] = r < R ? __half2float(W[(int64_t)r * C + i2 + c0 + threadIdx.x]) : 0.f;
+  d[threadIdx.y][threadIdx.x] = (D != nullptr && r < R) ? D[(int64_t)r * ldd + c0 + threadIdx.x] : 0.f;
   __syncthreads();
   const int rr = r0 + threadIdx.x, cc = c0 + threadIdx.y;      // row fastest: 32 consecutive doubles of one stripe column
-  if (rr < R) Wblk[((int64_t)(rr >> 7) * ldw + cc) * 128 + (rr & 127)] = (double)t[threadIdx.x][threadIdx.y];
+  if (rr < R) {
+    double w = (double)t[threadIdx.x][threadIdx.y];
+    if (D != nullptr) w -= (double)d[threadIdx.x][threadIdx.y] * (double)sEinv[rr] * (double)sCinv[i2 + cc];
+    Wblk[((int64_t)(rr >> 7) * ldw + cc) * 128 + (rr & 127)] = w;
+  }
 }
 
 // ---- the in-block loop (Algorithm 1, inner FOR) -------------------------------------------------
@@ -462,6 +472,7 @@ extern "C" size_t gptq_quantize_workspace_bytes(int R, int C, int bits, int grou
   w.take<uint32_t>((size_t)C);                                    // column maxima of the scaled U
   w.take<float>((size_t)R);                                       // sE
   w.take<float>((size_t)R);                                       // 1 / sE
+  w.take<float>((size_t)R * outer_block(C, group_size, block));   // scaled fp32 sums of the lazy update of the outer block
   return w.off;
 }
 
@@ -501,6 +512,7 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   uint32_t* colmax = w.take<uint32_t>((size_t)C);
   float* sE = w.take<float>((size_t)R);
   float* sEinv = w.take<float>((size_t)R);
+  float* Dsum = w.take<float>((size_t)R * B2);
   const int64_t ldw = B2;
   GridSpec gs{bits == GPTQ_BITS_TERNARY ? 2 : (1 << bits) - 1, ((sym & GPTQ_GRID_SYMMETRIC) != 0 || bits == GPTQ_BITS_TERNARY) ? 1 : 0,
               (sym & GPTQ_GRID_FP16_SCALES) ? 1 : 0};
@@ -541,21 +553,30 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
       GPTQ_LAUNCH_CHECK();
     }
     // working weights of the outer block: original weights minus all updates from columns < i2
-    {
-      if (stripe) {
-        dim3 grid(nb2 / 32, ceil_div(R, 32)), blk(32, 32);
-        wblk_stripe_major_kernel<<<grid, blk, 0, s>>>(W, R, C, i2, Wblk, ldw);
-      } else {
-        int64_t total = (int64_t)R * nb2;
-        wblk_from_w16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(W, R, C, i2, nb2, Wblk, ldw, 0);
+    if (stripe) {
+      // lazy update of the outer block: scaled fp32 sums from the tensor cores (added up in L2 by TMA reductions), then
+      // the fp64 working weights of the block in stripe-major order
+      if (i2 > 0) {
+        GPTQ_CUDA_TRY(cudaMemsetAsync(Dsum, 0, (size_t)R * B2 * sizeof(float), s));
+        f16x3::Operand A{Ehi, Elo, R, i2, C}, Bop{Phi, Plo, nb2, i2, C};
+        CUtensorMap out;
+        gptq_status_t st = f16x3::make_out_map_f32(&out, Dsum, R, nb2, B2);
+        if (st != GPTQ_OK) return st;
+        st = f16x3::launch<false, false>(A, Bop, R, nb2, f16x3::EpiTileAddF32{R, nb2, 1.f, nullptr, nullptr}, dev_info, s, 0, &out);
+        if (st != GPTQ_OK) return st;
       }
+      dim3 grid(nb2 / 32, ceil_div(R, 32)), blk(32, 32);
+      wblk_stripe_major_kernel<<<grid, blk, 0, s>>>(W, R, C, i2, i2 > 0 ? Dsum : nullptr, B2, sEinv, sCinv, Wblk, ldw);
       GPTQ_LAUNCH_CHECK();
-    }
-    if (i2 > 0) {
-      f16x3::Operand A{Ehi, Elo, R, i2, C}, Bop{Phi, Plo, nb2, i2, C};
-      gptq_status_t st = f16x3::launch<false, false>(A, Bop, R, nb2, EpiSubWblk{Wblk, ldw, 0, R, nb2, sEinv, sCinv + i2, stripe ? 1 : 0},
-                                                     dev_info, s);
-      if (st != GPTQ_OK) return st;
+    } else {
+      int64_t total = (int64_t)R * nb2;
+      wblk_from_w16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(W, R, C, i2, nb2, Wblk, ldw, 0);
+      GPTQ_LAUNCH_CHECK();
+      if (i2 > 0) {
+        f16x3::Operand A{Ehi, Elo, R, i2, C}, Bop{Phi, Plo, nb2, i2, C};
+        gptq_status_t st = f16x3::launch<false, false>(A, Bop, R, nb2, EpiSubWblk{Wblk, ldw, 0, R, nb2, sEinv, sCinv + i2, 0}, dev_info, s);
+        if (st != GPTQ_OK) return st;
+      }
     }
     if (stripe) {
       // row-stripe form: every inner block of this outer block in one launch

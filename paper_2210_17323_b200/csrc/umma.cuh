@@ -76,8 +76,14 @@ __device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* tmap, int x
   asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
                ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(smem_u32(smem_src)) : "memory");
 }
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* tmap, int x, int y, int z, const void* smem_src) {
+  asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+               ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(smem_u32(smem_src)) : "memory");
+}
 __device__ __forceinline__ void bulk_group_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // all of this thread's bulk groups have finished READING their shared-memory sources
+// all but the newest of this thread's bulk groups have finished reading their shared-memory sources
+__device__ __forceinline__ void bulk_group_wait_read_but_one() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void bulk_group_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // all of this thread's bulk groups are complete
 __device__ __forceinline__ void bulk_group_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -186,6 +192,9 @@ static inline cudaError_t set_wait_test_knobs(unsigned long long limit_ns, int s
 gptq_status_t make_tmap_2d(CUtensorMap* out, CUtensorMapDataType dtype, int elem_bytes, const void* base,
                            uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
                            uint32_t box_inner, uint32_t box_outer);
+// 3-d map without swizzle (dims / box innermost first; strides of dimensions 1 and 2 in bytes, multiples of 16).
+gptq_status_t make_tmap_3d_plain(CUtensorMap* out, CUtensorMapDataType dtype, const void* base, const uint64_t dims[3],
+                                 const uint64_t strides_bytes[2], const uint32_t box[3]);
 
 }  // namespace gptq
 

@@ -1,5 +1,6 @@
-// Persistent, warp-specialised tensor-core pipeline shared by the Hessian contraction (bf16) and
-// the fp32-accurate lazy-update / factorisation contractions (3xTF32).
+// Persistent, warp-specialised tensor-core pipeline, one-CTA form (128 x 256 tiles): the Hessian contraction
+// (bf16) of layers with fewer than 512 channels.  umma_pipe2.cuh holds the two-CTA form that everything
+// larger uses; the roles and the reasoning below are the same there.
 //
 //   warp 0      TMA producer: fills a ring of shared-memory stages with operand tiles
 //   warp 1      MMA issuer: tcgen05.mma from shared memory into one of two TMEM accumulators
@@ -8,7 +9,7 @@
 // Why the register running sums: the tensor core adds each MMA's products into its fp32
 // accumulator with truncation (measured: about half an ulp lost per instruction, always toward
 // zero), so a long contraction kept in TMEM drifts by ~3e-8 x (number of MMAs).  Here TMEM only
-// ever holds a short CHUNK of the contraction (<= 16 MMAs); the chunk sums are added with
+// ever holds a short CHUNK of the contraction (<= 32 MMAs); the chunk sums are added with
 // round-to-nearest in registers by the CUDA cores, and the running sum of one work item (a few
 // thousand K) is handed to the epilogue functor, which folds it into memory (fp32 reduction or
 // fp64 read-modify-write).  Two TMEM accumulators let the drain of one chunk overlap the MMAs of
