@@ -631,76 +631,33 @@ def run_block_sweep(args, wl):
 
 
 def run_e2e(args, wl, state, device_value):
-    """Same metric end to end through the C ABI's host-buffer call: every step, for every layer (and grid),
-    gptq_solve_layer_host streams X and W from pinned HOST memory to the device (copies overlapped with the
-    Hessian accumulation), solves, and copies codes, scales, zeros and loss back to the host."""
+    """Same metric end to end from HOST buffers through the package's host-input solver: every step, every layer's X and
+    W cross from pinned host memory to the device (copies overlapped with the Hessian accumulation and with the other
+    layers' stages), every grid is solved, and codes, scales, zeros and losses are copied back to pinned host memory."""
     import torch
-    from paper_2210_17323_b200 import binding as B
 
-    host = []
-    need = 256
+    from paper_2210_17323_b200 import pipeline
     grids = [(g.bits, g.group_size, g.sym) for g in wl.grids]
-    import ctypes
-    for st in state:
-        L = st["L"]
-        host.append(dict(L=L, X=st["X"].cpu().pin_memory(), W=st["W"].cpu().pin_memory(), outs=None))
-        ng = len(grids)
-        need = max(need, B._lib.gptq_solve_layer_host_grids_workspace_bytes(
-            L.R, L.C, L.n_tokens, ng, (ctypes.c_int * ng)(*[g[0] for g in grids]), (ctypes.c_int * ng)(*[g[1] for g in grids]), wl.block))
-    for st in state:                       # device copies are not needed any more: the call has its own staging
-        st["X"] = st["H"] = st["U"] = st["ws"] = None
+    layers = [(st["W"].cpu().pin_memory(), st["X"].cpu().pin_memory()) for st in state]
+    shapes = [(st["L"].R, st["L"].C, st["L"].n_tokens) for st in state]
+    for st in state:                       # the device copies of the device-timed leg are not needed any more
+        st["X"] = st["W"] = st["H"] = st["U"] = st["ws"] = None
+    state.clear()
     torch.cuda.empty_cache()
-    # Two calls in flight (two host threads, each with its own stream and device workspace): while one layer is being
-    # factored and quantized, the next layer's activations are already crossing PCIe.  Every call solves ALL grids of its
-    # layer, so a layer's activations cross once per step.
-    n_workers = 2 if need * 2 < 120e9 and len(host) > 1 else 1
-    dev = torch.cuda.current_device()
-    workers = [dict(ws=torch.empty(need, dtype=torch.uint8, device="cuda"), stream=torch.cuda.Stream()) for _ in range(n_workers)]
+    solver = pipeline.HostLayerSolver(shapes, grids, block=wl.block, damp=wl.damp)
     torch.cuda.synchronize()
-    h2d = sum(h["X"].numel() * 2 + h["W"].numel() * 2 for h in host)
-    tasks = sorted(host, key=lambda h: -(h["L"].C ** 2) * (h["L"].n_tokens + h["L"].C))
-    import queue
-
-    def step():
-        q = queue.Queue()
-        for t in tasks:
-            q.put(t)
-        errors = []
-
-        def work(wk):
-            torch.cuda.set_device(dev)
-            try:
-                while True:
-                    try:
-                        h = q.get_nowait()
-                    except queue.Empty:
-                        return
-                    h["outs"] = B.gptq_solve_layer_host_grids(h["W"], h["X"], grids, wl.block, wl.damp, outs=h["outs"],
-                                                              dev_ws=wk["ws"], stream=wk["stream"])
-                    assert h["outs"][0]["info"].tolist()[0] == 0, h["outs"][0]["info"].tolist()
-            except Exception as e:          # surfaced after the join
-                errors.append(e)
-
-        threads = [threading.Thread(target=work, args=(wk,)) for wk in workers]
-        for t in threads:
-            t.start()
-        for t in threads:
-            t.join()
-        if errors:
-            raise errors[0]
-        return sum(o[k].numel() * o[k].element_size() for h in host for o in h["outs"] for k in ("qweight", "scales", "zeros")) + \
-            sum(8 * len(h["outs"]) + 8 for h in host)
-
     steps = max(1, min(args.steps, 5))      # each step moves every layer's activations across PCIe again (seconds)
-    d2h = step()
+    solver.solve(layers)                    # warm-up (kernel attributes, allocator)
+    solver.solve(layers)
     t0 = time.perf_counter()
     for _ in range(steps):
-        d2h = step()                        # every call returns with its results on the host: wall clock is the e2e time
+        solver.solve(layers)                # returns with the results on the host: wall clock is the e2e time
     dt = (time.perf_counter() - t0) / steps
-    return dict(value=wl.weights * len(wl.grids) / dt, unit=UNIT, h2d_bytes_per_step=int(h2d),
-                d2h_bytes_per_step=int(d2h), ms_per_step=dt * 1e3, steps=steps,
-                api=f"gptq_solve_layer_host_grids (pinned host buffers; per layer X streamed once in 512 MiB chunks on a copy stream, "
-                    f"all {len(grids)} grid(s) solved from one Hessian and factor); {n_workers} call(s) in flight from {n_workers} host thread(s)")
+    return dict(value=wl.weights * len(wl.grids) / dt, unit=UNIT, h2d_bytes_per_step=int(solver.h2d_bytes()),
+                d2h_bytes_per_step=int(solver.d2h_bytes()), ms_per_step=dt * 1e3, steps=steps,
+                api="pipeline.HostLayerSolver.solve (pinned host buffers; one copy stream, the most expensive layer's activations "
+                    "first, in 2 GiB token chunks; Hessians accumulated chunk by chunk as the chunks land; every layer's stages "
+                    f"2-3 on its own stream, all {len(grids)} grid(s) from one Hessian and factor; results copied back to pinned memory)")
 
 
 def run_inference(args, wl):

@@ -7,7 +7,7 @@
 namespace gptq {
 namespace {
 
-constexpr int64_t kChunkBytes = (int64_t)512 << 20;   // per X staging buffer
+constexpr int64_t kChunkBytes = (int64_t)2048 << 20;  // per X staging buffer: every chunk costs one pass over H (read + write)
 
 struct HostWs {
   float* H; float* U; __half* W; __nv_bfloat16* X[2];
@@ -126,7 +126,11 @@ extern "C" gptq_status_t gptq_solve_layer_host_grids(const void* W_fp16_host, co
   HostWs w = carve_host(dev_ws, R, C, n_tokens, n_grids, bits, group_size, block);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   StreamGuard g;
-  GPTQ_CUDA_TRY(cudaStreamCreateWithFlags(&g.s, cudaStreamNonBlocking));
+  // the copy stream takes the caller's stream priority: of several calls in flight, the one on the higher-priority
+  // stream gets its activations across first
+  int prio = 0;
+  GPTQ_CUDA_TRY(cudaStreamGetPriority(s, &prio));
+  GPTQ_CUDA_TRY(cudaStreamCreateWithPriority(&g.s, cudaStreamNonBlocking, prio));
   for (int i = 0; i < 2; ++i) {
     GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&g.loaded[i], cudaEventDisableTiming));
     GPTQ_CUDA_TRY(cudaEventCreateWithFlags(&g.freed[i], cudaEventDisableTiming));

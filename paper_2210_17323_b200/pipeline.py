@@ -128,3 +128,103 @@ class BlockSolver:
             for ms in st["members"]:
                 if ms["m"].out and ms["m"].out["dev_info"].tolist()[0] != 0:
                     raise B.GptqError(ms["m"].out["dev_info"].tolist()[0], f"gptq_quantize_layer ({ms['m'].name})")
+
+
+class HostLayerSolver:
+    """Solves a set of independent layers whose weights and calibration activations sit in (pinned) HOST memory: every
+    grid of `grids` for every layer, results back in pinned host memory.
+
+    One copy stream carries all activations to the device, the most expensive layer first, in token chunks; on a second
+    stream every layer's Hessian is accumulated chunk by chunk as its chunks land (H is a sum over tokens, Section 2), so
+    the first Hessian starts after one chunk and the later layers' activations cross while the earlier layers are being
+    solved; stages 2 and 3 of a layer run on that layer's own stream as soon as its Hessian is complete, and its packed
+    codes, scales, zero-points and losses are copied back on that stream.  All layers' activations are resident at once
+    (buffers are allocated once, for the shapes given, and reused by every solve()).
+    """
+
+    def __init__(self, shapes: Sequence[tuple], grids: Sequence[tuple], block=128, damp=0.01, chunk_bytes=2 << 30, device=None):
+        """shapes: (R, C, n_tokens) per layer; grids: (bits, group_size, sym) per grid."""
+        dev = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+        self.grids, self.block, self.damp = list(grids), block, damp
+        self.order = sorted(range(len(shapes)), key=lambda i: -(shapes[i][1] ** 2) * (shapes[i][2] + shapes[i][1]))
+        self.copy_stream = torch.cuda.Stream(device=dev)
+        self.main = torch.cuda.Stream(device=dev)
+        self.state = []
+        for (R, C, n) in shapes:
+            ct = max(64, (chunk_bytes // (2 * C)) // 64 * 64)
+            chunks = [(t0, min(n, t0 + ct)) for t0 in range(0, n, ct)]
+            ws_bytes = max([256, B.gptq_hessian_workspace_bytes(C, n), B.gptq_prepare_hinv_workspace_bytes(C)] +
+                           [B.gptq_quantize_workspace_bytes(R, C, b, g, block) for (b, g, _) in self.grids])
+            outs = []
+            for (b, g, _) in self.grids:
+                G = C // g if g > 0 else 1
+                outs.append(dict(qweight=torch.empty((R, C * B.field_bits(b) // 32), dtype=torch.int32).pin_memory(),
+                                 scales=torch.empty((R, G), dtype=torch.float32).pin_memory(),
+                                 zeros=torch.empty((R, G), dtype=torch.float32).pin_memory(),
+                                 loss=torch.empty(1, dtype=torch.float64).pin_memory(),
+                                 info=torch.empty(2, dtype=torch.int32).pin_memory()))
+            self.state.append(dict(R=R, C=C, n=n, chunks=chunks,
+                                   X=torch.empty((n, C), dtype=torch.bfloat16, device=dev),
+                                   W=torch.empty((R, C), dtype=torch.float16, device=dev),
+                                   H=torch.empty((C, C), dtype=torch.float32, device=dev),
+                                   U=torch.empty((C, C), dtype=torch.float32, device=dev),
+                                   info_h=torch.zeros((len(chunks), 2), dtype=torch.int32, device=dev),
+                                   info_u=torch.zeros(2, dtype=torch.int32, device=dev),
+                                   info_host=torch.empty((len(chunks) + 1, 2), dtype=torch.int32).pin_memory(),
+                                   ws=torch.empty(ws_bytes, dtype=torch.uint8, device=dev),
+                                   stream=torch.cuda.Stream(device=dev), outs=outs))
+
+    def h2d_bytes(self):
+        return sum(st["X"].numel() * 2 + st["W"].numel() * 2 for st in self.state)
+
+    def d2h_bytes(self):
+        return sum(t.numel() * t.element_size() for st in self.state for o in st["outs"] for t in o.values()) + \
+            sum(st["info_host"].numel() * 4 for st in self.state)
+
+    def solve(self, layers: Sequence[tuple]):
+        """layers: (W_host [R, C] fp16, X_host [n_tokens, C] bf16) per layer, in the order of `shapes`.  Returns, per
+        layer, one dict(qweight, scales, zeros, loss, info) of pinned CPU tensors per grid (reused by the next call).
+        Returns when every result is on the host; raises GptqError on a device-side failure."""
+        cur = torch.cuda.current_stream()
+        start = torch.cuda.Event(); start.record(cur)
+        self.copy_stream.wait_event(start); self.main.wait_event(start)
+        landed = {}
+        with torch.cuda.stream(self.copy_stream):
+            for li in self.order:
+                st, (Wh, Xh) = self.state[li], layers[li]
+                for ci, (t0, t1) in enumerate(st["chunks"]):
+                    st["X"][t0:t1].copy_(Xh[t0:t1], non_blocking=True)
+                    e = torch.cuda.Event(); e.record(self.copy_stream); landed[(li, ci)] = e
+                st["W"].copy_(Wh, non_blocking=True)
+                e = torch.cuda.Event(); e.record(self.copy_stream); landed[(li, "W")] = e
+        ends = []
+        for li in self.order:
+            st = self.state[li]
+            with torch.cuda.stream(self.main):
+                st["H"].zero_()
+                for ci, (t0, t1) in enumerate(st["chunks"]):
+                    self.main.wait_event(landed[(li, ci)])
+                    B.gptq_hessian_accumulate(st["H"], st["X"][t0:t1], ws=st["ws"], dev_info=st["info_h"][ci])
+                h_done = torch.cuda.Event(); h_done.record(self.main)
+            s = st["stream"]
+            with torch.cuda.stream(s):
+                s.wait_event(h_done); s.wait_event(landed[(li, "W")])
+                B.gptq_prepare_hinv(st["H"], self.damp, U=st["U"], ws=st["ws"], dev_info=st["info_u"])
+                st["info_host"][:-1].copy_(st["info_h"], non_blocking=True)
+                st["info_host"][-1].copy_(st["info_u"], non_blocking=True)
+                for (b, g, sym), o in zip(self.grids, st["outs"]):
+                    r = B.gptq_quantize_layer(st["W"], st["U"], b, g, sym, self.block, ws=st["ws"])
+                    for k, src in (("qweight", r["qweight"]), ("scales", r["scales"]), ("zeros", r["zeros"]), ("loss", r["loss"]),
+                                   ("info", r["dev_info"])):
+                        o[k].copy_(src, non_blocking=True)
+                e = torch.cuda.Event(); e.record(s); ends.append(e)
+        for e in ends:
+            e.synchronize()
+        for li, st in enumerate(self.state):
+            for row in st["info_host"].tolist():
+                if row[0] != 0:
+                    raise B.GptqError(row[0], f"layer {li}: stage 1 / 2 (detail {row[1]})")
+            for o in st["outs"]:
+                if o["info"].tolist()[0] != 0:
+                    raise B.GptqError(o["info"].tolist()[0], f"layer {li}: gptq_quantize_layer")
+        return [st["outs"] for st in self.state]

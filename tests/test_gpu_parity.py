@@ -550,3 +550,28 @@ def test_solve_layer_from_host_buffers_several_grids(B):
     a = O.unpack_codes(single["qweight"].numpy().view(np.uint32), 3, L.C)
     b = O.unpack_codes(outs[1]["qweight"].numpy().view(np.uint32), 3, L.C)
     assert (a == b).mean() >= 0.999
+
+
+def test_host_layer_solver_matches_the_oracle(B):
+    """pipeline.HostLayerSolver: several layers from pinned host buffers in one overlapped schedule (one copy stream,
+    Hessians chunk by chunk as the chunks land, every layer's stages 2-3 on its own stream, results back on the host).
+    Small chunks so that every Hessian is accumulated over several ragged pieces; every grid of every layer against the
+    oracle; a second solve() reuses all buffers."""
+    from paper_2210_17323_b200 import pipeline
+    cases = [_layer(64, 1280, 3000, cfg=11, kind="fc2"), _layer(96, 512, 2500, cfg=12, kind="q"), _layer(40, 768, 1000, cfg=13, kind="o")]
+    grids = [(4, 0, False), (3, 128, False)]
+    layers, refs = [], []
+    for L in cases:
+        xb, W16 = L.x_bits(), L.w()
+        layers.append((torch.from_numpy(W16).pin_memory(), torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()))
+        refs.append([O.solve_layer(W16, xb, b, g, s, 128, 0.01) for (b, g, s) in grids])
+    solver = pipeline.HostLayerSolver([(L.R, L.C, L.n_tokens) for L in cases], grids, block=128, damp=0.01, chunk_bytes=1 << 20)
+    assert any(len(st["chunks"]) > 2 for st in solver.state)
+    for _ in range(2):
+        outs = solver.solve(layers)
+    for L, (Wh, _), per_grid, ref_grids in zip(cases, layers, outs, refs):
+        for (b, g, s), out, ref in zip(grids, per_grid, ref_grids):
+            assert out["info"].tolist() == [0, 0]
+            gpu = dict(qweight=out["qweight"].numpy(), scales=out["scales"].numpy(), zeros=out["zeros"].numpy(),
+                       loss=out["loss"].item())
+            check_quantize_outputs(gpu, ref, Wh.numpy(), b, L.C, ref["H"])
