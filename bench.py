@@ -408,19 +408,19 @@ def run_gpu(args, wl):
     # the stage sums overlap one another in the overlapped schedule, so the dominant kernel is chosen against the step
     if tot["hessian_ms"] >= tot["quantize_ms"] or tot["hessian_ms"] >= 0.3 * ms_per_step:
         ach = hess_flops / (tot["hessian_ms"] * 1e-3) / 1e12
-        # DRAM traffic per launch: dram__bytes_read + dram__bytes_write of this kernel were captured on two smaller
-        # launches (profiles/hessian_two_cta_kernel_4096ch_65536tok.md): 2.4 x the algorithmic bytes (X once + H once) at
-        # 4096 channels and 10.9 x at 16384 channels (every band of tile rows streams the column strips to its right
-        # again); the ratio is interpolated linearly in C between them and extrapolated beyond, and scaled to these
-        # launches by their algorithmic bytes
-        def traffic_ratio(C):
-            return 2.4 if C <= 4096 else 2.4 + (10.9 - 2.4) * (C - 4096) / (16384 - 4096)
+        # DRAM traffic per launch: dram__bytes_read + dram__bytes_write of this kernel, captured at 4096, 12288, 16384 and
+        # 49152 channels x 65536 tokens, is 1.39 - 1.45e-3 bytes per token and channel^2 at every size (18 % of the operand
+        # fill of the CTA pairs comes from DRAM): it grows with the flops, not with the algorithmic bytes, so the full-size
+        # launches' figure is that rate x C^2 x tokens
+        kTrafficPerTokenChannel2 = 1.41e-3
         algo_bytes = sum(L.n_tokens * L.C * 2 + L.C * L.C * 4 for L in layers) / len(layers)
-        est_traffic = sum(traffic_ratio(L.C) * (L.n_tokens * L.C * 2 + L.C * L.C * 4) for L in layers) / len(layers)
+        est_traffic = sum(max(kTrafficPerTokenChannel2 * L.C * L.C * L.n_tokens, L.n_tokens * L.C * 2 + L.C * L.C * 4)
+                          for L in layers) / len(layers)
         roof = dict(kernel="hessian_accumulate", bound="tensor", achieved=ach, peak=peaks["bf16_sustained"],
                     unit="TFLOP/s", frac=ach / peaks["bf16_sustained"], traffic=est_traffic,
-                    traffic_note=f"bytes per launch, mean over layers = {est_traffic / algo_bytes:.1f} x algorithmic bytes; from ncu "
-                                 "captures of 4096- and 16384-channel launches (2.4 x and 10.9 x), interpolated in C",
+                    traffic_note=f"bytes per launch, mean over layers = {est_traffic / algo_bytes:.1f} x algorithmic bytes (X once + H "
+                                 "once); 1.41e-3 bytes per token and channel^2, from ncu captures of 4096- to 49152-channel "
+                                 "launches of 65536 tokens (1.39 - 1.45e-3 at every size)",
                     peak_source=f"bf16 sustained, {peaks['source']}")
     else:
         ach = 3 * upd_flops / (tot["quantize_ms"] * 1e-3) / 1e12
