@@ -32,26 +32,49 @@ dequantize_kernel(const uint32_t* __restrict__ qweight, const float* __restrict_
   const bool two = o + 8 * F > 32;
   const int gi0 = c0 / g;
   const int64_t wpr = (int64_t)(C / 32) * F;                  // words per row
-  for (int r = blockIdx.y; r < R; r += gridDim.y) {
-    const uint32_t* rowp = qweight + r * wpr;
-    uint64_t v = __ldg(rowp + k);
-    if (two) v |= (uint64_t)__ldg(rowp + k + 1) << 32;
-    v >>= o;
-    __align__(16) __half h[8];
-    if (g >= 8) {
-      const float s = __ldg(scales + (int64_t)r * G + gi0), z = __ldg(zeros + (int64_t)r * G + gi0);
+  // four rows per trip: their loads are issued together, so that a thread has four independent round trips to
+  // memory in flight instead of one
+  constexpr int kRows = 4;
+  const int stride = gridDim.y;
+  for (int r0 = blockIdx.y; r0 < R; r0 += kRows * stride) {
+    uint64_t v[kRows];
+    float s[kRows], z[kRows];
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
-        h[i] = __float2half_rn(__fmul_rn(s, (float)(uint32_t)((v >> (i * F)) & ((1u << F) - 1u)) - z));
-    } else {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int gi = (c0 + i) / g;
-        const float s = __ldg(scales + (int64_t)r * G + gi), z = __ldg(zeros + (int64_t)r * G + gi);
-        h[i] = __float2half_rn(__fmul_rn(s, (float)(uint32_t)((v >> (i * F)) & ((1u << F) - 1u)) - z));
+    for (int u = 0; u < kRows; ++u) {
+      const int r = r0 + u * stride;
+      v[u] = 0; s[u] = 0.f; z[u] = 0.f;
+      if (r < R) {
+        const uint32_t* rowp = qweight + r * wpr;
+        v[u] = __ldg(rowp + k);
+        if (two) v[u] |= (uint64_t)__ldg(rowp + k + 1) << 32;
+        if (g >= 8) { s[u] = __ldg(scales + (int64_t)r * G + gi0); z[u] = __ldg(zeros + (int64_t)r * G + gi0); }
       }
     }
-    __stcs(reinterpret_cast<uint4*>(out + (int64_t)r * C + c0), *reinterpret_cast<const uint4*>(h));
+#pragma unroll
+    for (int u = 0; u < kRows; ++u) {
+      const int r = r0 + u * stride;
+      if (r >= R) break;
+      const uint64_t w64 = v[u] >> o;
+      const uint32_t w32 = (uint32_t)w64;            // the 8 F bits of the eight codes fit one word unless F = 8
+      // code -> float without an integer conversion: the bit pattern (code | 0x4B000000) is 2^23 + code exactly
+      auto code_f = [&](int i) -> float {
+        const uint32_t q = (F < 8 ? (w32 >> (i * F)) : (uint32_t)(w64 >> (i * F))) & ((1u << F) - 1u);
+        return __fsub_rn(__uint_as_float(q | 0x4B000000u), 8388608.f);
+      };
+      __align__(16) __half h[8];
+      if (g >= 8) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) h[i] = __float2half_rn(__fmul_rn(s[u], __fsub_rn(code_f(i), z[u])));
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int gi = (c0 + i) / g;
+          const float sc = __ldg(scales + (int64_t)r * G + gi), zz = __ldg(zeros + (int64_t)r * G + gi);
+          h[i] = __float2half_rn(__fmul_rn(sc, __fsub_rn(code_f(i), zz)));
+        }
+      }
+      __stcs(reinterpret_cast<uint4*>(out + (int64_t)r * C + c0), *reinterpret_cast<const uint4*>(h));
+    }
   }
 }
 
