@@ -575,3 +575,27 @@ def test_host_layer_solver_matches_the_oracle(B):
             gpu = dict(qweight=out["qweight"].numpy(), scales=out["scales"].numpy(), zeros=out["zeros"].numpy(),
                        loss=out["loss"].item())
             check_quantize_outputs(gpu, ref, Wh.numpy(), b, L.C, ref["H"])
+
+
+def test_two_hessian_launches_side_by_side_on_two_streams(B):
+    """Two Hessian accumulations of different shapes enqueued on two streams at once.  Each launch hands its work items
+    out among its own running clusters (a cluster takes over the items of clusters of ITS grid that have not started);
+    with both grids resident at the same time every item must still be done exactly once: on integer-valued inputs the
+    results are exact, so one lost or repeated item would show."""
+    r = np.random.default_rng(11)
+    shapes = [(1280, 9000), (768, 20000)]
+    Xs = [torch.from_numpy(r.integers(-4, 5, size=(m, C)).astype(np.float32)).cuda().to(torch.bfloat16) for C, m in shapes]
+    Hs = [torch.zeros((C, C), dtype=torch.float32, device="cuda") for C, _ in shapes]
+    infos = [torch.zeros(2, dtype=torch.int32, device="cuda") for _ in shapes]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    for rep in range(3):                      # three rounds: 3 x the exact sum
+        for X, H, info, s in zip(Xs, Hs, infos, streams):
+            with torch.cuda.stream(s):
+                B.gptq_hessian_accumulate(H, X, dev_info=info)
+    torch.cuda.synchronize()
+    for X, H, info in zip(Xs, Hs, infos):
+        assert info.tolist() == [0, 0]
+        Xd = X.double()
+        exact = (6.0 * (Xd.T @ Xd)).cpu().numpy()
+        assert np.array_equal(H.cpu().numpy().astype(np.float64), exact)
