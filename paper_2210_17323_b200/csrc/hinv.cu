@@ -117,8 +117,11 @@ rchol_diag_kernel(float* __restrict__ U, int C, int k0, int nb, float* __restric
     for (int q = 0; q < kDiagBatch; ++q) {
       const int j = jt - q;
       if (ty == (j & 15)) {
-        // owner warp of column j (its slots have b == j >> 4): dispatch once on b so that the
-        // four slots are addressed with compile-time indices
+        // owner warp of column j (its slots have b == j >> 4).  Inside a batch a column is handed from its owner to
+        // the next column's owner alone (a two-warp named barrier; consecutive columns have different owners): the
+        // other fourteen warps have nothing to do until the batch is complete and wait for the full barrier below.
+        if (q > 0) asm volatile("bar.sync %0, 64;" ::"r"(q) : "memory");
+        // dispatch once on b so that the four slots are addressed with compile-time indices
         switch (j >> 4) {
           case 0: diag_owner_step<0>(M, colv, pd, q, j, jt, tx, k0, dev_info); break;
           case 1: diag_owner_step<1>(M, colv, pd, q, j, jt, tx, k0, dev_info); break;
@@ -129,9 +132,10 @@ rchol_diag_kernel(float* __restrict__ U, int C, int k0, int nb, float* __restric
           case 6: diag_owner_step<6>(M, colv, pd, q, j, jt, tx, k0, dev_info); break;
           default: diag_owner_step<7>(M, colv, pd, q, j, jt, tx, k0, dev_info); break;
         }
+        if (q + 1 < kDiagBatch) asm volatile("bar.arrive %0, 64;" ::"r"(q + 1) : "memory");
       }
-      __syncthreads();
     }
+    __syncthreads();
     // the batch's four rank-1 updates on every element left of the batch
     const int jlow = jt - (kDiagBatch - 1);
     double x[kDiagBatch][4];
