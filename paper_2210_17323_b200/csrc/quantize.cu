@@ -109,26 +109,41 @@ __global__ void wblk_from_w16_kernel(const __half* __restrict__ W, int R, int C,
   const int64_t o = stripe_major ? ((int64_t)(r >> 7) * ldw + c) * 128 + (r & 127) : (int64_t)r * ldw + c;
   Wblk[o] = (double)__half2float(W[(int64_t)r * C + i2 + c]);
 }
-// The same for the stripe-major layout through a 32 x 32 shared-memory tile, so that both the reads (along a row of W)
-// and the writes (along a column of a stripe) are coalesced; and with the lazy update folded in:
+// The same for the stripe-major layout through a shared-memory tile of one stripe's 128 rows x 32 columns, so that both
+// the reads (along rows of W and D) and the writes (along a column of the stripe: 1 KB of consecutive doubles) are
+// coalesced and a thread has sixteen loads in flight; and with the lazy update folded in:
 //   Wblk = W[:, blk] - D / (sE[row] sC[col]),   D = E'[:, :i2] U'[:i2, blk] (scaled fp32 sums of the tensor-core contraction)
-// formed in fp64.  D == nullptr for the first outer block.  grid (nb / 32, ceil(R / 32)), block (32, 32).
-__global__ void wblk_stripe_major_kernel(const __half* __restrict__ W, int R, int C, int i2,
-                                         const float* __restrict__ D, int64_t ldd,
-                                         const float* __restrict__ sEinv, const float* __restrict__ sCinv,
-                                         double* __restrict__ Wblk, int64_t ldw) {
-  __shared__ float t[32][33];
-  __shared__ float d[32][33];
-  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
-  const int r = r0 + threadIdx.y;
-  t[threadIdx.y][threadIdx.x] = r < R ? __half2float(W[(int64_t)r * C + i2 + c0 + threadIdx.x]) : 0.f;
-  d[threadIdx.y][threadIdx.x] = (D != nullptr && r < R) ? D[(int64_t)r * ldd + c0 + threadIdx.x] : 0.f;
+// formed in fp64.  D == nullptr for the first outer block.  grid (nb / 32, ceil(R / 128)), block (32, 8).
+__global__ void __launch_bounds__(256)
+wblk_stripe_major_kernel(const __half* __restrict__ W, int R, int C, int i2,
+                         const float* __restrict__ D, int64_t ldd,
+                         const float* __restrict__ sEinv, const float* __restrict__ sCinv,
+                         double* __restrict__ Wblk, int64_t ldw) {
+  __shared__ float t[128][33];
+  __shared__ float d[128][33];
+  const int r0 = blockIdx.y * 128, c0 = blockIdx.x * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+#pragma unroll
+  for (int k = 0; k < 16; ++k) {
+    const int rr = ty + 8 * k, r = r0 + rr;
+    t[rr][tx] = r < R ? __half2float(W[(int64_t)r * C + i2 + c0 + tx]) : 0.f;
+    d[rr][tx] = (D != nullptr && r < R) ? D[(int64_t)r * ldd + c0 + tx] : 0.f;
+  }
   __syncthreads();
-  const int rr = r0 + threadIdx.x, cc = c0 + threadIdx.y;      // row fastest: 32 consecutive doubles of one stripe column
-  if (rr < R) {
-    double w = (double)t[threadIdx.x][threadIdx.y];
-    if (D != nullptr) w -= (double)d[threadIdx.x][threadIdx.y] * (double)sEinv[rr] * (double)sCinv[i2 + cc];
-    Wblk[((int64_t)(rr >> 7) * ldw + cc) * 128 + (rr & 127)] = w;
+  double* out = Wblk + ((int64_t)blockIdx.y * ldw + c0) * 128;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int cc = ty + 8 * k;
+    const double sc = D != nullptr ? (double)sCinv[i2 + c0 + cc] : 0.0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int rr = tx + 32 * q, r = r0 + rr;
+      if (r < R) {
+        double w = (double)t[rr][cc];
+        if (D != nullptr) w -= (double)d[rr][cc] * (double)sEinv[r] * sc;
+        out[(int64_t)cc * 128 + rr] = w;
+      }
+    }
   }
 }
 
@@ -565,7 +580,7 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
         st = f16x3::launch<false, false>(A, Bop, R, nb2, f16x3::EpiTileAddF32{R, nb2, 1.f, nullptr, nullptr}, dev_info, s, 0, &out);
         if (st != GPTQ_OK) return st;
       }
-      dim3 grid(nb2 / 32, ceil_div(R, 32)), blk(32, 32);
+      dim3 grid(nb2 / 32, ceil_div(R, 128)), blk(32, 8);
       wblk_stripe_major_kernel<<<grid, blk, 0, s>>>(W, R, C, i2, i2 > 0 ? Dsum : nullptr, B2, sEinv, sCinv, Wblk, ldw);
       GPTQ_LAUNCH_CHECK();
     } else {
