@@ -404,19 +404,38 @@ __global__ void rowscale_kernel(const __half* __restrict__ W, int R, int C, floa
 // ---- U panel -> transposed, scaled fp16 hi / lo pair ------------------------------------------------
 // Pt[c][r] = U[r][i2 + c] / sK[r] * sC[i2 + c] for r < rows, c < nb2 (row stride ldp): the right factor of the
 // lazy updates, transposed so the contraction index is contiguous, split so that hi + lo ~ value to 2^-22.
-__global__ void split_panel_t_kernel(const float* __restrict__ U, int C, int i2, int rows,
-                                     const float* __restrict__ sK, const float* __restrict__ sC,
-                                     __half* __restrict__ Phi, __half* __restrict__ Plo, int64_t ldp) {
-  __shared__ float t[32][33];
-  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
-  t[threadIdx.y][threadIdx.x] = U[(int64_t)(r0 + threadIdx.y) * C + i2 + c0 + threadIdx.x] / sK[r0 + threadIdx.y];
+// A CTA transposes 128 rows x 32 columns through shared memory: sixteen coalesced loads in flight per thread, and per
+// column 256 consecutive bytes of each output written as half2 pairs.  grid (nb2 / 32, rows / 128 rounded up), block (32, 8).
+__global__ void __launch_bounds__(256)
+split_panel_t_kernel(const float* __restrict__ U, int C, int i2, int rows,
+                     const float* __restrict__ sK, const float* __restrict__ sC,
+                     __half* __restrict__ Phi, __half* __restrict__ Plo, int64_t ldp) {
+  __shared__ float t[128][33];
+  const int r0 = blockIdx.y * 128, c0 = blockIdx.x * 32;
+  const int tx = threadIdx.x, ty = threadIdx.y;
+#pragma unroll
+  for (int k = 0; k < 16; ++k) {
+    const int rr = ty + 8 * k, r = r0 + rr;
+    t[rr][tx] = r < rows ? U[(int64_t)r * C + i2 + c0 + tx] / sK[r] : 0.f;
+  }
   __syncthreads();
-  __half h, l;
-  bool sat = false;
-  f16x3::split_f16(t[threadIdx.x][threadIdx.y] * sC[i2 + c0 + threadIdx.y], h, l, sat);
-  const int64_t o = (int64_t)(c0 + threadIdx.y) * ldp + r0 + threadIdx.x;
-  Phi[o] = h; Plo[o] = l;
-  (void)rows;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int cc = ty + 8 * k;
+    const float sc = sC[i2 + c0 + cc];
+    const int64_t o = (int64_t)(c0 + cc) * ldp + r0;
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const int rr = 64 * q + 2 * tx;
+      if (r0 + rr >= rows) continue;               // (rows is a multiple of 32)
+      __half h0, l0, h1, l1;
+      bool sat = false;
+      f16x3::split_f16(t[rr][cc] * sc, h0, l0, sat);
+      f16x3::split_f16(t[rr + 1][cc] * sc, h1, l1, sat);
+      *reinterpret_cast<__half2*>(Phi + o + rr) = __halves2half2(h0, h1);
+      *reinterpret_cast<__half2*>(Plo + o + rr) = __halves2half2(l0, l1);
+    }
+  }
 }
 
 // ---- contraction epilogue (one thread: one row, 32 consecutive columns of a partial sum) --------
@@ -563,7 +582,7 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   for (int i2 = 0; i2 < C; i2 += B2) {
     const int nb2 = (C - i2 < B2) ? C - i2 : B2;
     {  // transposed tf32 hi/lo pair of U[0 : i2 + nb2, i2 : i2 + nb2] for the contractions of this outer block
-      dim3 grid(nb2 / 32, (i2 + nb2) / 32), blk(32, 32);
+      dim3 grid(nb2 / 32, ceil_div(i2 + nb2, 128)), blk(32, 8);
       split_panel_t_kernel<<<grid, blk, 0, s>>>(U, C, i2, i2 + nb2, sK, sC, Phi, Plo, (int64_t)C);
       GPTQ_LAUNCH_CHECK();
     }
