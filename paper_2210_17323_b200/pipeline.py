@@ -142,7 +142,7 @@ class HostLayerSolver:
     (buffers are allocated once, for the shapes given, and reused by every solve()).
     """
 
-    def __init__(self, shapes: Sequence[tuple], grids: Sequence[tuple], block=128, damp=0.01, chunk_bytes=2 << 30, device=None):
+    def __init__(self, shapes: Sequence[tuple], grids: Sequence[tuple], block=128, damp=0.01, chunk_bytes=4 << 30, device=None):
         """shapes: (R, C, n_tokens) per layer; grids: (bits, group_size, sym) per grid."""
         dev = torch.device("cuda", torch.cuda.current_device()) if device is None else device
         self.grids, self.block, self.damp = list(grids), block, damp
@@ -150,9 +150,16 @@ class HostLayerSolver:
         self.copy_stream = torch.cuda.Stream(device=dev)
         self.main = torch.cuda.Stream(device=dev)
         self.state = []
-        for (R, C, n) in shapes:
-            ct = max(64, (chunk_bytes // (2 * C)) // 64 * 64)
-            chunks = [(t0, min(n, t0 + ct)) for t0 in range(0, n, ct)]
+        for li, (R, C, n) in enumerate(shapes):
+            # token chunks of about chunk_bytes; the layer whose activations cross first starts with two short chunks
+            # (1/8 and 1/2 of a chunk) so that its Hessian is under way after a few tens of milliseconds
+            sizes = ([chunk_bytes // 8, chunk_bytes // 2] if li == self.order[0] else []) + [chunk_bytes]
+            chunks, t0 = [], 0
+            while t0 < n:
+                cb = sizes[min(len(chunks), len(sizes) - 1)]
+                ct = max(64, (cb // (2 * C)) // 64 * 64)
+                chunks.append((t0, min(n, t0 + ct)))
+                t0 += ct
             ws_bytes = max([256, B.gptq_hessian_workspace_bytes(C, n), B.gptq_prepare_hinv_workspace_bytes(C)] +
                            [B.gptq_quantize_workspace_bytes(R, C, b, g, block) for (b, g, _) in self.grids])
             outs = []
