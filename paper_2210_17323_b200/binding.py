@@ -48,6 +48,8 @@ def _load():
     lib.gptq_prepare_hinv_workspace_bytes.argtypes = [c.c_int]
     lib.gptq_prepare_hinv.restype = c.c_int
     lib.gptq_prepare_hinv.argtypes = [c.c_void_p, c.c_float, c.c_int, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
+    lib.gptq_prepare_factor.restype = c.c_int
+    lib.gptq_prepare_factor.argtypes = lib.gptq_prepare_hinv.argtypes
     lib.gptq_prepare_hinv_static.restype = c.c_int
     lib.gptq_prepare_hinv_static.argtypes = [c.c_void_p, c.c_float, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p]
     lib.gptq_quantize_workspace_bytes.restype = c.c_size_t
@@ -56,6 +58,8 @@ def _load():
     lib.gptq_quantize_layer.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_int, c.c_int, c.c_int,
                                         c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
                                         c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
+    lib.gptq_quantize_layer_factor.restype = c.c_int
+    lib.gptq_quantize_layer_factor.argtypes = lib.gptq_quantize_layer.argtypes
     lib.gptq_set_stage3_variant.restype = c.c_int
     lib.gptq_set_stage3_variant.argtypes = [c.c_int]
     lib.gptq_solve_layer_host_workspace_bytes.restype = c.c_size_t
@@ -156,8 +160,10 @@ def gptq_hessian_accumulate(H, X, n_tokens=None, ws=None, dev_info=None, stream=
         return H
 
 
-def gptq_prepare_hinv(H, damp=0.01, U=None, ws=None, dev_info=None, stream=None):
-    """U = Cholesky((H + damp*mean(diag H) I)^-1)^T.  Returns (U, dev_info); dev_info is read by the caller after a sync."""
+def gptq_prepare_hinv(H, damp=0.01, U=None, ws=None, dev_info=None, stream=None, factor=False):
+    """U = Cholesky((H + damp*mean(diag H) I)^-1)^T.  Returns (U, dev_info); dev_info is read by the caller after a sync.
+    factor=True calls gptq_prepare_factor instead: the result holds U on its diagonal blocks of 1024 columns and the
+    upper factor of the damped H above them, the input of gptq_quantize_layer(..., factor=True)."""
     with _alloc_on(stream):
         _check(H, torch.float32, "H")
         C = H.shape[0]
@@ -165,7 +171,7 @@ def gptq_prepare_hinv(H, damp=0.01, U=None, ws=None, dev_info=None, stream=None)
         _check(U, torch.float32, "U")
         dev_info = torch.zeros(2, dtype=torch.int32, device=H.device) if dev_info is None else dev_info
         ws = _ws(_lib.gptq_prepare_hinv_workspace_bytes(C), H.device, ws)
-        st = _lib.gptq_prepare_hinv(H.data_ptr(), float(damp), C, U.data_ptr(), ws.data_ptr(), ws.numel(),
+        st = (_lib.gptq_prepare_factor if factor else _lib.gptq_prepare_hinv)(H.data_ptr(), float(damp), C, U.data_ptr(), ws.data_ptr(), ws.numel(),
                                     dev_info.data_ptr(), _stream_ptr(stream))
         if st != OK:
             raise GptqError(st, "gptq_prepare_hinv")
@@ -201,8 +207,10 @@ def _grid_flags(sym, scale_fp16):
     return (GRID_SYMMETRIC if sym else 0) | (GRID_FP16_SCALES if scale_fp16 else 0)
 
 
-def gptq_quantize_layer(W, U, bits, group_size=0, sym=False, block=128, ws=None, dev_info=None, stream=None, scale_fp16=False):
-    """Algorithm 1 on fp16 W (R x C) with U from gptq_prepare_hinv.
+def gptq_quantize_layer(W, U, bits, group_size=0, sym=False, block=128, ws=None, dev_info=None, stream=None, scale_fp16=False,
+                        factor=False):
+    """Algorithm 1 on fp16 W (R x C) with U from gptq_prepare_hinv (factor=True: gptq_quantize_layer_factor on the
+    output of gptq_prepare_hinv(..., factor=True)).
     Returns dict(qweight uint32 [R, C*f/32] (as int32 tensor), scales [R,G], zeros [R,G], loss double[1], dev_info)."""
     with _alloc_on(stream):
         _check(W, torch.float16, "W")
@@ -217,7 +225,7 @@ def gptq_quantize_layer(W, U, bits, group_size=0, sym=False, block=128, ws=None,
         loss = torch.zeros(1, dtype=torch.float64, device=dev)
         dev_info = torch.zeros(2, dtype=torch.int32, device=dev) if dev_info is None else dev_info
         ws = _ws(_lib.gptq_quantize_workspace_bytes(R, C, bits, group_size, block), dev, ws)
-        st = _lib.gptq_quantize_layer(W.data_ptr(), U.data_ptr(), R, C, bits, group_size, _grid_flags(sym, scale_fp16), block,
+        st = (_lib.gptq_quantize_layer_factor if factor else _lib.gptq_quantize_layer)(W.data_ptr(), U.data_ptr(), R, C, bits, group_size, _grid_flags(sym, scale_fp16), block,
                                       qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), loss.data_ptr(),
                                       ws.data_ptr(), ws.numel(), dev_info.data_ptr(), _stream_ptr(stream))
         if st != OK:

@@ -471,9 +471,12 @@ gptq_status_t launch_split_scaled(const float* src, int64_t ld_src, int rows, in
 }  // namespace
 }  // namespace gptq
 
-extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, float* U,
-                                           void* ws, size_t ws_bytes, int* dev_info, void* stream) {
-  using namespace gptq;
+namespace gptq {
+namespace {
+// Both forms of stage 2: the whole of it (U = U~^-1), or phase 1 alone (factor_only: U~ above the diagonal blocks of
+// 1024 columns, the inverses of U~'s diagonal blocks -- which are U's diagonal blocks -- on them).
+gptq_status_t prepare_impl(const float* H, float damp, int C, float* U, void* ws, size_t ws_bytes, int* dev_info,
+                           void* stream, bool factor_only) {
   if (!H || !U || !dev_info || C <= 0 || C % 32 != 0 || !(damp >= 0.f)) return GPTQ_ERR_INVALID_ARG;
   // U == H is allowed: lambda is taken from H's diagonal first, then every element of U is written from the element
   // of H at the same position by the same thread.
@@ -631,6 +634,7 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
     if (st == GPTQ_OK && (j1 != cudaSuccess || j2 != cudaSuccess || j3 != cudaSuccess || j4 != cudaSuccess)) st = GPTQ_ERR_CUDA;
   }
   if (st != GPTQ_OK) return st;
+  if (factor_only) return GPTQ_OK;
 
   // Phase 2: U = U~^-1, outer panel by outer panel, in place.  The diagonal blocks are already inverted;
   // rows above them: U[0:j0, J] = -U[0:j0, 0:j0] * (U~[0:j0, J] * V_JJ).
@@ -669,6 +673,18 @@ extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, fl
     }
   }
   return GPTQ_OK;
+}
+}  // namespace
+}  // namespace gptq
+
+extern "C" gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, float* U,
+                                           void* ws, size_t ws_bytes, int* dev_info, void* stream) {
+  return gptq::prepare_impl(H, damp, C, U, ws, ws_bytes, dev_info, stream, false);
+}
+
+extern "C" gptq_status_t gptq_prepare_factor(const float* H, float damp, int C, float* F,
+                                             void* ws, size_t ws_bytes, int* dev_info, void* stream) {
+  return gptq::prepare_impl(H, damp, C, F, ws, ws_bytes, dev_info, stream, true);
 }
 
 // ------------------------------------------------------------------------------------------------

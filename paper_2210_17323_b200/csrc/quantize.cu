@@ -117,7 +117,7 @@ __global__ void wblk_from_w16_kernel(const __half* __restrict__ W, int R, int C,
 __global__ void __launch_bounds__(256)
 wblk_stripe_major_kernel(const __half* __restrict__ W, int R, int C, int i2,
                          const float* __restrict__ D, int64_t ldd,
-                         const float* __restrict__ sEinv, const float* __restrict__ sCinv,
+                         const float* __restrict__ sEinv, const float* __restrict__ sCinv, double sign,
                          double* __restrict__ Wblk, int64_t ldw) {
   __shared__ float t[128][33];
   __shared__ float d[128][33];
@@ -140,7 +140,7 @@ wblk_stripe_major_kernel(const __half* __restrict__ W, int R, int C, int i2,
       const int rr = tx + 32 * q, r = r0 + rr;
       if (r < R) {
         double w = (double)t[rr][cc];
-        if (D != nullptr) w -= (double)d[rr][cc] * (double)sEinv[r] * sc;
+        if (D != nullptr) w += sign * ((double)d[rr][cc] * (double)sEinv[r] * sc);
         out[(int64_t)cc * 128 + rr] = w;
       }
     }
@@ -359,20 +359,24 @@ __global__ void kscale_kernel(const float* __restrict__ U, int C, float* __restr
   sK[k] = pow2_floor(U[(int64_t)k * C + k]);
   colmax[k] = 0u;
 }
-// colmax[c] = max over rows k <= c of |U[k][c]| / sK[k]   (bit pattern of a non-negative float: ordered as integers)
-__global__ void colmax_kernel(const float* __restrict__ U, int C, const float* __restrict__ sK, uint32_t* __restrict__ colmax) {
+// colmax[c] = max over rows k <= c of |U[k][c]| / sK[k]   (bit pattern of a non-negative float: ordered as integers).
+// Factor form (fblock > 0; U then holds U on its diagonal blocks of fblock columns and the factor U~ above them):
+// colmax covers the rows of c's own diagonal block only, and colmax2[c] = max over the rows above that block of |U~[k][c]|.
+__global__ void colmax_kernel(const float* __restrict__ U, int C, const float* __restrict__ sK, uint32_t* __restrict__ colmax,
+                              int fblock, uint32_t* __restrict__ colmax2) {
   __shared__ float red[8][33];
   const int c = blockIdx.x * 32 + threadIdx.x, r0 = blockIdx.y * 256;
   if (r0 > blockIdx.x * 32 + 31) return;               // block wholly below the diagonal
+  const bool above = fblock > 0 && r0 < (blockIdx.x * 32) / fblock * fblock;   // (256 divides fblock: uniform over the CTA)
   float m = 0.f;
   for (int r = r0 + threadIdx.y; r < min(C, r0 + 256); r += 8)
-    if (r <= c) m = fmaxf(m, fabsf(U[(int64_t)r * C + c]) / sK[r]);
+    if (r <= c) m = fmaxf(m, above ? fabsf(U[(int64_t)r * C + c]) : fabsf(U[(int64_t)r * C + c]) / sK[r]);
   red[threadIdx.y][threadIdx.x] = m;
   __syncthreads();
   if (threadIdx.y == 0) {
 #pragma unroll
     for (int y = 1; y < 8; ++y) m = fmaxf(m, red[y][threadIdx.x]);
-    if (m > 0.f && isfinite(m)) atomicMax(colmax + c, __float_as_uint(m));
+    if (m > 0.f && isfinite(m)) atomicMax((above ? colmax2 : colmax) + c, __float_as_uint(m));
   }
 }
 // sC[c] = power of two that brings the column's largest scaled entry just below 2^13; sCinv = 1 / sC
@@ -408,7 +412,7 @@ __global__ void rowscale_kernel(const __half* __restrict__ W, int R, int C, floa
 // column 256 consecutive bytes of each output written as half2 pairs.  grid (nb2 / 32, rows / 128 rounded up), block (32, 8).
 __global__ void __launch_bounds__(256)
 split_panel_t_kernel(const float* __restrict__ U, int C, int i2, int rows,
-                     const float* __restrict__ sK, const float* __restrict__ sC,
+                     const float* __restrict__ sK, const float* __restrict__ sC, const float* __restrict__ sC2,
                      __half* __restrict__ Phi, __half* __restrict__ Plo, int64_t ldp) {
   __shared__ float t[128][33];
   const int r0 = blockIdx.y * 128, c0 = blockIdx.x * 32;
@@ -416,13 +420,16 @@ split_panel_t_kernel(const float* __restrict__ U, int C, int i2, int rows,
 #pragma unroll
   for (int k = 0; k < 16; ++k) {
     const int rr = ty + 8 * k, r = r0 + rr;
-    t[rr][tx] = r < rows ? U[(int64_t)r * C + i2 + c0 + tx] / sK[r] : 0.f;
+    // factor form (sC2 != nullptr): the rows above the outer block hold the factor U~, scaled per column only
+    const bool above = sC2 != nullptr && r < i2;
+    t[rr][tx] = r < rows ? (above ? U[(int64_t)r * C + i2 + c0 + tx] : U[(int64_t)r * C + i2 + c0 + tx] / sK[r]) : 0.f;
   }
   __syncthreads();
+  const bool above_blk = sC2 != nullptr && r0 < i2;          // (i2 is a multiple of 128: uniform over the CTA)
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const int cc = ty + 8 * k;
-    const float sc = sC[i2 + c0 + cc];
+    const float sc = above_blk ? sC2[i2 + c0 + cc] : sC[i2 + c0 + cc];
     const int64_t o = (int64_t)(c0 + cc) * ldp + r0;
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
@@ -436,6 +443,33 @@ split_panel_t_kernel(const float* __restrict__ U, int C, int i2, int rows,
       *reinterpret_cast<__half2*>(Plo + o + rr) = __halves2half2(l0, l1);
     }
   }
+}
+
+// Factor form: the fp32 sums D = (R U~[before, blk]) sE[row] sC2[col] of the first contraction become the left operand
+// of the second one, D' = D sK[col] / sC2[col] (the size of a scaled weight correction), as an fp16 hi / lo pair.
+__global__ void split_dsum_kernel(const float* __restrict__ D, int64_t ldd, int R, int nb2, int i2,
+                                  const float* __restrict__ sK, const float* __restrict__ sC2inv,
+                                  __half* __restrict__ Dhi, __half* __restrict__ Dlo, int* dev_info) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;       // one thread: 8 consecutive columns
+  const int per_row = nb2 / 8;
+  if (idx >= (int64_t)R * per_row) return;
+  const int r = (int)(idx / per_row), c = (int)(idx % per_row) * 8;
+  const float4 a = *reinterpret_cast<const float4*>(D + (int64_t)r * ldd + c);
+  const float4 b = *reinterpret_cast<const float4*>(D + (int64_t)r * ldd + c + 4);
+  const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+  uint32_t hw[4], lw[4];
+  bool sat = false;
+#pragma unroll
+  for (int u = 0; u < 8; u += 2) {
+    __half h0, l0, h1, l1;
+    f16x3::split_f16(v[u] * (sK[i2 + c + u] * sC2inv[i2 + c + u]), h0, l0, sat);
+    f16x3::split_f16(v[u + 1] * (sK[i2 + c + u + 1] * sC2inv[i2 + c + u + 1]), h1, l1, sat);
+    hw[u >> 1] = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
+    lw[u >> 1] = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
+  }
+  *reinterpret_cast<uint4*>(Dhi + (int64_t)r * ldd + c) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+  *reinterpret_cast<uint4*>(Dlo + (int64_t)r * ldd + c) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+  if (sat) report_error(dev_info, GPTQ_ERR_NONFINITE, r);
 }
 
 // ---- contraction epilogue (one thread: one row, 32 consecutive columns of a partial sum) --------
@@ -507,14 +541,21 @@ extern "C" size_t gptq_quantize_workspace_bytes(int R, int C, int bits, int grou
   w.take<float>((size_t)R);                                       // sE
   w.take<float>((size_t)R);                                       // 1 / sE
   w.take<float>((size_t)R * outer_block(C, group_size, block));   // scaled fp32 sums of the lazy update of the outer block
+  w.take<uint32_t>((size_t)C);                                    // factor form: column maxima of U~ above the diagonal blocks,
+  w.take<float>((size_t)C);                                       //   sC2,
+  w.take<float>((size_t)C);                                       //   1 / sC2,
+  w.take<__half>((size_t)R * outer_block(C, group_size, block));  //   left operand of the second contraction, high parts
+  w.take<__half>((size_t)R * outer_block(C, group_size, block));  //   remainders
   return w.off;
 }
 
-extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U, int R, int C,
-                                             int bits, int group_size, int sym, int block,
-                                             uint32_t* qweight, float* scales, float* zeros, double* loss,
-                                             void* ws, size_t ws_bytes, int* dev_info, void* stream) {
-  using namespace gptq;
+namespace gptq {
+namespace {
+// factor: U holds gptq_prepare_factor's output (U on the diagonal blocks of 1024 columns, the factor U~ above them)
+gptq_status_t quantize_impl(const void* W_fp16, const float* U, int R, int C,
+                            int bits, int group_size, int sym, int block,
+                            uint32_t* qweight, float* scales, float* zeros, double* loss,
+                            void* ws, size_t ws_bytes, int* dev_info, void* stream, bool factor) {
   if (!W_fp16 || !U || !qweight || !scales || !zeros || !loss || !dev_info || R <= 0 || C <= 0 || C % 32 != 0)
     return GPTQ_ERR_INVALID_ARG;
   if (!aligned_to(W_fp16, 16) || !aligned_to(U, 16)) return GPTQ_ERR_INVALID_ARG;
@@ -547,6 +588,11 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   float* sE = w.take<float>((size_t)R);
   float* sEinv = w.take<float>((size_t)R);
   float* Dsum = w.take<float>((size_t)R * B2);
+  uint32_t* colmax2 = w.take<uint32_t>((size_t)C);
+  float* sC2 = w.take<float>((size_t)C);
+  float* sC2inv = w.take<float>((size_t)C);
+  __half* Dhi = w.take<__half>((size_t)R * B2);
+  __half* Dlo = w.take<__half>((size_t)R * B2);
   const int64_t ldw = B2;
   GridSpec gs{bits == GPTQ_BITS_TERNARY ? 2 : (1 << bits) - 1, ((sym & GPTQ_GRID_SYMMETRIC) != 0 || bits == GPTQ_BITS_TERNARY) ? 1 : 0,
               (sym & GPTQ_GRID_FP16_SCALES) ? 1 : 0};
@@ -561,13 +607,18 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   // power-of-two scales of the fp16 operand pairs: per contraction index (from U's diagonal), per column of U, per row of W
   kscale_kernel<<<ceil_div(C, 256), 256, 0, s>>>(U, C, sK, colmax);
   GPTQ_LAUNCH_CHECK();
+  if (factor) GPTQ_CUDA_TRY(cudaMemsetAsync(colmax2, 0, (size_t)C * sizeof(uint32_t), s));
   {
     dim3 grid(C / 32, ceil_div(C, 256)), blk(32, 8);
-    colmax_kernel<<<grid, blk, 0, s>>>(U, C, sK, colmax);
+    colmax_kernel<<<grid, blk, 0, s>>>(U, C, sK, colmax, factor ? GPTQ_FACTOR_BLOCK : 0, colmax2);
     GPTQ_LAUNCH_CHECK();
   }
   cscale_kernel<<<ceil_div(C, 256), 256, 0, s>>>(colmax, C, sC, sCinv);
   GPTQ_LAUNCH_CHECK();
+  if (factor) {
+    cscale_kernel<<<ceil_div(C, 256), 256, 0, s>>>(colmax2, C, sC2, sC2inv);
+    GPTQ_LAUNCH_CHECK();
+  }
   rowscale_kernel<<<ceil_div(R, 8), 256, 0, s>>>(W, R, C, sE, sEinv);
   GPTQ_LAUNCH_CHECK();
   auto inblock_smem = [&](int B) { return (size_t)((size_t)B * kLDS + (size_t)kSB * B + kSB) * sizeof(double) + (size_t)(kSB * kRPB + kSB) * sizeof(float); };
@@ -576,14 +627,16 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
   // form of the loops inside an outer block (see gptq_set_stage3_variant)
   // A block wider than the row-stripe kernel's 128 columns (256) is run there as 128-column inner blocks: the same updates
   // in the same column order, regrouped (Section 3, Step 2) -- groups still nest with 128 whenever they nest with 256.
-  const bool stripe = g_stage3_variant.load(std::memory_order_relaxed) == 1 && B2 <= kStripeMaxNb2 &&
+  const bool stripe = (g_stage3_variant.load(std::memory_order_relaxed) == 1 || factor) && B2 <= kStripeMaxNb2 &&
                       (block <= kStripeMaxB || block % kStripeMaxB == 0);
   const int stripe_block = block <= kStripeMaxB ? block : kStripeMaxB;
+  // the factor form rests on the outer blocks being the factorisation's diagonal blocks, and runs in the row-stripe form only
+  if (factor && C > GPTQ_FACTOR_BLOCK && (!stripe || B2 != GPTQ_FACTOR_BLOCK)) return GPTQ_ERR_UNSUPPORTED;
   for (int i2 = 0; i2 < C; i2 += B2) {
     const int nb2 = (C - i2 < B2) ? C - i2 : B2;
     {  // transposed tf32 hi/lo pair of U[0 : i2 + nb2, i2 : i2 + nb2] for the contractions of this outer block
       dim3 grid(nb2 / 32, ceil_div(i2 + nb2, 128)), blk(32, 8);
-      split_panel_t_kernel<<<grid, blk, 0, s>>>(U, C, i2, i2 + nb2, sK, sC, Phi, Plo, (int64_t)C);
+      split_panel_t_kernel<<<grid, blk, 0, s>>>(U, C, i2, i2 + nb2, sK, sC, factor ? sC2 : nullptr, Phi, Plo, (int64_t)C);
       GPTQ_LAUNCH_CHECK();
     }
     // working weights of the outer block: original weights minus all updates from columns < i2
@@ -598,9 +651,21 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
         if (st != GPTQ_OK) return st;
         st = f16x3::launch<false, false>(A, Bop, R, nb2, f16x3::EpiTileAddF32{R, nb2, 1.f, nullptr, nullptr}, dev_info, s, 0, &out);
         if (st != GPTQ_OK) return st;
+        if (factor) {
+          // A holds the plain residuals R' and the panel rows above the block hold U~: the sums are (R U~[before, blk]);
+          // times the block's own U (the rows of the panel inside the block) they are the correction of the block
+          const int64_t n8 = (int64_t)R * (nb2 / 8);
+          split_dsum_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, s>>>(Dsum, B2, R, nb2, i2, sK, sC2inv, Dhi, Dlo, dev_info);
+          GPTQ_LAUNCH_CHECK();
+          GPTQ_CUDA_TRY(cudaMemsetAsync(Dsum, 0, (size_t)R * B2 * sizeof(float), s));
+          f16x3::Operand A2{Dhi, Dlo, R, nb2, B2}, B2op{Phi + i2, Plo + i2, nb2, nb2, C};
+          st = f16x3::launch<false, false>(A2, B2op, R, nb2, f16x3::EpiTileAddF32{R, nb2, 1.f, nullptr, nullptr}, dev_info, s, 0, &out);
+          if (st != GPTQ_OK) return st;
+        }
       }
       dim3 grid(nb2 / 32, ceil_div(R, 128)), blk(32, 8);
-      wblk_stripe_major_kernel<<<grid, blk, 0, s>>>(W, R, C, i2, i2 > 0 ? Dsum : nullptr, B2, sEinv, sCinv, Wblk, ldw);
+      wblk_stripe_major_kernel<<<grid, blk, 0, s>>>(W, R, C, i2, i2 > 0 ? Dsum : nullptr, B2, sEinv, sCinv, factor ? 1.0 : -1.0,
+                                                    Wblk, ldw);
       GPTQ_LAUNCH_CHECK();
     } else {
       int64_t total = (int64_t)R * nb2;
@@ -615,7 +680,7 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
     if (stripe) {
       // row-stripe form: every inner block of this outer block in one launch
       StripeArgs a{Wblk, ldw, nb2, U, C, i2, stripe_block, R, gs, g, scales, zeros, G, Ehi, Elo, Phi, Plo, (int64_t)C,
-                   sK, sE, sEinv, sCinv, codes, loss, dev_info};
+                   sK, sE, sEinv, sCinv, codes, loss, dev_info, factor ? W : nullptr};
       gptq_status_t st = launch_stripe(a, Phi, Plo, s);
       if (st != GPTQ_OK) return st;
       continue;
@@ -648,6 +713,24 @@ extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U,
     GPTQ_LAUNCH_CHECK();
   }
   return GPTQ_OK;
+}
+}  // namespace
+}  // namespace gptq
+
+extern "C" gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U, int R, int C,
+                                             int bits, int group_size, int sym, int block,
+                                             uint32_t* qweight, float* scales, float* zeros, double* loss,
+                                             void* ws, size_t ws_bytes, int* dev_info, void* stream) {
+  return gptq::quantize_impl(W_fp16, U, R, C, bits, group_size, sym, block, qweight, scales, zeros, loss, ws, ws_bytes,
+                             dev_info, stream, false);
+}
+
+extern "C" gptq_status_t gptq_quantize_layer_factor(const void* W_fp16, const float* F, int R, int C,
+                                                    int bits, int group_size, int sym, int block,
+                                                    uint32_t* qweight, float* scales, float* zeros, double* loss,
+                                                    void* ws, size_t ws_bytes, int* dev_info, void* stream) {
+  return gptq::quantize_impl(W_fp16, F, R, C, bits, group_size, sym, block, qweight, scales, zeros, loss, ws, ws_bytes,
+                             dev_info, stream, true);
 }
 
 namespace gptq {

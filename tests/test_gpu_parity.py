@@ -599,3 +599,50 @@ def test_two_hessian_launches_side_by_side_on_two_streams(B):
         Xd = X.double()
         exact = (6.0 * (Xd.T @ Xd)).cpu().numpy()
         assert np.array_equal(H.cpu().numpy().astype(np.float64), exact)
+
+
+# ------------------------------------------------------------------ factor form (stage 2 without the inverse)
+def test_prepare_factor_holds_the_factor_above_and_u_on_the_diagonal_blocks(B):
+    """gptq_prepare_factor against the oracle: diagonal blocks of 1024 columns = the blocks of U, blocks above them = the
+    blocks of U^-1 (the upper factor of the damped Hessian)."""
+    C = 2304
+    L = _layer(8, C, 2 * C + 100)
+    H64 = O.hessian_accumulate(np.zeros((C, C)), L.x_bits())
+    F, info = B.gptq_prepare_hinv(torch.from_numpy(H64.astype(np.float32)).cuda(), 0.01, factor=True)
+    torch.cuda.synchronize()
+    assert info.tolist() == [0, 0]
+    Fg = F.cpu().numpy().astype(np.float64)
+    U = O.cholesky_inverse_upper(O.dampen(H64.astype(np.float32).astype(np.float64), 0.01)[0])
+    Ut = np.linalg.inv(U)
+    assert np.array_equal(Fg, np.triu(Fg))
+    for j0 in range(0, C, 1024):
+        j1 = min(C, j0 + 1024)
+        assert rel_fro(Fg[j0:j1, j0:j1], U[j0:j1, j0:j1]) <= TOL_U_FRO
+        if j0 > 0:
+            assert rel_fro(Fg[:j0, j0:j1], Ut[:j0, j0:j1]) <= TOL_U_FRO
+
+
+@pytest.mark.parametrize("R,C,bits,group,block", [(200, 2304, 4, 0, 128), (130, 3072, 3, 128, 128), (96, 2048, 2, 32, 64),
+                                                  (64, 2304, O.BITS_TERNARY, 8, 32), (100, 2048, 4, 1024, 256), (70, 768, 4, 0, 128)])
+def test_factor_form_matches_the_oracle(B, R, C, bits, group, block):
+    """Stages 2 and 3 in the factor form (no inverse; plain residuals fed back through the factor across blocks of 1024
+    columns) against the oracle, which runs Algorithm 1 as written with U."""
+    L = _layer(R, C, 2 * C + 64, cfg=9)
+    xb, W16 = L.x_bits(), L.w()
+    ref = O.solve_layer(W16, xb, bits, group, False, block, 0.01)
+    H = torch.from_numpy(ref["H"].astype(np.float32)).cuda()
+    F, info = B.gptq_prepare_hinv(H, 0.01, factor=True)
+    out = B.gptq_quantize_layer(torch.from_numpy(W16).cuda(), F, bits, group, False, block, factor=True)
+    torch.cuda.synchronize()
+    assert info.tolist() == [0, 0] and out["dev_info"].tolist() == [0, 0]
+    gpu = dict(qweight=out["qweight"].cpu().numpy(), scales=out["scales"].cpu().numpy(), zeros=out["zeros"].cpu().numpy(),
+               loss=out["loss"].item())
+    check_quantize_outputs(gpu, ref, W16, bits, C, ref["H"])
+
+
+def test_factor_form_rejects_blockings_it_cannot_run(B):
+    W = torch.zeros((32, 2304), dtype=torch.float16, device="cuda")
+    F = torch.eye(2304, device="cuda")
+    with pytest.raises(B.GptqError) as e:
+        B.gptq_quantize_layer(W, F, 4, 0, False, 96, factor=True)      # outer blocks of 960 columns
+    assert e.value.status == B.ERR_UNSUPPORTED
