@@ -269,14 +269,18 @@ def run_gpu(args, wl):
     torch.cuda.synchronize()
 
     stage_events = []                             # (layer idx, events) of the timed steps
+    factor = _factor_form(args, wl)
+    for st in state:                              # per layer: the factor form where it pays (wide layers), else the inverse form
+        st["factor"] = factor and B.factor_form_pays(st["L"].R, st["L"].C, len(wl.grids))
 
     graphs = []                                   # per layer: CUDA graphs of the three stages (launch-bound inner loops)
 
     def stage_fns(st):
         return ([("H", lambda: (st["H"].zero_(), B.gptq_hessian_accumulate(st["H"], st["X"], ws=st["ws"]))),
-                 ("U", lambda: B.gptq_prepare_hinv(st["H"], wl.damp, U=st["U"], ws=st["ws"], dev_info=st["info"]))] +
+                 ("U", lambda: B.gptq_prepare_hinv(st["H"], wl.damp, U=st["U"], ws=st["ws"], dev_info=st["info"],
+                                                   factor=factor and st["factor"]))] +
                 [(f"Q{gi}", (lambda gi=gi, g=g: st["out"].__setitem__(gi, B.gptq_quantize_layer(
-                    st["W"], st["U"], g.bits, g.group_size, g.sym, wl.block, ws=st["ws"]))))
+                    st["W"], st["U"], g.bits, g.group_size, g.sym, wl.block, ws=st["ws"], factor=factor and st["factor"]))))
                  for gi, g in enumerate(wl.grids)])
 
     def run_stage(li, name, fn):
@@ -405,6 +409,9 @@ def run_gpu(args, wl):
     # roofline of the dominant kernel.  Hessian: algorithmic flops C (C + 1) m per launch (symmetric half).
     hess_flops = sum(L.C * (L.C + 1) * L.n_tokens for L in layers)
     upd_flops = sum(2 * L.R * (L.C * L.C - L.C * wl.block) / 2 * n_grids for L in layers)   # lazy updates, R (C^2 - C B)
+    uses_factor = {st["L"].name: st["factor"] for st in state}
+    if factor:      # + per outer block of 1024 columns the product with the block's own U (triangular: half of R 1024^2 MACs)
+        upd_flops += sum(L.R * 1024 * max(0, L.C - 1024) * n_grids for L in layers if uses_factor[L.name])
     # the stage sums overlap one another in the overlapped schedule, so the dominant kernel is chosen against the step
     if tot["hessian_ms"] >= tot["quantize_ms"] or tot["hessian_ms"] >= 0.3 * ms_per_step:
         ach = hess_flops / (tot["hessian_ms"] * 1e-3) / 1e12
@@ -432,7 +439,7 @@ def run_gpu(args, wl):
     # every stage against the roofline that bounds it (CUDA events around the stage's launches; in the overlapped
     # schedules the stages of different layers run side by side, so these are in-context rates)
     f16_peak = peaks["bf16_sustained"]           # kind::f16 instructions run at the bf16 rate
-    fac_flops = sum(2.0 * L.C ** 3 / 3.0 for L in layers)
+    fac_flops = sum((1.0 if uses_factor[L.name] else 2.0) * L.C ** 3 / 3.0 for L in layers)
     hess_ach = hess_flops / (tot["hessian_ms"] * 1e-3) / 1e12
     fac_ach = fac_flops / (tot["hinv_ms"] * 1e-3) / 1e12
     upd_ach = upd_flops / (tot["quantize_ms"] * 1e-3) / 1e12
@@ -441,11 +448,14 @@ def run_gpu(args, wl):
              unit="TFLOP/s", frac=hess_ach / peaks["bf16_sustained"], flops="algorithmic C (C + 1) m"),
         dict(stage="prepare_hinv", bound="tensor", dtype="fp16 pairs, 3 products per term", achieved=fac_ach, executed=3 * fac_ach,
              peak=f16_peak, unit="TFLOP/s", frac=3 * fac_ach / f16_peak, useful_frac=fac_ach / f16_peak,
-             flops="useful 2 C^3 / 3; executed = 3 x (hi*hi + hi*lo + lo*hi); the serial 128 x 128 diagonal-block chain and the "
+             flops=("useful C^3 / 3 for the layers in the factor form (the backwards factorisation alone), 2 C^3 / 3 for the others"
+                    if factor else "useful 2 C^3 / 3") +
+                   "; executed = 3 x (hi*hi + hi*lo + lo*hi); the serial 128 x 128 diagonal-block chain and the "
                    "CUDA-core work inside an outer panel are inside this time"),
         dict(stage="quantize_layer", bound="tensor", dtype="fp16 pairs, 3 products per term", achieved=upd_ach, executed=3 * upd_ach,
              peak=f16_peak, unit="TFLOP/s", frac=3 * upd_ach / f16_peak, useful_frac=upd_ach / f16_peak,
-             flops="useful R (C^2 - C B) per grid (lazy updates); the column chains, packing and grids are inside this time"),
+             flops="useful R (C^2 - C B) per grid (lazy updates)" + (" + R C 1024 (the blocks' own U, factor form)" if factor else "") +
+                   "; the column chains, packing and grids are inside this time"),
     ]
     for r in stage_rooflines:
         r["peak_source"] = f"bf16 sustained, {peaks['source']}"
@@ -457,6 +467,10 @@ def run_gpu(args, wl):
                 config=dict(workload=wl.name, layers=[l.name for l in wl.layers],
                             grids=[dict(bits=g.bits, group_size=g.group_size, sym=g.sym) for g in wl.grids],
                             block=wl.block, damp=wl.damp, calib_tokens=wl.layers[0].n_tokens,
+                            form=("factor where it pays (wide layers): gptq_prepare_factor + gptq_quantize_layer_factor (E = (W - Q) U~; "
+                                  "the factor's inverse is never formed); inverse form for: " +
+                                  (", ".join(n for n, f in uses_factor.items() if not f) or "no layer")) if factor
+                                 else "inverse: gptq_prepare_hinv + gptq_quantize_layer (U = Cholesky(H^-1)^T)",
                             cache="inputs larger than L2 (X >= 0.4 GB per layer); no flush needed",
                             launch="CUDA graphs, one per stage per layer" if graphs else "host-issued launches",
                             schedule={"pipelined": "pipelined: Hessians back to back on one stream, each layer's stages 2-3 on its own "
@@ -630,6 +644,19 @@ def run_block_sweep(args, wl):
     return 0
 
 
+def _factor_form(args, wl):
+    """True if the run uses the factor form: asked for, in the row-stripe form of stage 3, and the workload's block and
+    group sizes give outer blocks of 1024 columns."""
+    if getattr(args, "form", "factor") != "factor" or getattr(args, "stage3_variant", 1) != 1:
+        return False
+    block = getattr(args, "block", None) or wl.block
+    for g in wl.grids:
+        unit = max(g.group_size if g.group_size > 0 else 0, block)
+        if 1024 % unit != 0:
+            return False
+    return True
+
+
 def run_e2e(args, wl, state, device_value):
     """Same metric end to end from HOST buffers through the package's host-input solver: every step, every layer's X and
     W cross from pinned host memory to the device (copies overlapped with the Hessian accumulation and with the other
@@ -644,7 +671,7 @@ def run_e2e(args, wl, state, device_value):
         st["X"] = st["W"] = st["H"] = st["U"] = st["ws"] = None
     state.clear()
     torch.cuda.empty_cache()
-    solver = pipeline.HostLayerSolver(shapes, grids, block=wl.block, damp=wl.damp)
+    solver = pipeline.HostLayerSolver(shapes, grids, block=wl.block, damp=wl.damp, factor=_factor_form(args, wl))
     torch.cuda.synchronize()
     steps = max(1, min(args.steps, 5))      # each step moves every layer's activations across PCIe again (seconds)
     solver.solve(layers)                    # warm-up (kernel attributes, allocator)
@@ -718,7 +745,7 @@ def run_block(args, wl):
     dev = torch.device("cuda", 0)
     g = wl.grids[min(args.grid, len(wl.grids) - 1)]
     groups = P.group_by_shared_input(wl.layers, lambda L: D.fill_x(L, device=dev), lambda L: D.fill_w(L, device=dev))
-    solver = P.BlockSolver(groups, g.bits, g.group_size, g.sym, wl.block, wl.damp)
+    solver = P.BlockSolver(groups, g.bits, g.group_size, g.sym, wl.block, wl.damp, factor=_factor_form(args, wl))
     main = solver.main
     torch.cuda.synchronize()
     graphs = {}
@@ -801,6 +828,11 @@ def main():
                          "one Hessian and one factor")
     ap.add_argument("--grid", type=int, default=0, help="--mode block: index of the workload's grid to run")
     ap.add_argument("--block", type=int, default=None, help="block size B of Algorithm 1 (default: the workload's, 128)")
+    ap.add_argument("--form", default="factor", choices=["factor", "inverse"],
+                    help="factor (default): stage 2 stops after the backwards factorisation and stage 3 feeds the plain residuals "
+                         "back through the factor (gptq_prepare_factor / gptq_quantize_layer_factor: same results, the factor's "
+                         "inverse is never formed); inverse: U = Cholesky(H^-1)^T as Algorithm 1 writes it "
+                         "(gptq_prepare_hinv / gptq_quantize_layer)")
     ap.add_argument("--stage3-variant", type=int, default=1, choices=[0, 1],
                     help="form of the loops inside an outer block: 1 row-stripe kernel (default), 0 one in-block kernel plus one "
                          "small contraction per inner block")

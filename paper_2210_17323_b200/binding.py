@@ -233,6 +233,21 @@ def gptq_quantize_layer(W, U, bits, group_size=0, sym=False, block=128, ws=None,
         return dict(qweight=qweight, scales=scales, zeros=zeros, loss=loss, dev_info=dev_info)
 
 
+def factor_form_supported(C, block, group_sizes=()):
+    """True if gptq_quantize_layer(..., factor=True) can run this layer: outer blocks of 1024 columns."""
+    if C <= 1024:
+        return True
+    return all(1024 % max(block, g if g and g > 0 else 0) == 0 for g in (list(group_sizes) or [0]))
+
+
+def factor_form_pays(R, C, n_grids=1):
+    """Rule of thumb for choosing between the two forms of stages 2 and 3.  The factor form leaves out the second half of
+    stage 2 (about C^3 / 3 multiply-adds, once per layer) and adds, per grid and outer block of 1024 columns, one product of
+    the block's update sums with the block's own U (R * 1024 * C multiply-adds per grid over the layer): it pays for
+    layers that are wide rather than tall."""
+    return C > 1024 and C * C > 3 * 1024 * R * max(1, n_grids)
+
+
 def gptq_set_stage3_variant(variant: int) -> int:
     """1: row-stripe kernel inside an outer block (default); 0: per-inner-block kernels.  Returns the previous value."""
     return int(_lib.gptq_set_stage3_variant(int(variant)))

@@ -53,8 +53,12 @@ def group_by_shared_input(layers: Sequence, x_of, w_of) -> List[InputGroup]:
 class BlockSolver:
     """Holds the buffers, workspaces and streams of one block and enqueues its solve."""
 
-    def __init__(self, groups: Sequence[InputGroup], bits, group_size=0, sym=False, block=128, damp=0.01, scale_fp16=False):
+    def __init__(self, groups: Sequence[InputGroup], bits, group_size=0, sym=False, block=128, damp=0.01, scale_fp16=False,
+                 factor=False):
+        """factor=True: stages 2 and 3 in the factor form (gptq_prepare_factor / gptq_quantize_layer_factor: same results,
+        the factor's inverse is never formed) for the input groups where that is supported and pays."""
         self.bits, self.group_size, self.sym, self.block, self.damp, self.scale_fp16 = bits, group_size, sym, block, damp, scale_fp16
+        self.factor_form = factor
         dev = groups[0].X.device
         # most expensive Hessian first: the longest dependency chain starts earliest
         self.groups = sorted(groups, key=lambda g: -(g.X.shape[1] ** 2) * (g.X.shape[0] + g.X.shape[1]))
@@ -66,7 +70,10 @@ class BlockSolver:
                       info=torch.zeros(2, dtype=torch.int32, device=dev),
                       ws=torch.empty(max(256, B.gptq_hessian_workspace_bytes(C, n), B.gptq_prepare_hinv_workspace_bytes(C)),
                                      dtype=torch.uint8, device=dev),
-                      stream=torch.cuda.Stream(device=dev), members=[])
+                      stream=torch.cuda.Stream(device=dev), members=[],
+                      # the factor form where it pays: the group's members all use the group's one factor
+                      factor_form=bool(factor) and B.factor_form_supported(C, block, [group_size]) and
+                      B.factor_form_pays(sum(m.W.shape[0] for m in g.members), C, 1))
             for m in g.members:
                 R = m.W.shape[0]
                 st["members"].append(dict(m=m, stream=torch.cuda.Stream(device=dev),
@@ -81,11 +88,11 @@ class BlockSolver:
         B.gptq_hessian_accumulate(st["H"], st["g"].X, ws=st["ws"])
 
     def factor(self, st):
-        B.gptq_prepare_hinv(st["H"], self.damp, U=st["U"], ws=st["ws"], dev_info=st["info"])
+        B.gptq_prepare_hinv(st["H"], self.damp, U=st["U"], ws=st["ws"], dev_info=st["info"], factor=st["factor_form"])
 
     def quantize(self, st, ms):
         ms["m"].out = B.gptq_quantize_layer(ms["m"].W, st["U"], self.bits, self.group_size, self.sym, self.block, ws=ms["ws"],
-                                            scale_fp16=self.scale_fp16)
+                                            scale_fp16=self.scale_fp16, factor=st["factor_form"])
 
     def enqueue(self, run=None):
         """Enqueues the whole block.  `run(key, fn)` may replace the plain call of a stage (e.g. by a CUDA-graph
@@ -142,10 +149,12 @@ class HostLayerSolver:
     (buffers are allocated once, for the shapes given, and reused by every solve()).
     """
 
-    def __init__(self, shapes: Sequence[tuple], grids: Sequence[tuple], block=128, damp=0.01, chunk_bytes=4 << 30, device=None):
+    def __init__(self, shapes: Sequence[tuple], grids: Sequence[tuple], block=128, damp=0.01, chunk_bytes=4 << 30, device=None,
+                 factor=False):
         """shapes: (R, C, n_tokens) per layer; grids: (bits, group_size, sym) per grid."""
         dev = torch.device("cuda", torch.cuda.current_device()) if device is None else device
         self.grids, self.block, self.damp = list(grids), block, damp
+        # factor: stages 2 and 3 in the factor form (see BlockSolver) for the layers where it pays
         self.order = sorted(range(len(shapes)), key=lambda i: -(shapes[i][1] ** 2) * (shapes[i][2] + shapes[i][1]))
         self.copy_stream = torch.cuda.Stream(device=dev)
         self.main = torch.cuda.Stream(device=dev)
@@ -171,6 +180,8 @@ class HostLayerSolver:
                                  loss=torch.empty(1, dtype=torch.float64).pin_memory(),
                                  info=torch.empty(2, dtype=torch.int32).pin_memory()))
             self.state.append(dict(R=R, C=C, n=n, chunks=chunks,
+                                   factor=bool(factor) and B.factor_form_pays(R, C, len(self.grids)) and
+                                   B.factor_form_supported(C, block, [g for (_, g, _) in self.grids]),
                                    X=torch.empty((n, C), dtype=torch.bfloat16, device=dev),
                                    W=torch.empty((R, C), dtype=torch.float16, device=dev),
                                    H=torch.empty((C, C), dtype=torch.float32, device=dev),
@@ -216,11 +227,11 @@ class HostLayerSolver:
             s = st["stream"]
             with torch.cuda.stream(s):
                 s.wait_event(h_done); s.wait_event(landed[(li, "W")])
-                B.gptq_prepare_hinv(st["H"], self.damp, U=st["U"], ws=st["ws"], dev_info=st["info_u"])
+                B.gptq_prepare_hinv(st["H"], self.damp, U=st["U"], ws=st["ws"], dev_info=st["info_u"], factor=st["factor"])
                 st["info_host"][:-1].copy_(st["info_h"], non_blocking=True)
                 st["info_host"][-1].copy_(st["info_u"], non_blocking=True)
                 for (b, g, sym), o in zip(self.grids, st["outs"]):
-                    r = B.gptq_quantize_layer(st["W"], st["U"], b, g, sym, self.block, ws=st["ws"])
+                    r = B.gptq_quantize_layer(st["W"], st["U"], b, g, sym, self.block, ws=st["ws"], factor=st["factor"])
                     for k, src in (("qweight", r["qweight"]), ("scales", r["scales"]), ("zeros", r["zeros"]), ("loss", r["loss"]),
                                    ("info", r["dev_info"])):
                         o[k].copy_(src, non_blocking=True)
