@@ -70,10 +70,38 @@ def _solve_gpu(B, D, L, wl, grids, keep_x=False):
     for g in grids:
         o = B.gptq_quantize_layer(W, U, g.bits, g.group_size, g.sym, wl.block)
         outs.append(o)
+    # the same layer in the factor form (stage 2 without the inverse, stage 3 on the factor)
+    F, info_f = B.gptq_prepare_hinv(H, wl.damp, factor=True)
+    outs_f = [B.gptq_quantize_layer(W, F, g.bits, g.group_size, g.sym, wl.block, factor=True) for g in grids]
     torch.cuda.synchronize()
-    assert info_h.tolist()[0] == 0 and info.tolist()[0] == 0
-    assert all(o["dev_info"].tolist()[0] == 0 for o in outs)
-    return dict(H=H, U=U, outs=outs, X=X if keep_x else None)
+    assert info_h.tolist()[0] == 0 and info.tolist()[0] == 0 and info_f.tolist()[0] == 0
+    assert all(o["dev_info"].tolist()[0] == 0 for o in outs + outs_f)
+    _check_factor_against_u(F, U)
+    del F
+    return dict(H=H, U=U, outs=outs, outs_factor=outs_f, X=X if keep_x else None)
+
+
+def _check_factor_against_u(F, U, blk=1024):
+    """gptq_prepare_factor's output against gptq_prepare_hinv's on the device: the same diagonal blocks up to rounding, and for the last
+    block of columns J the identity U[:j0, J] = -U[:j0, :j0] (U~[:j0, J] U_JJ) on a probe vector, in fp64 row chunks."""
+    C = U.shape[0]
+    for j0 in range(0, C, blk):
+        j1 = min(C, j0 + blk)
+        d = (F[j0:j1, j0:j1].double() - U[j0:j1, j0:j1].double()).norm() / U[j0:j1, j0:j1].double().norm()
+        assert d.item() <= 1e-5, (j0, d.item())      # (two runs of the factorisation: their reductions add in different orders)
+    j0 = (C - 1) // blk * blk
+    if j0 == 0:
+        return
+    g = torch.Generator(device="cuda").manual_seed(5)
+    z = torch.randn(C - j0, dtype=torch.float64, device="cuda", generator=g)
+    v = F[:j0, j0:].double() @ (U[j0:, j0:].double() @ z)
+    lhs = U[:j0, j0:].double() @ z
+    rhs = torch.empty_like(lhs)
+    for r0 in range(0, j0, 4096):
+        r1 = min(j0, r0 + 4096)
+        rhs[r0:r1] = -(U[r0:r1, :j0].double() @ v)
+    err = ((lhs - rhs).norm() / lhs.norm()).item()
+    assert err <= 1e-4, err
 
 
 def _gpu_out_rows(o, rows=None):
@@ -82,17 +110,27 @@ def _gpu_out_rows(o, rows=None):
                 zeros=o["zeros"][sl].cpu().numpy(), loss=o["loss"].item())
 
 
-def _check_rows(L, wl, g, U64, o, n_rows, H64=None, seed=7):
-    """Rows are independent sub-problems (Section 2): a sample of them, re-solved by the oracle with the GPU's U."""
+def _check_rows(L, wl, g, U64, o, n_rows, H64=None, seed=7, o_factor=None):
+    """Rows are independent sub-problems (Section 2): a sample of them, re-solved by the oracle with the GPU's U.
+    o_factor: the factor form's outputs for the same layer, checked against the same oracle result."""
     rows = np.sort(np.random.default_rng(seed + L.R).choice(L.R, n_rows, replace=False))
     W16 = L.w(rows=rows)
     ref = O.quantize_layer(W16, U64, g.bits, g.group_size, g.sym, wl.block)
-    gpu = _gpu_out_rows(o, rows)
-    layer_loss = gpu["loss"]
-    gpu["loss"] = ref["loss"]                  # the layer's loss covers all rows: checked below on the sample's share
-    figs = check_quantize_outputs(gpu, ref, W16, g.bits, L.C, H64)
     per_row = ref["loss"] / n_rows
-    assert 0.5 * per_row * L.R <= layer_loss <= 2.0 * per_row * L.R
+    figs = None
+    for out in (o_factor, o):                  # (the figures reported are the last one's: the form Algorithm 1 writes)
+        if out is None:
+            continue
+        gpu = _gpu_out_rows(out, rows)
+        layer_loss = gpu["loss"]
+        gpu["loss"] = ref["loss"]              # the layer's loss covers all rows: checked below on the sample's share
+        f = check_quantize_outputs(gpu, ref, W16, g.bits, L.C, H64)
+        assert 0.5 * per_row * L.R <= layer_loss <= 2.0 * per_row * L.R
+        if out is o_factor:
+            figs_factor = f
+        figs = f
+    if o_factor is not None:
+        figs["identical_factor_form"] = figs_factor["identical"]
     figs["rows"] = int(n_rows)
     return figs
 
@@ -114,9 +152,11 @@ def test_config1_block_end_to_end(B, D):
         h_err = rel_fro(s["H"].cpu().numpy(), H)
         u_err = rel_fro(s["U"].cpu().numpy(), U)
         assert h_err <= TOL_H_FRO and u_err <= TOL_U_FRO, (L.name, h_err, u_err)
-        for g, o in zip(wl.grids, s["outs"]):
+        for g, o, of in zip(wl.grids, s["outs"], s["outs_factor"]):
             ref = O.quantize_layer(W16, U, g.bits, g.group_size, g.sym, wl.block)
+            figs_f = check_quantize_outputs(_gpu_out_rows(of), ref, W16, g.bits, L.C, H)      # the factor form
             figs = check_quantize_outputs(_gpu_out_rows(o), ref, W16, g.bits, L.C, H)
+            figs["identical_factor_form"] = figs_f["identical"]
             figs.update(H_rel_fro=h_err, U_rel_fro=u_err, seconds=round(time.time() - t0, 1))
             FIGURES[f"c1 {L.kind} {L.R}x{L.C} bits={g.bits} end-to-end"] = figs
 
@@ -135,7 +175,7 @@ def test_config2_q_end_to_end_sampled_rows(B, D):
     h_err = rel_fro(s["H"].cpu().numpy(), H)
     u_err = rel_fro(s["U"].cpu().numpy(), U)
     assert h_err <= TOL_H_FRO and u_err <= TOL_U_FRO, (h_err, u_err)
-    figs = _check_rows(L, wl, g, U, s["outs"][0], 64, H)      # the ORACLE's U: end-to-end comparison
+    figs = _check_rows(L, wl, g, U, s["outs"][0], 64, H, o_factor=s["outs_factor"][0])   # the ORACLE's U: end-to-end comparison
     figs.update(H_rel_fro=h_err, U_rel_fro=u_err)
     FIGURES[f"c2 q {L.R}x{L.C} bits={g.bits} g{g.group_size} end-to-end (64 rows)"] = figs
 
@@ -149,8 +189,8 @@ def _stagewise(B, D, cfg, kind, n_rows):
     res, tail = check_factor_on_device(s["H"], s["U"], wl.damp)
     U64 = s["U"].cpu().numpy().astype(np.float64)
     s["H"] = None
-    for g, o in zip(wl.grids, s["outs"]):
-        figs = _check_rows(L, wl, g, U64, o, n_rows)
+    for g, o, of in zip(wl.grids, s["outs"], s["outs_factor"]):
+        figs = _check_rows(L, wl, g, U64, o, n_rows, o_factor=of)
         figs.update(H_sampled_rel_fro=h_fro, U_probe_residual=res, U_tail_rows_err=tail)
         FIGURES[f"c{cfg} {kind} {L.R}x{L.C} bits={g.bits} g{g.group_size} stage-isolated"] = figs
 
