@@ -182,12 +182,19 @@ gptq_status_t solve_layer_host_enqueue(const HostWs& w, StreamGuard& g, cudaStre
     GPTQ_CUDA_TRY(cudaEventRecord(g.freed[b], s));
   }
   GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, g.w_done, 0));
-  st = gptq_prepare_hinv(w.H, damp, C, w.U, w.stage_ws, w.stage_ws_bytes, w.info + 2, s);
+  // Factor form (stage 2 without the inverse; same results) where stage 3 can run it for every grid and it pays: it
+  // leaves out about C^3 / 3 multiply-adds once and adds R * 1024 * C per grid (see gptq_prepare_factor).
+  bool factor = C > GPTQ_FACTOR_BLOCK && block > 0 && block <= 256 && GPTQ_FACTOR_BLOCK % block == 0 &&
+                (double)C * C > 3.0 * GPTQ_FACTOR_BLOCK * (double)R * n_grids;
+  for (int gi = 0; gi < n_grids && factor; ++gi)
+    if (group_size[gi] > block && GPTQ_FACTOR_BLOCK % group_size[gi] != 0) factor = false;
+  st = factor ? gptq_prepare_factor(w.H, damp, C, w.U, w.stage_ws, w.stage_ws_bytes, w.info + 2, s)
+              : gptq_prepare_hinv(w.H, damp, C, w.U, w.stage_ws, w.stage_ws_bytes, w.info + 2, s);
   if (st != GPTQ_OK) return st;
   // one Hessian and one factor serve every grid: quantize and copy back grid after grid (the device output buffers are
   // reused, the stream keeps a grid's copies ahead of the next grid's kernels)
   for (int gi = 0; gi < n_grids; ++gi) {
-    st = gptq_quantize_layer(w.W, w.U, R, C, bits[gi], group_size[gi], sym[gi], block, w.qweight, w.scales, w.zeros, w.loss,
+    st = (factor ? gptq_quantize_layer_factor : gptq_quantize_layer)(w.W, w.U, R, C, bits[gi], group_size[gi], sym[gi], block, w.qweight, w.scales, w.zeros, w.loss,
                              w.stage_ws, w.stage_ws_bytes, w.info + 6, s);
     if (st != GPTQ_OK) return st;
     fold_info_kernel<<<1, 1, 0, s>>>(w.info + 4, w.info + 6);
