@@ -11,6 +11,9 @@
  *   gptq_quantize_layer       Algorithm 1's two loops -> packed codes, scales,
  *                             zeros, loss
  *
+ * Stages 2 and 3 also come as gptq_prepare_factor / gptq_quantize_layer_factor: the same results
+ * without the factor's inverse (a reformulation of Algorithm 1's updates, described at gptq_prepare_factor).
+ *
  * Conventions shared by every call
  *   - Every pointer except `stream` is DEVICE memory owned by the caller
  *     (unless a parameter says "host").  The library allocates no device
