@@ -129,11 +129,13 @@ gptq_status_t gptq_prepare_hinv(const float* H, float damp, int C, float* U,
  * errors, the update rule of Algorithm 1 gives Q + E U = W, i.e. E = R U~ with U~ = U^-1 the upper factor of
  * H~ = U~ U~^T.  For a block J of columns and the columns before it this reads
  *     (working weights of block J when the algorithm reaches it) = W_J + (R_before U~[before, J]) U_JJ,
- * where U_JJ = (U~_JJ)^-1 is the diagonal block of U.  So the solver needs U~ above the diagonal blocks and U on
- * them -- exactly what the backwards factorisation of H~ leaves when it stops before inverting -- and the second half
- * of stage 2 (C^3 / 3 of its 2 C^3 / 3 flops) is not needed.
+ * where U_JJ = (U~_JJ)^-1 is the diagonal block of U.  So the solver needs U on the diagonal blocks and the products
+ * U~[before, J] U_JJ above them -- what the backwards factorisation of H~ leaves when it stops before inverting, plus
+ * one 1024-deep product per block column -- and the rows of the inverse (C^3 / 3 of stage 2's 2 C^3 / 3 flops) are
+ * not needed.
  *   F   [C x C] fp32, fully overwritten: for diagonal blocks of GPTQ_FACTOR_BLOCK (1024) columns, block (J, J) holds
- *       U_JJ (upper triangular); block (I, J), I < J, holds U~_IJ; the strict lower triangle is 0.  For C <= 1024 F = U.
+ *       U_JJ (upper triangular); the blocks above it hold U~[:, J] U_JJ; the strict lower triangle is 0.  For
+ *       C <= 1024 F = U.
  *       F may be the same buffer as H.
  *   Everything else (H, damp, workspace, dev_info, streams, errors) as gptq_prepare_hinv; same workspace query.
  * Consumer: gptq_quantize_layer_factor. */
@@ -203,8 +205,8 @@ gptq_status_t gptq_quantize_layer(const void* W_fp16, const float* U, int R, int
 
 /* gptq_quantize_layer on the output F of gptq_prepare_factor instead of U: same arguments, same outputs (codes, scales,
  * zero-points and loss agree with the U form up to fp32-level rounding of the update sums).  Across blocks of 1024
- * columns it feeds back the plain residuals w - q through U~ and the block's own U (see gptq_prepare_factor); inside a
- * block it is Algorithm 1 as written.  Runs in the row-stripe form only: for C > 1024 the block size must divide 1024
+ * columns it feeds back the plain residuals w - q through the blocks of F above the diagonal (see gptq_prepare_factor);
+ * inside a block it is Algorithm 1 as written.  Runs in the row-stripe form only: for C > 1024 the block size must divide 1024
  * (32, 64, 128, 256) and a group wider than the block must divide 1024 too, else GPTQ_ERR_UNSUPPORTED.
  * Workspace: gptq_quantize_workspace_bytes. */
 gptq_status_t gptq_quantize_layer_factor(const void* W_fp16, const float* F, int R, int C,

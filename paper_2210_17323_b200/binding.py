@@ -241,11 +241,9 @@ def factor_form_supported(C, block, group_sizes=()):
 
 
 def factor_form_pays(R, C, n_grids=1):
-    """Rule of thumb for choosing between the two forms of stages 2 and 3.  The factor form leaves out the second half of
-    stage 2 (about C^3 / 3 multiply-adds, once per layer) and adds, per grid and outer block of 1024 columns, one product of
-    the block's update sums with the block's own U (R * 1024 * C multiply-adds per grid over the layer): it pays for
-    layers that are wide rather than tall."""
-    return C > 1024 and C * C > 3 * 1024 * R * max(1, n_grids)
+    """The factor form leaves out the rows of the inverse (about C^3 / 3 multiply-adds) and adds one 1024-deep product per
+    block column of the factor (C^2 * 512): it pays for every layer with more than one block of 1024 columns."""
+    return C > 1024
 
 
 def gptq_set_stage3_variant(variant: int) -> int:

@@ -271,6 +271,21 @@ struct EpiSubUpperRed {
     }
   }
 };
+// dst[row][col] = partial * sa[row] * sb[col] * factor (fp32).  Only valid when the contraction is a single super-chunk.
+struct EpiStoreScaledF32 {
+  float* p; int64_t ld; int M, N;
+  const float* sa; const float* sb; float factor;
+  __device__ __forceinline__ void operator()(int row, int col0, const float (&v)[32]) const {
+    if (row >= M || col0 >= N) return;
+    float4* d = reinterpret_cast<float4*>(p + (int64_t)row * ld + col0);
+    const float a = sa[row] * factor;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      const float4 b = *reinterpret_cast<const float4*>(sb + col0 + 4 * g);
+      d[g] = make_float4(v[4 * g] * a * b.x, v[4 * g + 1] * a * b.y, v[4 * g + 2] * a * b.z, v[4 * g + 3] * a * b.w);
+    }
+  }
+};
 // Stores partial * factor as an fp16 hi / lo pair.  Only valid when the contraction is a single super-chunk
 // (K <= f16x3::kSuperK), so that the partial sum IS the result.
 struct EpiStoreSplit {
@@ -634,7 +649,26 @@ gptq_status_t prepare_impl(const float* H, float damp, int C, float* U, void* ws
     if (st == GPTQ_OK && (j1 != cudaSuccess || j2 != cudaSuccess || j3 != cudaSuccess || j4 != cudaSuccess)) st = GPTQ_ERR_CUDA;
   }
   if (st != GPTQ_OK) return st;
-  if (factor_only) return GPTQ_OK;
+  if (factor_only) {
+    // The factor form's consumer multiplies residuals by U~[before, J] U_JJ (see gptq_prepare_factor): form that product
+    // once here, panel by panel, from the fp16 copies of the factor's rows and the transposed diagonal block -- the first
+    // of phase 2's two contractions per panel, written out in fp32 over U~[0:j0, J]; the second one (the inverse's rows,
+    // K up to C) is what this form leaves out.
+    for (int J = 1; J < n_outer; ++J) {
+      const int j0 = J * kNB2, wj = (C - j0 < kNB2) ? C - j0 : kNB2;
+      panel_scales_kernel<<<wj, 256, 0, s>>>(U + (int64_t)j0 * C + j0, C, wj, w.rinv + j0, w.g[0], w.ginv[0], w.gam, w.gam2inv);
+      GPTQ_LAUNCH_CHECK();
+      dim3 grid(ceil_div(wj, 32), ceil_div(wj, 32)), blk(32, 32);
+      split_diag_t_kernel<<<grid, blk, 0, s>>>(U, C, j0, w.gam, w.VThi, w.VTlo, kNB2);
+      GPTQ_LAUNCH_CHECK();
+      f16x3::Operand A{w.Fhi + j0, w.Flo + j0, j0, wj, C};          // U~[0:j0, J] rs_i
+      f16x3::Operand B{w.VThi, w.VTlo, wj, wj, kNB2};               // V_JJ[k][n] gam_n, as [n][k]
+      // partial = rs_i gam_n (U~ V)[i][n];  1 / gam_n = gam2inv_n / 32
+      st = f16x3::launch<false, false>(A, B, j0, wj, EpiStoreScaledF32{U + j0, C, j0, wj, w.rsinv, w.gam2inv, 1.f / 32.f}, dev_info, s);
+      if (st != GPTQ_OK) return st;
+    }
+    return GPTQ_OK;
+  }
 
   // Phase 2: U = U~^-1, outer panel by outer panel, in place.  The diagonal blocks are already inverted;
   // rows above them: U[0:j0, J] = -U[0:j0, 0:j0] * (U~[0:j0, J] * V_JJ).

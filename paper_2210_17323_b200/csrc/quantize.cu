@@ -445,33 +445,6 @@ split_panel_t_kernel(const float* __restrict__ U, int C, int i2, int rows,
   }
 }
 
-// Factor form: the fp32 sums D = (R U~[before, blk]) sE[row] sC2[col] of the first contraction become the left operand
-// of the second one, D' = D sK[col] / sC2[col] (the size of a scaled weight correction), as an fp16 hi / lo pair.
-__global__ void split_dsum_kernel(const float* __restrict__ D, int64_t ldd, int R, int nb2, int i2,
-                                  const float* __restrict__ sK, const float* __restrict__ sC2inv,
-                                  __half* __restrict__ Dhi, __half* __restrict__ Dlo, int* dev_info) {
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;       // one thread: 8 consecutive columns
-  const int per_row = nb2 / 8;
-  if (idx >= (int64_t)R * per_row) return;
-  const int r = (int)(idx / per_row), c = (int)(idx % per_row) * 8;
-  const float4 a = *reinterpret_cast<const float4*>(D + (int64_t)r * ldd + c);
-  const float4 b = *reinterpret_cast<const float4*>(D + (int64_t)r * ldd + c + 4);
-  const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-  uint32_t hw[4], lw[4];
-  bool sat = false;
-#pragma unroll
-  for (int u = 0; u < 8; u += 2) {
-    __half h0, l0, h1, l1;
-    f16x3::split_f16(v[u] * (sK[i2 + c + u] * sC2inv[i2 + c + u]), h0, l0, sat);
-    f16x3::split_f16(v[u + 1] * (sK[i2 + c + u + 1] * sC2inv[i2 + c + u + 1]), h1, l1, sat);
-    hw[u >> 1] = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
-    lw[u >> 1] = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
-  }
-  *reinterpret_cast<uint4*>(Dhi + (int64_t)r * ldd + c) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-  *reinterpret_cast<uint4*>(Dlo + (int64_t)r * ldd + c) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-  if (sat) report_error(dev_info, GPTQ_ERR_NONFINITE, r);
-}
-
 // ---- contraction epilogue (one thread: one row, 32 consecutive columns of a partial sum) --------
 // Wblk[row][nofs + col ..) -= partial / (sE[row] sC[column]), as fp64 reductions: partial sums of one tile
 // come from several CTA pairs (one per super-chunk of the contraction).
@@ -541,11 +514,9 @@ extern "C" size_t gptq_quantize_workspace_bytes(int R, int C, int bits, int grou
   w.take<float>((size_t)R);                                       // sE
   w.take<float>((size_t)R);                                       // 1 / sE
   w.take<float>((size_t)R * outer_block(C, group_size, block));   // scaled fp32 sums of the lazy update of the outer block
-  w.take<uint32_t>((size_t)C);                                    // factor form: column maxima of U~ above the diagonal blocks,
+  w.take<uint32_t>((size_t)C);                                    // factor form: column maxima above the diagonal blocks,
   w.take<float>((size_t)C);                                       //   sC2,
-  w.take<float>((size_t)C);                                       //   1 / sC2,
-  w.take<__half>((size_t)R * outer_block(C, group_size, block));  //   left operand of the second contraction, high parts
-  w.take<__half>((size_t)R * outer_block(C, group_size, block));  //   remainders
+  w.take<float>((size_t)C);                                       //   1 / sC2
   return w.off;
 }
 
@@ -591,8 +562,6 @@ gptq_status_t quantize_impl(const void* W_fp16, const float* U, int R, int C,
   uint32_t* colmax2 = w.take<uint32_t>((size_t)C);
   float* sC2 = w.take<float>((size_t)C);
   float* sC2inv = w.take<float>((size_t)C);
-  __half* Dhi = w.take<__half>((size_t)R * B2);
-  __half* Dlo = w.take<__half>((size_t)R * B2);
   const int64_t ldw = B2;
   GridSpec gs{bits == GPTQ_BITS_TERNARY ? 2 : (1 << bits) - 1, ((sym & GPTQ_GRID_SYMMETRIC) != 0 || bits == GPTQ_BITS_TERNARY) ? 1 : 0,
               (sym & GPTQ_GRID_FP16_SCALES) ? 1 : 0};
@@ -651,21 +620,12 @@ gptq_status_t quantize_impl(const void* W_fp16, const float* U, int R, int C,
         if (st != GPTQ_OK) return st;
         st = f16x3::launch<false, false>(A, Bop, R, nb2, f16x3::EpiTileAddF32{R, nb2, 1.f, nullptr, nullptr}, dev_info, s, 0, &out);
         if (st != GPTQ_OK) return st;
-        if (factor) {
-          // A holds the plain residuals R' and the panel rows above the block hold U~: the sums are (R U~[before, blk]);
-          // times the block's own U (the rows of the panel inside the block) they are the correction of the block
-          const int64_t n8 = (int64_t)R * (nb2 / 8);
-          split_dsum_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, s>>>(Dsum, B2, R, nb2, i2, sK, sC2inv, Dhi, Dlo, dev_info);
-          GPTQ_LAUNCH_CHECK();
-          GPTQ_CUDA_TRY(cudaMemsetAsync(Dsum, 0, (size_t)R * B2 * sizeof(float), s));
-          f16x3::Operand A2{Dhi, Dlo, R, nb2, B2}, B2op{Phi + i2, Plo + i2, nb2, nb2, C};
-          st = f16x3::launch<false, false>(A2, B2op, R, nb2, f16x3::EpiTileAddF32{R, nb2, 1.f, nullptr, nullptr}, dev_info, s, 0, &out);
-          if (st != GPTQ_OK) return st;
-        }
       }
+      // (factor form: A holds the plain residuals and the panel rows above the block hold U~[before, blk] U_blk, scaled per
+      // column by sC2: the sums ARE the block's correction, with the opposite sign)
       dim3 grid(nb2 / 32, ceil_div(R, 128)), blk(32, 8);
-      wblk_stripe_major_kernel<<<grid, blk, 0, s>>>(W, R, C, i2, i2 > 0 ? Dsum : nullptr, B2, sEinv, sCinv, factor ? 1.0 : -1.0,
-                                                    Wblk, ldw);
+      wblk_stripe_major_kernel<<<grid, blk, 0, s>>>(W, R, C, i2, i2 > 0 ? Dsum : nullptr, B2, sEinv, factor ? sC2inv : sCinv,
+                                                    factor ? 1.0 : -1.0, Wblk, ldw);
       GPTQ_LAUNCH_CHECK();
     } else {
       int64_t total = (int64_t)R * nb2;

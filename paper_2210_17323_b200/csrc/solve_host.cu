@@ -182,10 +182,9 @@ gptq_status_t solve_layer_host_enqueue(const HostWs& w, StreamGuard& g, cudaStre
     GPTQ_CUDA_TRY(cudaEventRecord(g.freed[b], s));
   }
   GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, g.w_done, 0));
-  // Factor form (stage 2 without the inverse; same results) where stage 3 can run it for every grid and it pays: it
-  // leaves out about C^3 / 3 multiply-adds once and adds R * 1024 * C per grid (see gptq_prepare_factor).
-  bool factor = C > GPTQ_FACTOR_BLOCK && block > 0 && block <= 256 && GPTQ_FACTOR_BLOCK % block == 0 &&
-                (double)C * C > 3.0 * GPTQ_FACTOR_BLOCK * (double)R * n_grids;
+  // Factor form (stage 2 without the rows of the inverse; same results, see gptq_prepare_factor) where stage 3 can run
+  // it for every grid.
+  bool factor = C > GPTQ_FACTOR_BLOCK && block > 0 && block <= 256 && GPTQ_FACTOR_BLOCK % block == 0;
   for (int gi = 0; gi < n_grids && factor; ++gi)
     if (group_size[gi] > block && GPTQ_FACTOR_BLOCK % group_size[gi] != 0) factor = false;
   st = factor ? gptq_prepare_factor(w.H, damp, C, w.U, w.stage_ws, w.stage_ws_bytes, w.info + 2, s)

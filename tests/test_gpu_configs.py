@@ -83,7 +83,8 @@ def _solve_gpu(B, D, L, wl, grids, keep_x=False):
 
 def _check_factor_against_u(F, U, blk=1024):
     """gptq_prepare_factor's output against gptq_prepare_hinv's on the device: the same diagonal blocks up to rounding, and for the last
-    block of columns J the identity U[:j0, J] = -U[:j0, :j0] (U~[:j0, J] U_JJ) on a probe vector, in fp64 row chunks."""
+    block of columns J the identity U[:j0, J] = -U[:j0, :j0] F[:j0, J] (F[:j0, J] = U~[:j0, J] U_JJ) on a probe vector, in
+    fp64 row chunks."""
     C = U.shape[0]
     for j0 in range(0, C, blk):
         j1 = min(C, j0 + blk)
@@ -94,7 +95,7 @@ def _check_factor_against_u(F, U, blk=1024):
         return
     g = torch.Generator(device="cuda").manual_seed(5)
     z = torch.randn(C - j0, dtype=torch.float64, device="cuda", generator=g)
-    v = F[:j0, j0:].double() @ (U[j0:, j0:].double() @ z)
+    v = F[:j0, j0:].double() @ z
     lhs = U[:j0, j0:].double() @ z
     rhs = torch.empty_like(lhs)
     for r0 in range(0, j0, 4096):

@@ -603,8 +603,9 @@ def test_two_hessian_launches_side_by_side_on_two_streams(B):
 
 # ------------------------------------------------------------------ factor form (stage 2 without the inverse)
 def test_prepare_factor_holds_the_factor_above_and_u_on_the_diagonal_blocks(B):
-    """gptq_prepare_factor against the oracle: diagonal blocks of 1024 columns = the blocks of U, blocks above them = the
-    blocks of U^-1 (the upper factor of the damped Hessian)."""
+    """gptq_prepare_factor against the oracle: diagonal blocks of 1024 columns = the blocks of U; above a diagonal block
+    J the factor's block column times that diagonal block, U~[:j0, J] U_JJ with U~ = U^-1 the upper factor of the damped
+    Hessian."""
     C = 2304
     L = _layer(8, C, 2 * C + 100)
     H64 = O.hessian_accumulate(np.zeros((C, C)), L.x_bits())
@@ -619,7 +620,7 @@ def test_prepare_factor_holds_the_factor_above_and_u_on_the_diagonal_blocks(B):
         j1 = min(C, j0 + 1024)
         assert rel_fro(Fg[j0:j1, j0:j1], U[j0:j1, j0:j1]) <= TOL_U_FRO
         if j0 > 0:
-            assert rel_fro(Fg[:j0, j0:j1], Ut[:j0, j0:j1]) <= TOL_U_FRO
+            assert rel_fro(Fg[:j0, j0:j1], Ut[:j0, j0:j1] @ U[j0:j1, j0:j1]) <= TOL_U_FRO
 
 
 @pytest.mark.parametrize("R,C,bits,group,block", [(200, 2304, 4, 0, 128), (130, 3072, 3, 128, 128), (96, 2048, 2, 32, 64),
