@@ -445,6 +445,45 @@ split_panel_t_kernel(const float* __restrict__ U, int C, int i2, int rows,
   }
 }
 
+// Factor form: R'[r][c] = (w[r][c] - scale (code - zero)) sE[r] for the columns [i2, i2 + nb2) of every row, as an fp16
+// hi / lo pair in Ehi / Elo: the plain residuals, formed in fp64 from the original weights and the codes, scales and
+// zero-points the block's solve has just written.  One thread: 8 consecutive columns.
+__global__ void residual_pair_kernel(const __half* __restrict__ W, const uint8_t* __restrict__ codes,
+                                     const float* __restrict__ scales, const float* __restrict__ zeros, int G, int g,
+                                     const float* __restrict__ sE, int R, int C, int i2, int nb2,
+                                     __half* __restrict__ Ehi, __half* __restrict__ Elo, int* dev_info) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int per_row = nb2 / 8;
+  if (idx >= (int64_t)R * per_row) return;
+  const int r = (int)(idx / per_row), c = i2 + (int)(idx % per_row) * 8;
+  const int64_t o = (int64_t)r * C + c;
+  const uint4 wv = *reinterpret_cast<const uint4*>(W + o);
+  const uint2 cv = *reinterpret_cast<const uint2*>(codes + o);
+  const __half* wh = reinterpret_cast<const __half*>(&wv);
+  const uint8_t* cb = reinterpret_cast<const uint8_t*>(&cv);
+  const float se = sE[r];
+  uint32_t hw[4], lw[4];
+  bool sat = false;
+#pragma unroll
+  for (int u = 0; u < 8; u += 2) {
+    float rr[2];
+#pragma unroll
+    for (int v = 0; v < 2; ++v) {
+      const int gi = g > 0 ? (c + u + v) / g : 0;
+      const double sc = (double)scales[(int64_t)r * G + gi], ze = (double)zeros[(int64_t)r * G + gi];
+      rr[v] = (float)((double)__half2float(wh[u + v]) - sc * ((double)cb[u + v] - ze));
+    }
+    __half h0, l0, h1, l1;
+    f16x3::split_f16(rr[0] * se, h0, l0, sat);
+    f16x3::split_f16(rr[1] * se, h1, l1, sat);
+    hw[u >> 1] = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
+    lw[u >> 1] = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
+  }
+  *reinterpret_cast<uint4*>(Ehi + o) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+  *reinterpret_cast<uint4*>(Elo + o) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+  if (sat) report_error(dev_info, GPTQ_ERR_NONFINITE, r);
+}
+
 // ---- contraction epilogue (one thread: one row, 32 consecutive columns of a partial sum) --------
 // Wblk[row][nofs + col ..) -= partial / (sE[row] sC[column]), as fp64 reductions: partial sums of one tile
 // come from several CTA pairs (one per super-chunk of the contraction).
@@ -640,9 +679,16 @@ gptq_status_t quantize_impl(const void* W_fp16, const float* U, int R, int C,
     if (stripe) {
       // row-stripe form: every inner block of this outer block in one launch
       StripeArgs a{Wblk, ldw, nb2, U, C, i2, stripe_block, R, gs, g, scales, zeros, G, Ehi, Elo, Phi, Plo, (int64_t)C,
-                   sK, sE, sEinv, sCinv, codes, loss, dev_info, factor ? W : nullptr};
+                   sK, sE, sEinv, sCinv, codes, loss, dev_info, factor ? 0 : 1};
       gptq_status_t st = launch_stripe(a, Phi, Plo, s);
       if (st != GPTQ_OK) return st;
+      if (factor && i2 + nb2 < C) {
+        // factor form: what later outer blocks contract with is the plain residual of this block's columns
+        const int64_t n8 = (int64_t)R * (nb2 / 8);
+        residual_pair_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, s>>>(W, codes, scales, zeros, G, g, sE, R, C, i2, nb2, Ehi, Elo,
+                                                                          dev_info);
+        GPTQ_LAUNCH_CHECK();
+      }
       continue;
     }
     for (int i = i2; i < i2 + nb2; i += block) {

@@ -48,8 +48,9 @@ struct StripeArgs {
   const __half* Phi; const __half* Plo; int64_t ldp;   // scaled transposed panel of U: Pt[c - i2][k] (see quantize.cu)
   const float* sK; const float* sE; const float* sEinv; const float* sCinv;
   uint8_t* codes; double* loss; int* dev_info;
-  const __half* W16;                          // factor form: the original weights [R][C]; Ehi / Elo then receive the plain
-                                              // residuals (w - q) sE[row] instead of the scaled errors.  nullptr otherwise.
+  int keep_errors;                            // 1: the scaled errors also go to Ehi / Elo in global memory (the left operand of
+                                              // later outer blocks' contractions); 0: factor form, a separate kernel writes the
+                                              // plain residuals there from the codes
 };
 
 // shared memory (from a 1024-byte aligned base):
@@ -305,13 +306,7 @@ stripe_kernel(const __grid_constant__ StripeMaps maps, const StripeArgs a) {
         uint32_t cw[kStripeSB / 4];
 #pragma unroll
         for (int m = 0; m < kStripeSB / 4; ++m) cw[m] = 0;
-        // factor form: the sub-block's original weights, for the plain residuals w - q
-        float res[kStripeSB];
-        uint4 w16a = make_uint4(0, 0, 0, 0), w16b = make_uint4(0, 0, 0, 0);
-        if (a.W16 != nullptr && live) {
-          const uint4* wp = reinterpret_cast<const uint4*>(a.W16 + (int64_t)row * a.C + i + j0);
-          w16a = __ldg(wp); w16b = __ldg(wp + 1);
-        }
+
         const double* ud = Ud + (size_t)j0 * kStripeSB;    // this sub-block's 16 x 16 block of U
 #pragma unroll
         for (int jj = 0; jj < kStripeSB; ++jj) {
@@ -339,11 +334,6 @@ stripe_kernel(const __grid_constant__ StripeMaps maps, const StripeArgs a) {
           const double wq = scale * (q - zero);
           const double e = (wj - wq) * rdiag[j0 + jj];     // scaled error (w - q) / U_jj
           err[jj] = e;
-          {
-            const uint32_t pairw = jj < 8 ? (&w16a.x)[jj >> 1] : (&w16b.x)[(jj - 8) >> 1];
-            const float worig = __half2float(__ushort_as_half((unsigned short)((jj & 1) ? (pairw >> 16) : (pairw & 0xFFFFu))));
-            res[jj] = (float)((double)worig - wq);
-          }
           loss += e * e;
           bad |= !isfinite(e);
           cw[jj >> 2] |= (uint32_t)q << (8 * (jj & 3));
@@ -385,23 +375,7 @@ stripe_kernel(const __grid_constant__ StripeMaps maps, const StripeArgs a) {
           const int64_t o = (int64_t)row * a.C + i + j0;
           uint4* gh = reinterpret_cast<uint4*>(a.Ehi + o);
           uint4* gl = reinterpret_cast<uint4*>(a.Elo + o);
-          if (a.W16 == nullptr) {
-            gh[0] = h_a; gh[1] = h_b; gl[0] = l_a; gl[1] = l_b;
-          } else {
-            // the left operand of later outer blocks' contractions is the plain residual here
-            uint32_t rh[kStripeSB / 2], rl[kStripeSB / 2];
-#pragma unroll
-            for (int u = 0; u < kStripeSB; u += 2) {
-              __half h0, l0, h1, l1;
-              f16x3::split_f16(res[u] * se_row, h0, l0, sat);
-              f16x3::split_f16(res[u + 1] * se_row, h1, l1, sat);
-              rh[u >> 1] = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
-              rl[u >> 1] = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
-            }
-            bad |= sat;
-            gh[0] = make_uint4(rh[0], rh[1], rh[2], rh[3]); gh[1] = make_uint4(rh[4], rh[5], rh[6], rh[7]);
-            gl[0] = make_uint4(rl[0], rl[1], rl[2], rl[3]); gl[1] = make_uint4(rl[4], rl[5], rl[6], rl[7]);
-          }
+          if (a.keep_errors) { gh[0] = h_a; gh[1] = h_b; gl[0] = l_a; gl[1] = l_b; }
           *reinterpret_cast<uint4*>(a.codes + o) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
         }
         TOCK(4, ts4);
