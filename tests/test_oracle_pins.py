@@ -474,3 +474,26 @@ def test_dequantize_and_matvec_definitions():
     # fp16 storage reading: within half an fp16 ulp of the exact value
     d16 = O.dequantize(out["codes"], out["scales"], out["zeros"], to_fp16=True)
     assert d16.dtype == np.float16 and np.all(np.abs(d16.astype(np.float64) - deq) <= np.abs(deq) * 2.0 ** -11 + 1e-12)
+
+
+@pytest.mark.parametrize("bits,group", [(4, 0), (3, 16), (2, 0)])
+def test_residuals_through_the_factor_give_the_lazy_update(bits, group):
+    """The identity the CUDA path's factor form rests on, checked on the oracle's own trajectory.  Algorithm 1's updates
+    sum to W - Q = E U; hence E = (W - Q) U~ with U~ = U^-1 (the upper factor of the damped Hessian, H~ = U~ U~^T), and for
+    any block J of columns, what the lazy updates have subtracted from block J when the loop reaches it,
+    E[:, :j0] U[:j0, J], equals -((W - Q)[:, :j0] U~[:j0, J]) U[J, J]."""
+    C, blk = 96, 32
+    W, Xt = _random_problem(12, C, 400, 21)
+    H = O.hessian_accumulate(np.zeros((C, C)), Xt)
+    Ht, _ = O.dampen(H, 0.01)
+    U = O.cholesky_inverse_upper(Ht)
+    Ut = np.linalg.inv(U)
+    assert np.allclose(Ut @ Ut.T, Ht, rtol=1e-10, atol=1e-12 * np.abs(Ht).max())          # U~ is the factor of H~ itself
+    out = O.quantize_layer(W, U, bits, group, False, block=16)
+    Rm = W.astype(np.float64) - out["W_hat"]                                               # plain residuals w - q
+    assert np.allclose(out["E"], Rm @ Ut, rtol=1e-8, atol=1e-12)
+    for j0 in range(blk, C, blk):
+        J = slice(j0, j0 + blk)
+        lazy = out["E"][:, :j0] @ U[:j0, J]
+        through_factor = -(Rm[:, :j0] @ Ut[:j0, J]) @ U[J, J]
+        assert np.allclose(lazy, through_factor, rtol=1e-8, atol=1e-12)
