@@ -270,7 +270,7 @@ def run_gpu(args, wl):
 
     stage_events = []                             # (layer idx, events) of the timed steps
     factor = _factor_form(args, wl)
-    for st in state:                              # per layer: the factor form where it pays (wide layers), else the inverse form
+    for st in state:                              # per layer: the factor form where it pays (more than one block of 1024 columns)
         st["factor"] = factor and B.factor_form_pays(st["L"].R, st["L"].C, len(wl.grids))
 
     graphs = []                                   # per layer: CUDA graphs of the three stages (launch-bound inner loops)
@@ -467,7 +467,7 @@ def run_gpu(args, wl):
                 config=dict(workload=wl.name, layers=[l.name for l in wl.layers],
                             grids=[dict(bits=g.bits, group_size=g.group_size, sym=g.sym) for g in wl.grids],
                             block=wl.block, damp=wl.damp, calib_tokens=wl.layers[0].n_tokens,
-                            form=("factor where it pays (wide layers): gptq_prepare_factor + gptq_quantize_layer_factor (E = (W - Q) U~; "
+                            form=("factor: gptq_prepare_factor + gptq_quantize_layer_factor (E = (W - Q) U~; "
                                   "the factor's inverse is never formed); inverse form for: " +
                                   (", ".join(n for n, f in uses_factor.items() if not f) or "no layer")) if factor
                                  else "inverse: gptq_prepare_hinv + gptq_quantize_layer (U = Cholesky(H^-1)^T)",
