@@ -16,9 +16,12 @@ def rel_fro(a, b):
     return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
 
 
-def check_quantize_outputs(gpu, ref, W16, bits, C, H=None, min_identical=TOL_CODES_IDENTICAL):
+def check_quantize_outputs(gpu, ref, W16, bits, C, H=None, min_identical=TOL_CODES_IDENTICAL, scale_fp16=False):
     """gpu: dict of numpy arrays from the CUDA path (qweight uint32, scales, zeros, loss).
-    ref: oracle quantize_layer dict.  Returns a dict of measured figures."""
+    ref: oracle quantize_layer dict.  Returns a dict of measured figures.
+    scale_fp16: the scales are fp16 values, each a rounding decision taken from working weights that the two sides hold
+    to about 1e-7 of each other, so a scale next to an fp16 rounding boundary may fall on either side of it: they are
+    compared as fp16 numbers (at most one unit in the last place apart, the same fraction identical as for the codes)."""
     qw = gpu["qweight"].view(np.uint32)
     codes = O.unpack_codes(qw, bits, C)
     # packed layout: bit-exact against the oracle's packer applied to the same codes
@@ -30,7 +33,15 @@ def check_quantize_outputs(gpu, ref, W16, bits, C, H=None, min_identical=TOL_COD
     assert identical >= min_identical, f"only {identical:.5f} of the codes identical"
     s_err = rel_fro(gpu["scales"], ref["scales"])
     z_err = rel_fro(gpu["zeros"], ref["zeros"])
-    assert s_err <= TOL_SCALE_ZERO, f"scales rel err {s_err}"
+    if scale_fp16:
+        hg = gpu["scales"].astype(np.float16)
+        hr = ref["scales"].astype(np.float16)
+        assert np.array_equal(hg.astype(np.float32), gpu["scales"].astype(np.float32)), "a scale is not an fp16 value"
+        ulps = np.abs(hg.view(np.int16).astype(np.int32) - hr.view(np.int16).astype(np.int32))
+        assert ulps.max() <= 1, f"a scale is {ulps.max()} fp16 units from the oracle's"
+        assert (ulps == 0).mean() >= min_identical, f"only {(ulps == 0).mean():.5f} of the fp16 scales identical"
+    else:
+        assert s_err <= TOL_SCALE_ZERO, f"scales rel err {s_err}"
     assert z_err <= TOL_SCALE_ZERO, f"zeros rel err {z_err}"
     out = dict(identical=identical, scales_err=s_err, zeros_err=z_err)
     g = C // gpu["scales"].shape[1]

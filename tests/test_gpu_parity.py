@@ -624,7 +624,8 @@ def test_prepare_factor_holds_the_factor_above_and_u_on_the_diagonal_blocks(B):
 
 
 @pytest.mark.parametrize("R,C,bits,group,block", [(200, 2304, 4, 0, 128), (130, 3072, 3, 128, 128), (96, 2048, 2, 32, 64),
-                                                  (64, 2304, O.BITS_TERNARY, 8, 32), (100, 2048, 4, 1024, 256), (70, 768, 4, 0, 128)])
+                                                  (64, 2304, O.BITS_TERNARY, 8, 32), (100, 2048, 4, 1024, 256), (70, 768, 4, 0, 128),
+                                                  (1, 1056, 4, 0, 128), (129, 1280, 3, 64, 32), (33, 4128, 8, 0, 128)])
 def test_factor_form_matches_the_oracle(B, R, C, bits, group, block):
     """Stages 2 and 3 in the factor form (no inverse; plain residuals fed back through the factor across blocks of 1024
     columns) against the oracle, which runs Algorithm 1 as written with U."""
@@ -647,3 +648,54 @@ def test_factor_form_rejects_blockings_it_cannot_run(B):
     with pytest.raises(B.GptqError) as e:
         B.gptq_quantize_layer(W, F, 4, 0, False, 96, factor=True)      # outer blocks of 960 columns
     assert e.value.status == B.ERR_UNSUPPORTED
+
+
+def test_factor_form_with_symmetric_grid_and_fp16_scales(B):
+    """The grid options reach the factor form unchanged: symmetric grid and fp16-rounded scales, three outer blocks.
+    (With fp32 scales the symmetric grid has a built-in tie: the weight of largest magnitude in a group, when negative,
+    sits exactly between codes 0 and 1, and the rounding of the scale decides; fp16 rounding moves it off the tie.)"""
+    L = _layer(90, 2304, 5000, cfg=10)
+    xb, W16 = L.x_bits(), L.w()
+    H64 = O.hessian_accumulate(np.zeros((L.C, L.C)), xb)
+    Ht, _ = O.dampen(H64.astype(np.float32).astype(np.float64), 0.01)
+    U = O.cholesky_inverse_upper(Ht)
+    ref = O.quantize_layer(W16, U, 3, 128, True, 128, scale_fp16=True)
+    F, info = B.gptq_prepare_hinv(torch.from_numpy(H64.astype(np.float32)).cuda(), 0.01, factor=True)
+    out = B.gptq_quantize_layer(torch.from_numpy(W16).cuda(), F, 3, 128, True, 128, scale_fp16=True, factor=True)
+    torch.cuda.synchronize()
+    assert info.tolist() == [0, 0] and out["dev_info"].tolist() == [0, 0]
+    gpu = dict(qweight=out["qweight"].cpu().numpy(), scales=out["scales"].cpu().numpy(), zeros=out["zeros"].cpu().numpy(),
+               loss=out["loss"].item())
+    check_quantize_outputs(gpu, ref, W16, 3, L.C, H64, scale_fp16=True)
+
+
+@pytest.mark.parametrize("factor", [False, True])
+def test_symmetric_grid_with_fp32_scales_differs_only_after_its_tie(B, factor):
+    """The symmetric grid has a tie by construction: scale = 2a / maxq with a = max |w| of the group and an even number of
+    levels put -a exactly midway between codes 0 and 1.  When the weight of largest magnitude is negative and sits in the
+    group's first column (it is quantized before any feedback moves it), the fp32 rounding of the scale decides, and that
+    rounding follows the last bits of a working weight the two sides hold to ~1e-7.  Both codes are equally near, so the
+    check is: rows that never meet the tie are identical; every other row first differs at a group's first column, by the
+    0/1 pair; and the loss agrees."""
+    g, bits = 128, 3
+    L = _layer(90, 2304, 5000, cfg=10)
+    W16 = L.w()
+    H64 = O.hessian_accumulate(np.zeros((L.C, L.C)), L.x_bits())
+    Ht, _ = O.dampen(H64.astype(np.float32).astype(np.float64), 0.01)
+    ref = O.quantize_layer(W16, O.cholesky_inverse_upper(Ht), bits, g, True, 128)
+    F, info = B.gptq_prepare_hinv(torch.from_numpy(H64.astype(np.float32)).cuda(), 0.01, factor=factor)
+    out = B.gptq_quantize_layer(torch.from_numpy(W16).cuda(), F, bits, g, True, 128, factor=factor)
+    torch.cuda.synchronize()
+    assert info.tolist() == [0, 0] and out["dev_info"].tolist() == [0, 0]
+    codes = O.unpack_codes(out["qweight"].cpu().numpy().view(np.uint32), bits, L.C)
+    same = codes == ref["codes"]
+    scales = out["scales"].cpu().numpy()
+    assert same.mean() >= 0.99 and same.all(axis=1).mean() >= 0.85
+    for r in range(L.R):
+        j = L.C if same[r].all() else int(np.argmin(same[r]))
+        if j < L.C:
+            assert j % g == 0 and j >= g, f"row {r} first differs at column {j}, not at a group's first column"
+            assert {int(codes[r, j]), int(ref["codes"][r, j])} == {0, 1}
+        n = min(j // g + 1, L.C // g)            # the groups whose grids were drawn before the row met the tie
+        assert rel_fro(scales[r, :n], ref["scales"][r, :n]) <= 1e-5
+    assert abs(out["loss"].item() - ref["loss"]) <= 0.01 * ref["loss"]
