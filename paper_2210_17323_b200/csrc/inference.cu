@@ -5,6 +5,8 @@
 // Dequantized value of code q in group gi of row r:  scales[r][gi] * (q - zeros[r][gi]), formed in fp32.
 #include "common.cuh"
 
+#include <type_traits>
+
 namespace gptq {
 namespace {
 
@@ -182,11 +184,12 @@ __host__ __device__ constexpr int mv_perm(int p) {
   if (F == 4) { constexpr int o[8] = {0, 4, 2, 6, 1, 5, 3, 7}; return (p & ~7) + o[p & 7]; }
   if (F == 2) { constexpr int o[16] = {0, 8, 2, 10, 4, 12, 6, 14, 1, 9, 3, 11, 5, 13, 7, 15}; return (p & ~15) + o[p & 15]; }
   if (F == 8) { constexpr int o[4] = {0, 2, 1, 3}; return (p & ~3) + o[p & 3]; }
-  return p;                                                                        // 3-bit: natural order
+  { constexpr int o[8] = {0, 1, 4, 5, 2, 3, 6, 7}; return (p & ~7) + o[p & 7]; }            // 3-bit
 }
 template <int F> struct MvScale2 { static constexpr float inv = 0.f; };            // 1 / factor of the second accumulator
 template <> struct MvScale2<4> { static constexpr float inv = 1.f / 16.f; };
 template <> struct MvScale2<2> { static constexpr float inv = 1.f / 4.f; };
+template <> struct MvScale2<3> { static constexpr float inv = 1.f / 64.f; };
 
 // One 32-column chunk of two rows (A fragment rows g and g + 8) against the staged x: 8 MMAs.
 template <int F>
@@ -232,22 +235,28 @@ __device__ __forceinline__ void mv_chunk<8>(const uint32_t (&wa)[8], const uint3
   }
 }
 
-// 3-bit: codes 2m and 2m + 1 sit next to each other at stream bit 6m; (v & 63) * 0x2001 copies the second
-// one to bit 16, and the mask keeps one code per half.
-__device__ __forceinline__ uint32_t pair3(const uint32_t (&w)[3], int m) {
-  const int bit = 6 * m, k = bit >> 5, o = bit & 31;
-  uint32_t v = w[k] >> o;
-  if (o + 6 > 32 && k + 1 < 3) v |= w[k + 1] << (32 - o);
-  return ((v & 63u) * 0x2001u) & 0x00070007u;
+// 3-bit: four consecutive codes are 12 bits of the stream.  With those 12 bits alone in a register (v),
+// v * 0x2001 = v | v << 13 holds code 0 at bit 0 and code 1 at bit 16 (one half2 operand under the mask 0x00070007,
+// factor 1), and code 2 at bit 6 and code 3 at bit 22 (a second operand under 0x01C001C0, factor 64, which goes to
+// the second accumulator): shift, mask, multiply and two ANDs for four codes.  Returns v * 0x2001 for run j (0..7)
+// of the chunk's three words.
+__device__ __forceinline__ uint32_t quad3(const uint32_t (&w)[3], int j) {
+  const int bit = 12 * j, k = bit >> 5, o = bit & 31;
+  uint32_t v;
+  if (o + 12 < 32) v = (w[k] >> o) & 0xFFFu;
+  else if (o + 12 == 32) v = w[k] >> 20;
+  else v = __funnelshift_r(w[k], w[k + 1 < 3 ? k + 1 : k], o) & 0xFFFu;
+  return v * 0x2001u;
 }
 template <>
 __device__ __forceinline__ void mv_chunk<3>(const uint32_t (&wa)[3], const uint32_t (&wb)[3], const uint4* xs,
-                                            float (&c1)[4], float (&)[4]) {
+                                            float (&c1)[4], float (&c2)[4]) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < 4; ++i) {          // runs 2i and 2i + 1: codes 8i .. 8i + 7
     const uint4 x = xs[i];
-    mma_16816(c1, pair3(wa, 4 * i), pair3(wb, 4 * i), pair3(wa, 4 * i + 1), pair3(wb, 4 * i + 1), x.x, x.y);
-    mma_16816(c1, pair3(wa, 4 * i + 2), pair3(wb, 4 * i + 2), pair3(wa, 4 * i + 3), pair3(wb, 4 * i + 3), x.z, x.w);
+    const uint32_t a0 = quad3(wa, 2 * i), a1 = quad3(wa, 2 * i + 1), b0 = quad3(wb, 2 * i), b1 = quad3(wb, 2 * i + 1);
+    mma_16816(c1, a0 & 0x00070007u, b0 & 0x00070007u, a1 & 0x00070007u, b1 & 0x00070007u, x.x, x.y);
+    mma_16816(c2, a0 & 0x01C001C0u, b0 & 0x01C001C0u, a1 & 0x01C001C0u, b1 & 0x01C001C0u, x.z, x.w);
   }
 }
 
@@ -372,6 +381,224 @@ matvec_mma_kernel(const uint32_t* __restrict__ qweight, const float* __restrict_
   }
 }
 
+// ---- y = dequant(Q) x, tensor path with the codes staged through shared memory --------------------------------
+// Same arithmetic as matvec_mma_kernel; what differs is how the codes travel.  There a lane loads its own fragment
+// words from global memory (16 row segments of 64 bytes per warp instruction, held in registers while in flight).
+// Here every warp owns a ring of kDepth stages in shared memory and fills it with asynchronous 16-byte copies
+// (cp.async.cg: global -> shared, no register, no L1 allocation) whose lanes cover whole consecutive pieces of a row;
+// the lanes then read their fragments from the stage.  Waiting is cp.async.wait_group + __syncwarp only: no
+// barrier object and no spin.  A stage is 16 rows x up to kSB blocks of 128 columns; a row of a stage is padded so
+// that the fragment reads of a warp fall on distinct banks.
+// A task is 16 consecutive rows; warp w of the CTA takes the blocks [w bpw, (w + 1) bpw) of every task in `nsub`
+// stages of `sbk` blocks, and the warps' partial sums meet in shared memory as before.
+// x is staged once per CTA, permuted as the unpacking wants it and interleaved inside a block: the 16-byte piece i
+// (0..3) of chunk t (0..3) sits at piece 4 i + t of the block, so that a warp's four lane groups read 64 consecutive
+// bytes.
+// 12 warps with rings of 3 stages (C = 12288, 4-bit) measured best: 8 warps leave issue slots idle, 16 warps leave room
+// for 2 stages only.
+#ifndef GPTQ_MP_WARPS
+#define GPTQ_MP_WARPS 12
+#endif
+constexpr int kMpWarps = GPTQ_MP_WARPS, kMpThreads = kMpWarps * 32;
+
+template <int F> struct MpGeom {
+  static constexpr int kSB = F == 4 ? 4 : F == 8 ? 2 : 8;                     // blocks per stage at most
+  static constexpr int kPiecesPerRow = kSB * F;                               // 16-byte pieces of one row of a stage (<= 32)
+  static constexpr int kRowsPerCopy = 32 / kPiecesPerRow;                     // rows one warp-wide copy instruction covers
+  static constexpr int kPad = F == 4 ? 64 : F == 3 ? 48 : F == 2 ? 32 : 16;   // makes the fragment reads conflict-free
+  static constexpr int kPitch = (kSB * 16 * F + 127) / 128 * 128 + kPad;      // bytes between rows of a stage
+  static constexpr int kStageBytes = 16 * kPitch;
+};
+
+__device__ __forceinline__ void cp_async_16(uint32_t sdst, const void* gsrc, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(sdst), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+template <int F>
+__device__ __forceinline__ void mp_read(const unsigned char* p, uint32_t (&w)[F]) {
+  if constexpr (F == 4) {
+    const uint4 v = *reinterpret_cast<const uint4*>(p);
+    w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+  } else if constexpr (F == 2) {
+    const uint2 v = *reinterpret_cast<const uint2*>(p);
+    w[0] = v.x; w[1] = v.y;
+  } else if constexpr (F == 8) {
+    const uint4 v0 = *reinterpret_cast<const uint4*>(p), v1 = *(reinterpret_cast<const uint4*>(p) + 1);
+    w[0] = v0.x; w[1] = v0.y; w[2] = v0.z; w[3] = v0.w; w[4] = v1.x; w[5] = v1.y; w[6] = v1.z; w[7] = v1.w;
+  } else {
+#pragma unroll
+    for (int k = 0; k < F; ++k) w[k] = reinterpret_cast<const uint32_t*>(p)[k];
+  }
+}
+
+// The eight MMAs of one block for fragment rows a and b, x read in the interleaved order.
+template <int F>
+__device__ __forceinline__ void mp_block(const uint32_t (&wa)[F], const uint32_t (&wb)[F], const uint4* xb, int t4,
+                                         float (&c1)[4], float (&c2)[4]) {
+  uint4 xs[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) xs[i] = xb[4 * i + t4];
+  mv_chunk<F>(wa, wb, xs, c1, c2);
+}
+
+// grid: min(tasks, SMs) CTAs of kMpThreads threads.  dynamic shared memory: x (fp16, C rounded up to 128), the block
+// sums of x (fp32), two buffers of partial sums, then kMpWarps rings of kDepth stages.
+template <int F, int kDepth>
+__global__ void __launch_bounds__(kMpThreads, 1)
+matvec_staged_kernel(const uint32_t* __restrict__ qweight, const float* __restrict__ scales, const float* __restrict__ zeros,
+                     const __half* __restrict__ x, int R, int C, int g, int G, int bpw, int nsub, int sbk,
+                     float* __restrict__ y) {
+  using Geo = MpGeom<F>;
+  extern __shared__ uint4 mv_smem[];
+  const int chunks = C / 32, n_blk = (C + 127) / 128, Cpad = n_blk * 128;
+  uint4* xs = mv_smem;                                                    // [n_blk][16] pieces
+  float* sx = reinterpret_cast<float*>(xs + (size_t)n_blk * 16);          // [n_blk]
+  float* red = sx + ((n_blk + 3) & ~3);                                   // [2][kMpWarps][16]
+  unsigned char* rings = reinterpret_cast<unsigned char*>(red + 2 * kMpWarps * 16);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gq = lane >> 2, t4 = lane & 3;
+  const int n_tasks = (R + 15) / 16;
+  const int my_tasks = blockIdx.x < n_tasks ? (n_tasks - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+  const bool per_block = g < C;
+  const int64_t row_bytes = (int64_t)chunks * F * 4;
+  const int blk_lo = warp * bpw, blk_hi = min(blk_lo + bpw, n_blk);        // this warp's blocks of every task
+  const int valid_pieces_row = (int)(row_bytes / 16);                     // pieces of a row that exist in memory
+  unsigned char* ring = rings + (size_t)warp * kDepth * Geo::kStageBytes;
+  const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
+  const unsigned char* qbytes = reinterpret_cast<const unsigned char*>(qweight);
+
+  // copy side: lane -> (row within the copy instruction, piece within the row)
+  const int c_row = lane / Geo::kPiecesPerRow, c_piece = lane % Geo::kPiecesPerRow;
+  const bool c_lane = lane < Geo::kRowsPerCopy * Geo::kPiecesPerRow;
+  int lk = 0, lj = 0, ls = 0;                                             // load cursor: task number, stage of the task, ring slot
+  auto issue = [&]() {
+    if (lk < my_tasks) {
+      const int task = blockIdx.x + lk * gridDim.x;
+      const int b0 = blk_lo + lj * sbk, nb = min(sbk, blk_hi - b0);       // blocks of this stage (nb may be <= 0)
+      const int piece0 = b0 * F;                                          // first piece of the stage inside the row
+      if (c_lane && c_piece < nb * F) {
+        const uint32_t fill = piece0 + c_piece < valid_pieces_row ? 16u : 0u;   // past the row's end: zeros
+        const int64_t col_off = fill ? (int64_t)(piece0 + c_piece) * 16 : 0;
+        uint32_t dst = ring_s + ls * Geo::kStageBytes + c_row * Geo::kPitch + c_piece * 16;
+        if (task * 16 + 16 <= R) {
+          const unsigned char* src = qbytes + (int64_t)(task * 16 + c_row) * row_bytes + col_off;
+#pragma unroll
+          for (int r = 0; r < 16; r += Geo::kRowsPerCopy) {
+            cp_async_16(dst, src, fill);
+            src += Geo::kRowsPerCopy * row_bytes;
+            dst += Geo::kRowsPerCopy * Geo::kPitch;
+          }
+        } else {                                                          // ragged last task: rows clamped, copies stay in range
+#pragma unroll
+          for (int r = 0; r < 16; r += Geo::kRowsPerCopy) {
+            const int row = min(task * 16 + r + c_row, R - 1);
+            cp_async_16(dst, qbytes + row * row_bytes + col_off, fill);
+            dst += Geo::kRowsPerCopy * Geo::kPitch;
+          }
+        }
+      }
+      if (++lj == nsub) { lj = 0; ++lk; }
+    }
+    cp_async_commit();                                                    // one group per slot, empty or not
+    if (++ls == kDepth) ls = 0;
+  };
+#pragma unroll
+  for (int d = 0; d < kDepth - 1; ++d) issue();            // the first stages are on their way while x is staged
+
+  // x: one 32-column chunk (64 bytes) per thread, permuted, written interleaved; the four threads of a block add up
+  // their chunks' sums
+  for (int base = warp * 32; base < Cpad / 32; base += blockDim.x) {
+    const int ch = base + lane;
+    float t = 0.f;
+    if (ch < Cpad / 32) {
+      __align__(16) __half in[32], out[32];
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        reinterpret_cast<uint4*>(in)[q] = ch < chunks ? __ldg(reinterpret_cast<const uint4*>(x + ch * 32) + q) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int p = 0; p < 32; ++p) { out[p] = in[mv_perm<F>(p)]; t += __half2float(in[p]); }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) xs[(ch >> 2) * 16 + 4 * q + (ch & 3)] = reinterpret_cast<const uint4*>(out)[q];
+    }
+    t += __shfl_xor_sync(0xffffffffu, t, 1);
+    t += __shfl_xor_sync(0xffffffffu, t, 2);
+    if ((lane & 3) == 0 && ch < Cpad / 32) sx[ch >> 2] = t;
+  }
+  __syncthreads();
+
+  int k = 0, j = 0, cs = 0, par = 0;
+  float ya = 0.f, yb = 0.f, ya2 = 0.f, yb2 = 0.f;
+  float xsum_w = 0.f;                                                     // sum of x over this warp's blocks (the same for every task)
+  for (int b = blk_lo; b < blk_hi; ++b) xsum_w += sx[b];
+  const int total = my_tasks * nsub;
+  for (int it = 0; it < total; ++it) {
+    const int task = blockIdx.x + k * gridDim.x;
+    const int ra = min(task * 16 + gq, R - 1), rb = min(task * 16 + gq + 8, R - 1);
+    const int b0 = blk_lo + j * sbk, nb = min(sbk, blk_hi - b0);
+    // grouped grids: the stage's scales and zero-points are requested before the wait for its codes
+    float gsa[Geo::kSB], gza[Geo::kSB], gsb[Geo::kSB], gzb[Geo::kSB];
+    if (per_block) {
+#pragma unroll
+      for (int b = 0; b < Geo::kSB; ++b) {
+        if (b < nb) {
+          const int gi = ((b0 + b) * 128) / g;
+          gsa[b] = __ldg(scales + (int64_t)ra * G + gi); gza[b] = __ldg(zeros + (int64_t)ra * G + gi);
+          gsb[b] = __ldg(scales + (int64_t)rb * G + gi); gzb[b] = __ldg(zeros + (int64_t)rb * G + gi);
+        }
+      }
+    }
+    cp_async_wait<kDepth - 2>();                                          // this stage's copies have landed (this lane's)
+    __syncwarp();                                                         // ... and every lane's; the previous stage is read
+    issue();                                                              // refill the slot read in the previous iteration
+    const unsigned char* st = ring + (size_t)cs * Geo::kStageBytes + gq * Geo::kPitch + t4 * (4 * F);
+    // a full stage runs without per-block branches, so that the blocks' loads and MMA chains interleave
+    auto run_stage = [&](auto full) {
+#pragma unroll
+    for (int b = 0; b < Geo::kSB; ++b) {
+      if (decltype(full)::value || b < nb) {
+        const int blk = b0 + b;
+        uint32_t wa[F], wb[F];
+        mp_read<F>(st + b * 16 * F, wa);
+        mp_read<F>(st + b * 16 * F + 8 * Geo::kPitch, wb);
+        float c1[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};
+        mp_block<F>(wa, wb, xs + (size_t)blk * 16, t4, c1, c2);
+        if (per_block) {
+          const float da = (c1[0] + c2[0] * MvScale2<F>::inv) * 16777216.f;
+          const float db = (c1[2] + c2[2] * MvScale2<F>::inv) * 16777216.f;
+          const float bx = sx[blk];
+          ya = fmaf(gsa[b], da - gza[b] * bx, ya);
+          yb = fmaf(gsb[b], db - gzb[b] * bx, yb);
+        } else {                                                          // one grid per row: the two factors' sums stay apart
+          ya += c1[0]; yb += c1[2]; ya2 += c2[0]; yb2 += c2[2];           // until the task ends
+        }
+      }
+    }
+    };
+    if (nb == Geo::kSB) run_stage(std::true_type{}); else run_stage(std::false_type{});
+    if (++cs == kDepth) cs = 0;
+    if (++j == nsub) {                                                    // the task is complete: combine the warps' partial sums
+      if (!per_block) {
+        ya = __ldg(scales + ra) * ((ya + ya2 * MvScale2<F>::inv) * 16777216.f - __ldg(zeros + ra) * xsum_w);
+        yb = __ldg(scales + rb) * ((yb + yb2 * MvScale2<F>::inv) * 16777216.f - __ldg(zeros + rb) * xsum_w);
+      }
+      float* rp = red + (par * kMpWarps + warp) * 16;
+      if (t4 == 0) { rp[gq] = ya; rp[gq + 8] = yb; }
+      __syncthreads();
+      if (threadIdx.x < 16) {
+        float t = 0.f;
+#pragma unroll
+        for (int w = 0; w < kMpWarps; ++w) t += red[(par * kMpWarps + w) * 16 + threadIdx.x];
+        const int r = task * 16 + threadIdx.x;
+        if (r < R) y[r] = t;
+      }
+      j = 0; ++k; par ^= 1; ya = yb = ya2 = yb2 = 0.f;
+    }
+  }
+  cp_async_wait<0>();
+}
+
 inline bool group_ok(int C, int g) { return g > 0 && C % g == 0 && (g % 32 == 0 || 32 % g == 0); }
 
 inline int device_sm_count_inference() {
@@ -402,6 +629,29 @@ gptq_status_t launch_matvec(const uint32_t* qweight, const float* scales, const 
   if (g == C || g % 128 == 0) {
     // tensor path: x staged as fp16
     const int n_blk = (C + 127) / 128;
+    // codes staged through shared memory when a row is a whole number of 16-byte pieces and the rings fit beside x
+    using Geo = gptq::MpGeom<F>;
+    const size_t fixed = (size_t)n_blk * 256 + (size_t)((n_blk + 3) & ~3) * sizeof(float) +
+                         (size_t)2 * gptq::kMpWarps * 16 * sizeof(float);
+    const size_t ring1 = (size_t)gptq::kMpWarps * Geo::kStageBytes, budget = 227 * 1024;
+    if (((int64_t)(C / 32) * F * 4) % 16 == 0 && gptq::aligned_to(qweight, 16) && fixed + 2 * ring1 <= budget) {
+      const int depth = fixed + 4 * ring1 <= budget ? 4 : fixed + 3 * ring1 <= budget ? 3 : 2;
+      const int bpw = (n_blk + gptq::kMpWarps - 1) / gptq::kMpWarps, nsub = (bpw + Geo::kSB - 1) / Geo::kSB,
+                sbk = (bpw + nsub - 1) / nsub;
+      const int tasks = (R + 15) / 16;
+      int grid = gptq::device_sm_count_inference();
+      if (grid > tasks) grid = tasks;
+      const size_t smem = fixed + depth * ring1;
+      auto go = [&](auto kern) -> gptq_status_t {
+        GPTQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        kern<<<grid, gptq::kMpThreads, smem, s>>>(qweight, scales, zeros, x, R, C, g, G, bpw, nsub, sbk, y);
+        GPTQ_LAUNCH_CHECK();
+        return GPTQ_OK;
+      };
+      if (depth == 4) return go(gptq::matvec_staged_kernel<F, 4>);
+      if (depth == 3) return go(gptq::matvec_staged_kernel<F, 3>);
+      return go(gptq::matvec_staged_kernel<F, 2>);
+    }
     const size_t smem = (size_t)n_blk * 128 * sizeof(__half) + (size_t)((n_blk + 3) & ~3) * sizeof(float) +
                         (size_t)2 * gptq::kMvWarps * 16 * sizeof(float);
     if (smem > 220 * 1024 / gptq::kMvCtasPerSm) return GPTQ_ERR_UNSUPPORTED;

@@ -452,6 +452,28 @@ def test_dequantize_and_matvec_match_oracle(B, bits, group, C):
     assert (np.abs(y - yref) <= bound).all(), float(np.max(np.abs(y - yref) / bound))
 
 
+@pytest.mark.parametrize("R,C,bits,group", [(5000, 6272, 4, 0), (2500, 12288, 3, 128), (4800, 8256, 2, 0), (2400, 5120, 8, 128),
+                                            (37, 4160, 4, 0), (2385, 49152, 4, 0), (2385, 16384, 3, 0), (300, 12288, 2, 128)])
+def test_matvec_over_several_row_tasks_and_stages_per_warp(B, bits, group, R, C):
+    """The tensor-core matvec with the codes staged through shared memory: more row tasks than CTAs (the rings run
+    across task boundaries), several stages per warp and task, a ragged last row task, a last block of 64 or 32 columns,
+    and x so long that the rings shrink to fewer stages.  Random codes and grids; oracle: the fp64 definition."""
+    r = np.random.default_rng(R + C + bits)
+    maxq = O.maxq_of(bits)
+    g = group if group > 0 else C
+    codes = r.integers(0, maxq + 1, size=(R, C))
+    scales = np.exp(r.normal(size=(R, C // g)) * 0.3).astype(np.float32).astype(np.float64) * 0.01
+    zeros = r.integers(0, maxq + 1, size=(R, C // g)).astype(np.float64)
+    x16 = r.normal(size=C).astype(np.float16)
+    qw = torch.from_numpy(O.pack_codes(codes, bits).view(np.int32)).cuda()
+    sc, zr = torch.from_numpy(scales.astype(np.float32)).cuda(), torch.from_numpy(zeros.astype(np.float32)).cuda()
+    y = B.gptq_matvec(qw, sc, zr, torch.from_numpy(x16).cuda(), C, bits, group).cpu().numpy().astype(np.float64)
+    yref = O.matvec(codes, scales.astype(np.float32).astype(np.float64), zeros, x16)
+    mag = np.repeat(scales, g, 1) * (codes + np.repeat(zeros, g, 1))
+    bound = 4e-6 * (mag @ np.abs(x16.astype(np.float64))) + 1e-12
+    assert (np.abs(y - yref) <= bound).all(), float(np.max(np.abs(y - yref) / bound))
+
+
 def test_block_pipeline_shares_hessian_and_factor_for_q_k_v(B, D):
     """Section 5, Setup: a block's layers are quantized from one pass of calibration inputs.  q, k and v read the same
     input, so the pipeline computes ONE Hessian and ONE factor for them; every member's outputs are bit-identical to
