@@ -406,18 +406,16 @@ matvec_mma_kernel(const uint32_t* __restrict__ qweight, const float* __restrict_
 // x is staged once per CTA, permuted as the unpacking wants it and interleaved inside a block: the 16-byte piece i
 // (0..3) of chunk t (0..3) sits at piece 4 i + t of the block, so that a warp's four lane groups read 64 consecutive
 // bytes.
-// 12 warps with rings of 3 stages (C = 12288, 4-bit) measured best: 8 warps leave issue slots idle, 16 warps leave room
-// for 2 stages only.
-#ifndef GPTQ_MP_WARPS
-#define GPTQ_MP_WARPS 12
-#endif
-constexpr int kMpWarps = GPTQ_MP_WARPS, kMpThreads = kMpWarps * 32;
-
+// 12 warps per SM with rings of 3 stages (4-bit) or 2 (3-bit, 2-bit at C = 12288) measured best: every warp waits on its
+// own chain copy -> fragment read -> mask -> MMA, so fewer warps leave issue slots idle, while more warps leave each ring
+// fewer or smaller stages and each warp fewer independent blocks to interleave (8, 16, 20, 24 warps: 3-10 % slower).
 template <int F> struct MpGeom {
+  static constexpr int kWarps = 12;                                           // warps per CTA (one CTA per SM)
+  static constexpr int kThreads = kWarps * 32;
   static constexpr int kSB = F == 4 ? 4 : F == 8 ? 2 : 8;                     // blocks per stage at most
   static constexpr int kPiecesPerRow = kSB * F;                               // 16-byte pieces of one row of a stage (<= 32)
   static constexpr int kRowsPerCopy = 32 / kPiecesPerRow;                     // rows one warp-wide copy instruction covers
-  static constexpr int kPad = F == 4 ? 64 : F == 3 ? 48 : F == 2 ? 32 : 16;   // makes the fragment reads conflict-free
+  static constexpr int kPad = F == 4 ? 64 : F == 3 ? 16 : F == 2 ? 32 : 16;   // makes the fragment reads conflict-free
   static constexpr int kPitch = (kSB * 16 * F + 127) / 128 * 128 + kPad;      // bytes between rows of a stage
   static constexpr int kStageBytes = 16 * kPitch;
 };
@@ -455,14 +453,15 @@ __device__ __forceinline__ void mp_block(const uint32_t (&wa)[F], const uint32_t
   mv_chunk<F>(wa, wb, xs, c1, c2);
 }
 
-// grid: min(tasks, SMs) CTAs of kMpThreads threads.  dynamic shared memory: x (fp16, C rounded up to 128), the block
-// sums of x (fp32), two buffers of partial sums, then kMpWarps rings of kDepth stages.
+// grid: min(tasks, SMs) CTAs of MpGeom<F>::kThreads threads.  dynamic shared memory: x (fp16, C rounded up to 128), the block
+// sums of x (fp32), two buffers of partial sums, then one ring of kDepth stages per warp.
 template <int F, int kDepth>
-__global__ void __launch_bounds__(kMpThreads, 1)
+__global__ void __launch_bounds__(MpGeom<F>::kThreads, 1)
 matvec_staged_kernel(const uint32_t* __restrict__ qweight, const float* __restrict__ scales, const float* __restrict__ zeros,
                      const __half* __restrict__ x, int R, int C, int g, int G, int bpw, int nsub, int sbk,
                      float* __restrict__ y) {
   using Geo = MpGeom<F>;
+  constexpr int kMpWarps = Geo::kWarps;
   extern __shared__ uint4 mv_smem[];
   const int chunks = C / 32, n_blk = (C + 127) / 128, Cpad = n_blk * 128;
   uint4* xs = mv_smem;                                                    // [n_blk][16] pieces
@@ -644,11 +643,11 @@ gptq_status_t launch_matvec(const uint32_t* qweight, const float* scales, const 
     // codes staged through shared memory when a row is a whole number of 16-byte pieces and the rings fit beside x
     using Geo = gptq::MpGeom<F>;
     const size_t fixed = (size_t)n_blk * 256 + (size_t)((n_blk + 3) & ~3) * sizeof(float) +
-                         (size_t)2 * gptq::kMpWarps * 16 * sizeof(float);
-    const size_t ring1 = (size_t)gptq::kMpWarps * Geo::kStageBytes, budget = 227 * 1024;
+                         (size_t)2 * Geo::kWarps * 16 * sizeof(float);
+    const size_t ring1 = (size_t)Geo::kWarps * Geo::kStageBytes, budget = 227 * 1024;
     if (((int64_t)(C / 32) * F * 4) % 16 == 0 && gptq::aligned_to(qweight, 16) && fixed + 2 * ring1 <= budget) {
       const int depth = fixed + 4 * ring1 <= budget ? 4 : fixed + 3 * ring1 <= budget ? 3 : 2;
-      const int bpw = (n_blk + gptq::kMpWarps - 1) / gptq::kMpWarps, nsub = (bpw + Geo::kSB - 1) / Geo::kSB,
+      const int bpw = (n_blk + Geo::kWarps - 1) / Geo::kWarps, nsub = (bpw + Geo::kSB - 1) / Geo::kSB,
                 sbk = (bpw + nsub - 1) / nsub;
       const int tasks = (R + 15) / 16;
       int grid = gptq::device_sm_count_inference();
@@ -656,7 +655,7 @@ gptq_status_t launch_matvec(const uint32_t* qweight, const float* scales, const 
       const size_t smem = fixed + depth * ring1;
       auto go = [&](auto kern) -> gptq_status_t {
         GPTQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        kern<<<grid, gptq::kMpThreads, smem, s>>>(qweight, scales, zeros, x, R, C, g, G, bpw, nsub, sbk, y);
+        kern<<<grid, Geo::kThreads, smem, s>>>(qweight, scales, zeros, x, R, C, g, G, bpw, nsub, sbk, y);
         GPTQ_LAUNCH_CHECK();
         return GPTQ_OK;
       };
