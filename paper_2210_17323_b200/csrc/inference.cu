@@ -406,18 +406,31 @@ matvec_mma_kernel(const uint32_t* __restrict__ qweight, const float* __restrict_
 // x is staged once per CTA, permuted as the unpacking wants it and interleaved inside a block: the 16-byte piece i
 // (0..3) of chunk t (0..3) sits at piece 4 i + t of the block, so that a warp's four lane groups read 64 consecutive
 // bytes.
-// 12 warps per SM with rings of 3 stages (4-bit) or 2 (3-bit, 2-bit at C = 12288) measured best: every warp waits on its
-// own chain copy -> fragment read -> mask -> MMA, so fewer warps leave issue slots idle, while more warps leave each ring
-// fewer or smaller stages and each warp fewer independent blocks to interleave (8, 16, 20, 24 warps: 3-10 % slower).
-template <int F> struct MpGeom {
-  static constexpr int kWarps = 12;                                           // warps per CTA (one CTA per SM)
+// Every warp waits on its own chain copy -> fragment read -> mask -> MMA, so the kernel lives on independent work inside a
+// warp (blocks per stage, all unrolled) and on warps per SM, and both cost ring memory.  Measured at C = 12288 (49152
+// rows): 4-bit 14 warps x 2 stages of 7 blocks 63 us; 12 x 3 x 4 blocks 67; 16 x 4 x 3 blocks 75; 8 x 4 x 4 blocks 71;
+// 3-bit 12 x 2 x 8 blocks 82; 12 x 4 x 4 blocks 85; 10 x 2 x 10 blocks 87; 16 x 2 x 6 blocks 83.  A long x leaves less
+// room: the launcher takes the first geometry of a short list that fits.
+// smallest pitch >= the row's bytes that keeps a warp's fragment reads on distinct banks: 4-bit (one 16-byte read per
+// lane, two rows per quarter warp) wants the rows 64 bytes apart modulo 128, 2-bit (8-byte reads, four rows per half
+// warp) 32 modulo 128, 3-bit (4-byte reads, eight rows per warp) and 8-bit (two 16-byte reads) 16 modulo 32.
+constexpr int mp_pitch(int F, int row_bytes) {
+  const int m = F == 4 ? 128 : F == 2 ? 128 : 32, want = F == 4 ? 64 : F == 2 ? 32 : 16;
+  int p = (row_bytes + 15) / 16 * 16;
+  while (p % m != want) p += 16;
+  return p;
+}
+// W warps per CTA (one CTA per SM), stages of at most SB blocks.
+template <int F_, int W, int SB> struct MpGeom {
+  static constexpr int F = F_;
+  static constexpr int kWarps = W;
   static constexpr int kThreads = kWarps * 32;
-  static constexpr int kSB = F == 4 ? 4 : F == 8 ? 2 : 8;                     // blocks per stage at most
+  static constexpr int kSB = SB;
   static constexpr int kPiecesPerRow = kSB * F;                               // 16-byte pieces of one row of a stage (<= 32)
   static constexpr int kRowsPerCopy = 32 / kPiecesPerRow;                     // rows one warp-wide copy instruction covers
-  static constexpr int kPad = F == 4 ? 64 : F == 3 ? 16 : F == 2 ? 32 : 16;   // makes the fragment reads conflict-free
-  static constexpr int kPitch = (kSB * 16 * F + 127) / 128 * 128 + kPad;      // bytes between rows of a stage
+  static constexpr int kPitch = mp_pitch(F, kSB * 16 * F);                    // bytes between rows of a stage
   static constexpr int kStageBytes = 16 * kPitch;
+  static_assert(kPiecesPerRow <= 32 && kSB <= 10, "a row of a stage is copied by one warp instruction");
 };
 
 __device__ __forceinline__ void cp_async_16(uint32_t sdst, const void* gsrc, uint32_t src_bytes) {
@@ -453,14 +466,14 @@ __device__ __forceinline__ void mp_block(const uint32_t (&wa)[F], const uint32_t
   mv_chunk<F>(wa, wb, xs, c1, c2);
 }
 
-// grid: min(tasks, SMs) CTAs of MpGeom<F>::kThreads threads.  dynamic shared memory: x (fp16, C rounded up to 128), the block
+// grid: min(tasks, SMs) CTAs of Geo::kThreads threads.  dynamic shared memory: x (fp16, C rounded up to 128), the block
 // sums of x (fp32), two buffers of partial sums, then one ring of kDepth stages per warp.
-template <int F, int kDepth>
-__global__ void __launch_bounds__(MpGeom<F>::kThreads, 1)
+template <class Geo, int kDepth>
+__global__ void __launch_bounds__(Geo::kThreads, 1)
 matvec_staged_kernel(const uint32_t* __restrict__ qweight, const float* __restrict__ scales, const float* __restrict__ zeros,
                      const __half* __restrict__ x, int R, int C, int g, int G, int bpw, int nsub, int sbk,
                      float* __restrict__ y) {
-  using Geo = MpGeom<F>;
+  constexpr int F = Geo::F;
   constexpr int kMpWarps = Geo::kWarps;
   extern __shared__ uint4 mv_smem[];
   const int chunks = C / 32, n_blk = (C + 127) / 128, Cpad = n_blk * 128;
@@ -497,7 +510,7 @@ matvec_staged_kernel(const uint32_t* __restrict__ qweight, const float* __restri
           const unsigned char* src = qbytes + (int64_t)(task * 16 + c_row) * row_bytes + col_off;
 #pragma unroll
           for (int r = 0; r < 16; r += Geo::kRowsPerCopy) {
-            cp_async_16(dst, src, fill);
+            if (16 % Geo::kRowsPerCopy == 0 || r + c_row < 16) cp_async_16(dst, src, fill);
             src += Geo::kRowsPerCopy * row_bytes;
             dst += Geo::kRowsPerCopy * Geo::kPitch;
           }
@@ -505,7 +518,7 @@ matvec_staged_kernel(const uint32_t* __restrict__ qweight, const float* __restri
 #pragma unroll
           for (int r = 0; r < 16; r += Geo::kRowsPerCopy) {
             const int row = min(task * 16 + r + c_row, R - 1);
-            cp_async_16(dst, qbytes + row * row_bytes + col_off, fill);
+            if (16 % Geo::kRowsPerCopy == 0 || r + c_row < 16) cp_async_16(dst, qbytes + row * row_bytes + col_off, fill);
             dst += Geo::kRowsPerCopy * Geo::kPitch;
           }
         }
@@ -541,6 +554,7 @@ matvec_staged_kernel(const uint32_t* __restrict__ qweight, const float* __restri
 
   int k = 0, j = 0, cs = 0, par = 0;
   float ya = 0.f, yb = 0.f, ya2 = 0.f, yb2 = 0.f;
+  float rsa = 0.f, rza = 0.f, rsb = 0.f, rzb = 0.f;                       // per-row grids: this task's scale and zero, rows a and b
   float xsum_w = 0.f;                                                     // sum of x over this warp's blocks (the same for every task)
   for (int b = blk_lo; b < blk_hi; ++b) xsum_w += sx[b];
   const int total = my_tasks * nsub;
@@ -550,6 +564,10 @@ matvec_staged_kernel(const uint32_t* __restrict__ qweight, const float* __restri
     const int b0 = blk_lo + j * sbk, nb = min(sbk, blk_hi - b0);
     // grouped grids: the stage's scales and zero-points are requested before the wait for its codes
     float gsa[Geo::kSB], gza[Geo::kSB], gsb[Geo::kSB], gzb[Geo::kSB];
+    if (!per_block && j == 0) {                                           // one grid per row: asked for when the task begins,
+      rsa = __ldg(scales + ra); rza = __ldg(zeros + ra);                  // used when it ends
+      rsb = __ldg(scales + rb); rzb = __ldg(zeros + rb);
+    }
     if (per_block) {
 #pragma unroll
       for (int b = 0; b < Geo::kSB; ++b) {
@@ -564,11 +582,11 @@ matvec_staged_kernel(const uint32_t* __restrict__ qweight, const float* __restri
     __syncwarp();                                                         // ... and every lane's; the previous stage is read
     issue();                                                              // refill the slot read in the previous iteration
     const unsigned char* st = ring + (size_t)cs * Geo::kStageBytes + gq * Geo::kPitch + t4 * (4 * F);
-    // a full stage runs without per-block branches, so that the blocks' loads and MMA chains interleave
-    auto run_stage = [&](auto full) {
+    // one instance per block count, without per-block branches, so that the blocks' loads and MMA chains interleave
+    auto run_stage = [&](auto count) {
 #pragma unroll
     for (int b = 0; b < Geo::kSB; ++b) {
-      if (decltype(full)::value || b < nb) {
+      if (b < decltype(count)::value) {
         const int blk = b0 + b;
         uint32_t wa[F], wb[F];
         mp_read<F>(st + b * 16 * F, wa);
@@ -587,12 +605,24 @@ matvec_staged_kernel(const uint32_t* __restrict__ qweight, const float* __restri
       }
     }
     };
-    if (nb == Geo::kSB) run_stage(std::true_type{}); else run_stage(std::false_type{});
+    switch (nb) {                                                         // (uniform over the warp)
+      case 10: if constexpr (Geo::kSB >= 10) run_stage(std::integral_constant<int, 10>{}); break;
+      case 9: if constexpr (Geo::kSB >= 9) run_stage(std::integral_constant<int, 9>{}); break;
+      case 8: if constexpr (Geo::kSB >= 8) run_stage(std::integral_constant<int, 8>{}); break;
+      case 7: if constexpr (Geo::kSB >= 7) run_stage(std::integral_constant<int, 7>{}); break;
+      case 6: if constexpr (Geo::kSB >= 6) run_stage(std::integral_constant<int, 6>{}); break;
+      case 5: if constexpr (Geo::kSB >= 5) run_stage(std::integral_constant<int, 5>{}); break;
+      case 4: if constexpr (Geo::kSB >= 4) run_stage(std::integral_constant<int, 4>{}); break;
+      case 3: if constexpr (Geo::kSB >= 3) run_stage(std::integral_constant<int, 3>{}); break;
+      case 2: if constexpr (Geo::kSB >= 2) run_stage(std::integral_constant<int, 2>{}); break;
+      case 1: run_stage(std::integral_constant<int, 1>{}); break;
+      default: break;
+    }
     if (++cs == kDepth) cs = 0;
     if (++j == nsub) {                                                    // the task is complete: combine the warps' partial sums
       if (!per_block) {
-        ya = __ldg(scales + ra) * ((ya + ya2 * MvScale2<F>::inv) * 16777216.f - __ldg(zeros + ra) * xsum_w);
-        yb = __ldg(scales + rb) * ((yb + yb2 * MvScale2<F>::inv) * 16777216.f - __ldg(zeros + rb) * xsum_w);
+        ya = rsa * ((ya + ya2 * MvScale2<F>::inv) * 16777216.f - rza * xsum_w);
+        yb = rsb * ((yb + yb2 * MvScale2<F>::inv) * 16777216.f - rzb * xsum_w);
       }
       float* rp = red + (par * kMpWarps + warp) * 16;
       if (t4 == 0) { rp[gq] = ya; rp[gq + 8] = yb; }
@@ -640,28 +670,45 @@ gptq_status_t launch_matvec(const uint32_t* qweight, const float* scales, const 
   if (g == C || g % 128 == 0) {
     // tensor path: x staged as fp16
     const int n_blk = (C + 127) / 128;
-    // codes staged through shared memory when a row is a whole number of 16-byte pieces and the rings fit beside x
-    using Geo = gptq::MpGeom<F>;
-    const size_t fixed = (size_t)n_blk * 256 + (size_t)((n_blk + 3) & ~3) * sizeof(float) +
-                         (size_t)2 * Geo::kWarps * 16 * sizeof(float);
-    const size_t ring1 = (size_t)Geo::kWarps * Geo::kStageBytes, budget = 227 * 1024;
-    if (((int64_t)(C / 32) * F * 4) % 16 == 0 && gptq::aligned_to(qweight, 16) && fixed + 2 * ring1 <= budget) {
-      const int depth = fixed + 4 * ring1 <= budget ? 4 : fixed + 3 * ring1 <= budget ? 3 : 2;
-      const int bpw = (n_blk + Geo::kWarps - 1) / Geo::kWarps, nsub = (bpw + Geo::kSB - 1) / Geo::kSB,
-                sbk = (bpw + nsub - 1) / nsub;
-      const int tasks = (R + 15) / 16;
-      int grid = gptq::device_sm_count_inference();
-      if (grid > tasks) grid = tasks;
-      const size_t smem = fixed + depth * ring1;
-      auto go = [&](auto kern) -> gptq_status_t {
-        GPTQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        kern<<<grid, Geo::kThreads, smem, s>>>(qweight, scales, zeros, x, R, C, g, G, bpw, nsub, sbk, y);
-        GPTQ_LAUNCH_CHECK();
-        return GPTQ_OK;
+    // codes staged through shared memory when a row is a whole number of 16-byte pieces and rings of at least two stages
+    // fit beside x: the first geometry that fits, from the one measured best at C = 12288 to smaller rings
+    if (((int64_t)(C / 32) * F * 4) % 16 == 0 && gptq::aligned_to(qweight, 16)) {
+      bool launched = false;
+      auto attempt = [&](auto geo) -> gptq_status_t {
+        using Geo = decltype(geo);
+        const size_t fixed = (size_t)n_blk * 256 + (size_t)((n_blk + 3) & ~3) * sizeof(float) +
+                             (size_t)2 * Geo::kWarps * 16 * sizeof(float);
+        const size_t ring1 = (size_t)Geo::kWarps * Geo::kStageBytes, budget = 227 * 1024;
+        if (fixed + 2 * ring1 > budget) return GPTQ_OK;                   // does not fit: the caller tries the next one
+        const int depth = fixed + 4 * ring1 <= budget ? 4 : fixed + 3 * ring1 <= budget ? 3 : 2;
+        const int bpw = (n_blk + Geo::kWarps - 1) / Geo::kWarps, nsub = (bpw + Geo::kSB - 1) / Geo::kSB,
+                  sbk = (bpw + nsub - 1) / nsub;
+        const int tasks = (R + 15) / 16;
+        int grid = gptq::device_sm_count_inference();
+        if (grid > tasks) grid = tasks;
+        const size_t smem = fixed + depth * ring1;
+        auto go = [&](auto kern) -> gptq_status_t {
+          GPTQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+          kern<<<grid, Geo::kThreads, smem, s>>>(qweight, scales, zeros, x, R, C, g, G, bpw, nsub, sbk, y);
+          GPTQ_LAUNCH_CHECK();
+          launched = true;
+          return GPTQ_OK;
+        };
+        if (depth == 4) return go(gptq::matvec_staged_kernel<Geo, 4>);
+        if (depth == 3) return go(gptq::matvec_staged_kernel<Geo, 3>);
+        return go(gptq::matvec_staged_kernel<Geo, 2>);
       };
-      if (depth == 4) return go(gptq::matvec_staged_kernel<F, 4>);
-      if (depth == 3) return go(gptq::matvec_staged_kernel<F, 3>);
-      return go(gptq::matvec_staged_kernel<F, 2>);
+      gptq_status_t st = GPTQ_OK;
+      if constexpr (F == 4) {
+        st = attempt(gptq::MpGeom<4, 14, 7>{});
+        if (st == GPTQ_OK && !launched) st = attempt(gptq::MpGeom<4, 12, 4>{});
+      } else if constexpr (F == 8) {
+        st = attempt(gptq::MpGeom<8, 12, 2>{});
+      } else {
+        st = attempt(gptq::MpGeom<F, 12, 8>{});
+        if (st == GPTQ_OK && !launched) st = attempt(gptq::MpGeom<F, 12, 4>{});
+      }
+      if (st != GPTQ_OK || launched) return st;
     }
     const size_t smem = (size_t)n_blk * 128 * sizeof(__half) + (size_t)((n_blk + 3) & ~3) * sizeof(float) +
                         (size_t)2 * gptq::kMvWarps * 16 * sizeof(float);
