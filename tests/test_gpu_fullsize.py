@@ -137,3 +137,35 @@ def test_config4_block_size_sweep_full_size(B):
             per_row = ref["loss"] / len(rows)
             assert 0.5 * per_row * L.R <= out["loss"].item() <= 2.0 * per_row * L.R
             print(f"c4 bits={g.bits} B={blk}:", figs, "words identical to B=32:", 1.0 if base is qw else same)
+
+
+@pytest.mark.parametrize("cfg,kind,bits,group", [(3, "fc1", 4, 0), (3, "fc1", 3, 0), (3, "fc2", 4, 0), (4, "fc1", 2, 128)])
+def test_inference_kernels_sampled_rows_full_size(B, cfg, kind, bits, group):
+    """gptq_rtn_layer, gptq_matvec and gptq_dequantize on the layers `bench.py --mode inference` times (49152 x 12288,
+    12288 x 49152, 57344 x 14336), checked on sampled rows: the oracle rounds the host-generated rows to the grid itself
+    (its codes and grids must equal the packed ones bit for bit), then the matvec is compared with the fp64 definition
+    and the dequantized rows bit for bit."""
+    from paper_2210_17323_b200.synth import device as D
+    L = [l for l in WL.workload(cfg).layers if l.kind == kind][0]
+    q = B.gptq_rtn_layer(D.fill_w(L), bits, group, False)
+    r = np.random.default_rng(11 + cfg + bits)
+    rows = np.unique(np.concatenate([[0, 1, 15, 16, L.R - 17, L.R - 16, L.R - 1], r.integers(0, L.R, 40)]))
+    W16 = L.w(rows=rows)
+    codes, _ = O.rtn(W16, bits, group, False)
+    g = group if group > 0 else L.C
+    grids = [O.find_params(W16[:, j:j + g].astype(np.float64), bits, False) for j in range(0, L.C, g)]
+    scales, zeros = np.stack([s for s, _ in grids], 1), np.stack([z for _, z in grids], 1)
+    idx = torch.from_numpy(rows).cuda()
+    assert np.array_equal(O.unpack_codes(q["qweight"][idx].cpu().numpy().view(np.uint32), bits, L.C), codes)
+    assert np.array_equal(q["scales"][idx].cpu().numpy().astype(np.float64), scales)
+    assert np.array_equal(q["zeros"][idx].cpu().numpy().astype(np.float64), zeros)
+    x16 = r.normal(size=L.C).astype(np.float16)
+    y = B.gptq_matvec(q["qweight"], q["scales"], q["zeros"], torch.from_numpy(x16).cuda(), L.C, bits, group)
+    yref = O.matvec(codes, scales, zeros, x16)
+    mag = np.repeat(scales, g, 1) * (codes + np.repeat(zeros, g, 1))
+    bound = 4e-6 * (mag @ np.abs(x16.astype(np.float64))) + 1e-12          # as in test_dequantize_and_matvec_match_oracle
+    err = np.abs(y[idx].cpu().numpy().astype(np.float64) - yref)
+    assert (err <= bound).all(), float(np.max(err / bound))
+    deq = B.gptq_dequantize(q["qweight"], q["scales"], q["zeros"], L.C, bits, group)
+    ref16 = O.dequantize(codes, scales, zeros, to_fp16=True)
+    assert np.array_equal(deq[idx].cpu().numpy().view(np.uint16), ref16.view(np.uint16))
