@@ -497,3 +497,29 @@ def test_residuals_through_the_factor_give_the_lazy_update(bits, group):
         lazy = out["E"][:, :j0] @ U[:j0, J]
         through_factor = -(Rm[:, :j0] @ Ut[:j0, J]) @ U[J, J]
         assert np.allclose(lazy, through_factor, rtol=1e-8, atol=1e-12)
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
+def test_symmetric_grid_puts_minus_max_on_a_tie(bits):
+    """The symmetric option (not defined by the paper): scale = 2a / maxq and zero = (maxq + 1) / 2 with an even number of
+    levels put -a exactly midway between codes 0 and 1, so in real arithmetic both are nearest; which one the oracle
+    returns follows the fp32 rounding of the scale.  Over many values of a both codes occur, the chosen grid value is
+    always one of the two nearest, and +a (which maps past the top level) always clamps to maxq.  This is why GPU parity
+    for symmetric grids compares rows only up to the first such tie."""
+    maxq = O.maxq_of(bits)
+    r = np.random.default_rng(bits)
+    a = np.exp(r.normal(size=4000)).astype(np.float16).astype(np.float64)
+    lo = np.stack([-a, 0.25 * a], 1)                         # the row's largest magnitude is negative
+    scale, zero = O.find_params(lo, bits, True)
+    assert np.array_equal(zero, np.full_like(zero, (maxq + 1) // 2))
+    assert np.array_equal(scale, (2.0 * a / maxq).astype(np.float32).astype(np.float64))
+    q, wq = O.quant(lo[:, 0], scale, zero, maxq)
+    assert set(np.unique(q)) == {0.0, 1.0}                   # both sides of the tie occur
+    exact = -a / (2.0 * a / maxq) + (maxq + 1) // 2          # position of -a on the exact grid
+    assert np.allclose(exact, 0.5)
+    d0, d1 = np.abs(lo[:, 0] - scale * (0 - zero)), np.abs(lo[:, 0] - scale * (1 - zero))
+    assert np.all(np.abs(d0 - d1) <= 1e-6 * a)               # equally near up to the scale's rounding
+    assert np.all(np.abs(lo[:, 0] - wq) <= np.minimum(d0, d1) + 1e-12)
+    hi = np.stack([a, -0.25 * a], 1)                         # largest magnitude positive: past the top level, clamped
+    scale, zero = O.find_params(hi, bits, True)
+    assert np.array_equal(O.quant(hi[:, 0], scale, zero, maxq)[0], np.full(len(a), float(maxq)))
