@@ -242,14 +242,17 @@ gptq_status_t gptq_rtn_layer(const void* W_fp16, int R, int C, int bits, int gro
  * group_size as in gptq_quantize_layer (<= 0: per row); 4, 8, 16 or a multiple of 32.
  *
  * gptq_dequantize: the whole matrix back to fp16 (round-to-nearest-even of the fp32 product).
- *   W_out_fp16 [R x C] half.
+ *   W_out_fp16 [R x C] half, starting on a 16-byte boundary (GPTQ_ERR_INVALID_ARG otherwise).
  * gptq_matvec: y = W^ x for ONE fp16 vector x (batch-1 generation: packed matrix times
  *   fp16 vector with dequantization on the fly, never materialising W^).
  *   x_fp16 [C] half, y [R] fp32; products exact, sums in fp32: per group the kernel forms
  *   sum q x and zero * sum x and combines them with the scale, so its rounding error is
  *   fp32-level relative to sum scale * (q + zero) * |x|.  Per-row grids and group sizes that
  *   are multiples of 128 run on the tensor cores (mma.sync f16), other group sizes on the
- *   CUDA cores.  C <= 51200 (x is staged in shared memory), else GPTQ_ERR_UNSUPPORTED. */
+ *   CUDA cores.  C <= 51200 (x is staged in shared memory), else GPTQ_ERR_UNSUPPORTED; x and qweight
+ *   must start on 16-byte boundaries (GPTQ_ERR_INVALID_ARG otherwise).  The tensor-core path moves
+ *   the codes through shared-memory rings when a packed row is a whole number of 16-byte pieces,
+ *   and through registers otherwise; the results are the same. */
 gptq_status_t gptq_dequantize(const uint32_t* qweight, const float* scales, const float* zeros,
                               int R, int C, int bits, int group_size, void* W_out_fp16, void* stream);
 gptq_status_t gptq_matvec(const uint32_t* qweight, const float* scales, const float* zeros,

@@ -672,7 +672,7 @@ gptq_status_t launch_matvec(const uint32_t* qweight, const float* scales, const 
     const int n_blk = (C + 127) / 128;
     // codes staged through shared memory when a row is a whole number of 16-byte pieces and rings of at least two stages
     // fit beside x: the first geometry that fits, from the one measured best at C = 12288 to smaller rings
-    if (((int64_t)(C / 32) * F * 4) % 16 == 0 && gptq::aligned_to(qweight, 16)) {
+    if (((int64_t)(C / 32) * F * 4) % 16 == 0) {
       bool launched = false;
       auto attempt = [&](auto geo) -> gptq_status_t {
         using Geo = decltype(geo);
@@ -735,6 +735,7 @@ extern "C" gptq_status_t gptq_dequantize(const uint32_t* qweight, const float* s
                                          int R, int C, int bits, int group_size, void* W_out_fp16, void* stream) {
   using namespace gptq;
   if (!qweight || !scales || !zeros || !W_out_fp16 || R <= 0 || C <= 0 || C % 32 != 0) return GPTQ_ERR_INVALID_ARG;
+  if (!aligned_to(W_out_fp16, 16) || !aligned_to(qweight, 4)) return GPTQ_ERR_INVALID_ARG;   // 16-byte stores, 4-byte loads
   const int g = group_size > 0 ? group_size : C;
   if (!group_ok(C, g)) return GPTQ_ERR_UNSUPPORTED;
   const int f = bits == GPTQ_BITS_TERNARY ? 2 : bits, G = C / g;
@@ -754,6 +755,7 @@ extern "C" gptq_status_t gptq_matvec(const uint32_t* qweight, const float* scale
                                      void* stream) {
   using namespace gptq;
   if (!qweight || !scales || !zeros || !x_fp16 || !y || R <= 0 || C <= 0 || C % 32 != 0) return GPTQ_ERR_INVALID_ARG;
+  if (!aligned_to(x_fp16, 16) || !aligned_to(qweight, 16)) return GPTQ_ERR_INVALID_ARG;   // both are read in 16-byte pieces
   const int g = group_size > 0 ? group_size : C;
   if (!group_ok(C, g)) return GPTQ_ERR_UNSUPPORTED;
   if (C > 51200) return GPTQ_ERR_UNSUPPORTED;   // x is staged in shared memory (4 bytes per column)

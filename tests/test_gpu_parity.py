@@ -474,6 +474,24 @@ def test_matvec_over_several_row_tasks_and_stages_per_warp(B, bits, group, R, C)
     assert (np.abs(y - yref) <= bound).all(), float(np.max(np.abs(y - yref) / bound))
 
 
+def test_matvec_rejects_misaligned_operands(B):
+    """x and the packed matrix are read in 16-byte pieces: operands that start elsewhere are refused at the call, before
+    anything is launched."""
+    R, C, bits = 70, 1024, 4
+    packed = torch.zeros(R * C // 8 + 4, dtype=torch.int32, device="cuda")
+    sc, zr = torch.ones((R, 1), device="cuda"), torch.zeros((R, 1), device="cuda")
+    xbuf = torch.zeros(C + 8, dtype=torch.float16, device="cuda")
+    y = torch.empty(R, dtype=torch.float32, device="cuda")
+    n0 = B.gptq_launch_count()
+    st = B._lib.gptq_matvec(packed.data_ptr(), sc.data_ptr(), zr.data_ptr(), xbuf.data_ptr() + 2, R, C, bits, 0, y.data_ptr(), None)
+    assert st == B.ERR_INVALID_ARG
+    st = B._lib.gptq_matvec(packed.data_ptr() + 4, sc.data_ptr(), zr.data_ptr(), xbuf.data_ptr(), R, C, bits, 0, y.data_ptr(), None)
+    assert st == B.ERR_INVALID_ARG
+    assert B.gptq_launch_count() == n0
+    assert B._lib.gptq_matvec(packed.data_ptr(), sc.data_ptr(), zr.data_ptr(), xbuf.data_ptr(), R, C, bits, 0, y.data_ptr(), None) == 0
+    torch.cuda.synchronize()
+
+
 def test_block_pipeline_shares_hessian_and_factor_for_q_k_v(B, D):
     """Section 5, Setup: a block's layers are quantized from one pass of calibration inputs.  q, k and v read the same
     input, so the pipeline computes ONE Hessian and ONE factor for them; every member's outputs are bit-identical to
