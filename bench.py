@@ -688,8 +688,9 @@ def run_e2e(args, wl, state, device_value):
 
 
 def run_inference(args, wl):
-    """Bandwidth of the inference-side kernels (packed-matrix x fp16-vector, whole-matrix dequantization) on the
-    workload's largest layer, quantized with the RTN entry point (the kernels' speed does not depend on the codes)."""
+    """Bandwidth of the inference-side kernels (packed-matrix x fp16-vector, whole-matrix dequantization) and of the
+    round-to-nearest entry point on the workload's largest layer, quantized with that entry point (the kernels' speed does
+    not depend on the codes)."""
     import torch
     from paper_2210_17323_b200 import binding as B
     from paper_2210_17323_b200.synth import device as D
@@ -711,7 +712,10 @@ def run_inference(args, wl):
         n_rot = max(2, -(-3 * L2_BYTES // (q["qweight"].numel() * 4)))
         qws = [q["qweight"]] + [q["qweight"].clone() for _ in range(n_rot - 1)]
         res = {}
+        Ws = [W] + [W.clone() for _ in range(max(1, -(-3 * L2_BYTES // (W.numel() * 2))) - 1)]   # rotated like the codes
         for name, fn, nbytes in (
+                ("rtn", lambda i: B.gptq_rtn_layer(Ws[i % len(Ws)], g.bits, g.group_size, g.sym),
+                 W.numel() * 2 + q["qweight"].numel() * 4 + q["scales"].numel() * 8),
                 ("matvec", lambda i: B.gptq_matvec(qws[i % n_rot], q["scales"], q["zeros"], x, L.C, g.bits, g.group_size, out=y),
                  q["qweight"].numel() * 4 + q["scales"].numel() * 8 + L.C * 2 + L.R * 4),
                 ("dequantize", lambda i: B.gptq_dequantize(qws[i % n_rot], q["scales"], q["zeros"], L.C, g.bits, g.group_size, out=out),
@@ -731,7 +735,7 @@ def run_inference(args, wl):
             ms = statistics.median(ts)
             res[name] = dict(ms=ms, gbs=nbytes / ms / 1e6, frac_of_hbm=nbytes / ms / 1e6 / peaks["hbm_gbs"], bytes=nbytes)
         rows.append(dict(bits=g.bits, group_size=g.group_size, **res))
-        del qws
+        del qws, Ws
     line = dict(metric="gptq_inference_kernel_bandwidth", unit="GB/s", value=rows[0]["matvec"]["gbs"], n_gpus=1,
                 higher_is_better=True, data="synthetic", dtype="packed codes -> f32 accumulate",
                 config=dict(workload=wl.name, layer=L.name,
