@@ -194,7 +194,7 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a
 template <int F>
 __host__ __device__ constexpr int mv_perm(int p) {
   if (F == 4) { constexpr int o[8] = {0, 4, 2, 6, 1, 5, 3, 7}; return (p & ~7) + o[p & 7]; }
-  if (F == 2) { constexpr int o[16] = {0, 8, 2, 10, 4, 12, 6, 14, 1, 9, 3, 11, 5, 13, 7, 15}; return (p & ~15) + o[p & 15]; }
+  if (F == 2) { constexpr int o[16] = {0, 8, 4, 12, 1, 9, 5, 13, 2, 10, 6, 14, 3, 11, 7, 15}; return (p & ~15) + o[p & 15]; }
   if (F == 8) { constexpr int o[4] = {0, 2, 1, 3}; return (p & ~3) + o[p & 3]; }
   { constexpr int o[8] = {0, 1, 4, 5, 2, 3, 6, 7}; return (p & ~7) + o[p & 7]; }            // 3-bit
 }
@@ -223,15 +223,20 @@ __device__ __forceinline__ void mv_chunk<4>(const uint32_t (&wa)[4], const uint3
 template <>
 __device__ __forceinline__ void mv_chunk<2>(const uint32_t (&wa)[2], const uint32_t (&wb)[2], const uint4* xs,
                                             float (&c1)[4], float (&c2)[4]) {
+  // a 2-bit field may start at bit 0, 2, 4 or 6 of a half and still be an fp16 subnormal: four factors (1, 4, 16, 64), one
+  // shift per word.  The factors 16 and 64 are summed apart and folded into the first two accumulators at the end.
+  float c3[4] = {0.f, 0.f, 0.f, 0.f}, c4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-  for (int i = 0; i < 2; ++i) {          // word i, t_s = w >> 4s: codes (2s, 2s+8) at factor 1, (2s+1, 2s+9) at factor 4
+  for (int i = 0; i < 2; ++i) {          // word i, v in {w, w >> 8}: field s of v holds codes (s / 2 [+ 4], 8 + s / 2 [+ 4])
     const uint4 x0 = xs[2 * i], x1 = xs[2 * i + 1];
-    const uint32_t a = wa[i], b = wb[i], a4 = a >> 4, b4 = b >> 4, a8 = a >> 8, b8 = b >> 8, a12 = a >> 12, b12 = b >> 12;
-    mma_16816(c1, a & 0x00030003u, b & 0x00030003u, a4 & 0x00030003u, b4 & 0x00030003u, x0.x, x0.y);
-    mma_16816(c1, a8 & 0x00030003u, b8 & 0x00030003u, a12 & 0x00030003u, b12 & 0x00030003u, x0.z, x0.w);
-    mma_16816(c2, a & 0x000C000Cu, b & 0x000C000Cu, a4 & 0x000C000Cu, b4 & 0x000C000Cu, x1.x, x1.y);
-    mma_16816(c2, a8 & 0x000C000Cu, b8 & 0x000C000Cu, a12 & 0x000C000Cu, b12 & 0x000C000Cu, x1.z, x1.w);
+    const uint32_t a = wa[i], b = wb[i], a8 = a >> 8, b8 = b >> 8;
+    mma_16816(c1, a & 0x00030003u, b & 0x00030003u, a8 & 0x00030003u, b8 & 0x00030003u, x0.x, x0.y);
+    mma_16816(c2, a & 0x000C000Cu, b & 0x000C000Cu, a8 & 0x000C000Cu, b8 & 0x000C000Cu, x0.z, x0.w);
+    mma_16816(c3, a & 0x00300030u, b & 0x00300030u, a8 & 0x00300030u, b8 & 0x00300030u, x1.x, x1.y);
+    mma_16816(c4, a & 0x00C000C0u, b & 0x00C000C0u, a8 & 0x00C000C0u, b8 & 0x00C000C0u, x1.z, x1.w);
   }
+  c1[0] = fmaf(c3[0], 1.f / 16.f, c1[0]); c1[2] = fmaf(c3[2], 1.f / 16.f, c1[2]);
+  c2[0] = fmaf(c4[0], 1.f / 16.f, c2[0]); c2[2] = fmaf(c4[2], 1.f / 16.f, c2[2]);
 }
 
 template <>
