@@ -21,6 +21,11 @@ import sys
 import threading
 import time
 
+# The overlapped schedule keeps about fifteen streams busy (one chain per layer, one more per extra grid, the library's
+# own side streams).  With the default of 8 hardware queues several of them share a queue and wait for each other's
+# kernels; the setting is read when the CUDA context is created, so it has to be in the environment before torch starts.
+os.environ.setdefault("CUDA_DEVICE_MAX_CONNECTIONS", "32")
+
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
@@ -266,6 +271,17 @@ def run_gpu(args, wl):
     order = sorted(range(len(state)), key=lambda i: -(state[i]["L"].C ** 2) * (state[i]["L"].n_tokens + state[i]["L"].C))
     main = torch.cuda.Stream(device=dev)
     chain_streams = [torch.cuda.Stream(device=dev) if overlap else main for _ in state]
+    # A layer's grids are independent once its factor exists: in the overlapped schedule every grid after the first gets
+    # a stream and a stage-3 workspace of its own, so one grid's column chains run beside the other's lazy-update GEMMs.
+    side_grids = overlap and not args.grids_in_turn and len(wl.grids) > 1
+    for st in state:
+        st["ws_g"] = [st["ws"]] * len(wl.grids)
+        st["grid_streams"] = []
+        if side_grids:
+            L = st["L"]
+            st["ws_g"] = [st["ws"]] + [torch.empty(max(256, B.gptq_quantize_workspace_bytes(L.R, L.C, g.bits, g.group_size, wl.block)),
+                                                   dtype=torch.uint8, device=dev) for g in wl.grids[1:]]
+            st["grid_streams"] = [torch.cuda.Stream(device=dev) for _ in wl.grids[1:]]
     torch.cuda.synchronize()
 
     stage_events = []                             # (layer idx, events) of the timed steps
@@ -280,7 +296,7 @@ def run_gpu(args, wl):
                  ("U", lambda: B.gptq_prepare_hinv(st["H"], wl.damp, U=st["U"], ws=st["ws"], dev_info=st["info"],
                                                    factor=factor and st["factor"]))] +
                 [(f"Q{gi}", (lambda gi=gi, g=g: st["out"].__setitem__(gi, B.gptq_quantize_layer(
-                    st["W"], st["U"], g.bits, g.group_size, g.sym, wl.block, ws=st["ws"], factor=factor and st["factor"]))))
+                    st["W"], st["U"], g.bits, g.group_size, g.sym, wl.block, ws=st["ws_g"][gi], factor=factor and st["factor"]))))
                  for gi, g in enumerate(wl.grids)])
 
     def run_stage(li, name, fn):
@@ -312,9 +328,19 @@ def run_gpu(args, wl):
                 cs.wait_event(after)
                 if record: ev[2].record(cs)
                 run_stage(li, *fns[1])
-                if record: ev[3].record(cs)
+                fac_done = ev[3] if record else torch.cuda.Event()
+                fac_done.record(cs)
+                joins = []
+                for gi, gs in enumerate(state[li]["grid_streams"], start=1):      # the other grids beside the first one
+                    with torch.cuda.stream(gs):
+                        gs.wait_event(fac_done)
+                        run_stage(li, *fns[2 + gi])
+                        joins.append(torch.cuda.Event()); joins[-1].record(gs)
                 for gi in range(len(wl.grids)):
-                    run_stage(li, *fns[2 + gi])
+                    if gi == 0 or not state[li]["grid_streams"]:
+                        run_stage(li, *fns[2 + gi])
+                for e in joins:
+                    cs.wait_event(e)
                 end = ev[4 + len(wl.grids) - 1] if record else torch.cuda.Event()
                 end.record(cs)
             done.append(end)
@@ -339,6 +365,13 @@ def run_gpu(args, wl):
                 main.wait_event(e)
             hessian(asc[-1])
             chain(asc[-1], h_done[asc[-1]])
+        elif args.schedule == "big-last":
+            # cheap layers first, each chain launched behind its Hessian; the most expensive layer's Hessian follows at once
+            # (the other chains get few SMs while it runs) and its chain, the longest, then shares the GPU with what is left
+            # of the others instead of running alone at the end
+            for li in list(layer_order)[::-1]:
+                hessian(li)
+                chain(li, h_done[li])
         else:
             for li in layer_order:
                 hessian(li)
@@ -404,6 +437,16 @@ def run_gpu(args, wl):
         d["hessian_ms"] += ev[0].elapsed_time(ev[1]) / args.steps
         d["hinv_ms"] += ev[2].elapsed_time(ev[3]) / args.steps
         d["quantize_ms"] += ev[3].elapsed_time(ev[3 + n_grids]) / args.steps
+    # when each layer's stages began and ended in the last timed step, in ms after the step's first launch
+    timeline = []
+    last_step = stage_events[-len(state):] if stage_events else []
+    if last_step:
+        t0 = last_step[0][1][0]
+        for li, ev in last_step:
+            timeline.append(dict(layer=state[li]["L"].name,
+                                 hessian=[round(t0.elapsed_time(ev[0]), 1), round(t0.elapsed_time(ev[1]), 1)],
+                                 factor=[round(t0.elapsed_time(ev[2]), 1), round(t0.elapsed_time(ev[3]), 1)],
+                                 quantize_end=round(t0.elapsed_time(ev[3 + n_grids]), 1)))
     peaks = _peaks()
     tot = {k: sum(d[k] for d in per.values()) for k in ("hessian_ms", "hinv_ms", "quantize_ms")}
     # roofline of the dominant kernel.  Hessian: algorithmic flops C (C + 1) m per launch (symmetric half).
@@ -480,10 +523,13 @@ def run_gpu(args, wl):
                                       "small-first": "small-first: the cheaper layers' Hessians back to back with their stages 2-3 side by side on "
                                                      "their own streams; the most expensive layer's Hessian starts when those have drained and "
                                                      "its stages 2-3 then run alone; stage 2-3 times of the cheaper layers overlap one another",
+                                      "big-last": "big-last: Hessians back to back, cheapest layer first, each layer's stages 2-3 on its own "
+                                                  "stream behind its Hessian; the most expensive layer's stages 2-3 run last, beside what is "
+                                                  "left of the others",
                                       "sequential": "sequential: one stream, layer after layer"}[args.schedule],
                             parallelism=f"layer-set replica per GPU x{world}"),
                 sec_per_layer=ms_per_step * 1e-3 / len(layers),
-                stage_ms=tot, per_layer=list(per.values()),
+                stage_ms=tot, per_layer=list(per.values()), timeline=timeline,
                 roofline=roof, stage_rooflines=stage_rooflines, gpu_launches=int(launches), clocks=clocks)
 
     if rank == 0 and world == 1 and not args.no_e2e:
@@ -825,11 +871,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-graphs", action="store_true", help="issue every kernel launch from the host instead of replaying CUDA graphs")
-    ap.add_argument("--schedule", default="pipelined", choices=["pipelined", "hessians-first", "small-first", "sequential"],
+    ap.add_argument("--schedule", default="pipelined", choices=["pipelined", "hessians-first", "small-first", "big-last", "sequential"],
                     help="pipelined: Hessians back to back on one stream, each layer's stages 2-3 on its own stream as soon as "
                          "its Hessian is done; hessians-first: all Hessians, then all layers' stages 2-3 side by side; "
                          "sequential: one stream, layer after layer")
     ap.add_argument("--no-overlap", action="store_true", help="same as --schedule sequential")
+    ap.add_argument("--grids-in-turn", action="store_true",
+                    help="overlapped schedules: run a layer's grids one after the other on the layer's stream (default: every "
+                         "grid after the first on a stream and workspace of its own, beside the first)")
     ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
                     help="weak (default): every rank solves its own copy of the layer set; strong: the same layer set, tokens of "
                          "every Hessian and rows of every layer sharded over the ranks with one all-reduce of H per layer")
