@@ -144,7 +144,8 @@ class HostLayerSolver:
     One copy stream carries all activations to the device, the most expensive layer first, in token chunks; on a second
     stream every layer's Hessian is accumulated chunk by chunk as its chunks land (H is a sum over tokens, Section 2), so
     the first Hessian starts after one chunk and the later layers' activations cross while the earlier layers are being
-    solved; stages 2 and 3 of a layer run on that layer's own stream as soon as its Hessian is complete, and its packed
+    solved; stages 2 and 3 of a layer run on that layer's own stream as soon as its Hessian is complete (every grid after the
+    first on a stream and workspace of its own, beside the first: the grids are independent once the factor exists), and its packed
     codes, scales, zero-points and losses are copied back on that stream.  All layers' activations are resident at once
     (buffers are allocated once, for the shapes given, and reused by every solve()).
     """
@@ -190,7 +191,12 @@ class HostLayerSolver:
                                    info_u=torch.zeros(2, dtype=torch.int32, device=dev),
                                    info_host=torch.empty((len(chunks) + 1, 2), dtype=torch.int32).pin_memory(),
                                    ws=torch.empty(ws_bytes, dtype=torch.uint8, device=dev),
-                                   stream=torch.cuda.Stream(device=dev), outs=outs))
+                                   stream=torch.cuda.Stream(device=dev), outs=outs,
+                                   # a layer's grids are independent once its factor exists: every grid after the first
+                                   # has a stream and a stage-3 workspace of its own and runs beside the first
+                                   grid_ws=[torch.empty(max(256, B.gptq_quantize_workspace_bytes(R, C, b, g, block)),
+                                                        dtype=torch.uint8, device=dev) for (b, g, _) in self.grids[1:]],
+                                   grid_streams=[torch.cuda.Stream(device=dev) for _ in self.grids[1:]]))
 
     def h2d_bytes(self):
         return sum(st["X"].numel() * 2 + st["W"].numel() * 2 for st in self.state)
@@ -230,11 +236,24 @@ class HostLayerSolver:
                 B.gptq_prepare_hinv(st["H"], self.damp, U=st["U"], ws=st["ws"], dev_info=st["info_u"], factor=st["factor"])
                 st["info_host"][:-1].copy_(st["info_h"], non_blocking=True)
                 st["info_host"][-1].copy_(st["info_u"], non_blocking=True)
-                for (b, g, sym), o in zip(self.grids, st["outs"]):
-                    r = B.gptq_quantize_layer(st["W"], st["U"], b, g, sym, self.block, ws=st["ws"], factor=st["factor"])
+                fac_done = torch.cuda.Event(); fac_done.record(s)
+
+                def grid(gi, ws):                 # stage 3 for one grid and its results' way back, on the current stream
+                    (b, g, sym), o = self.grids[gi], st["outs"][gi]
+                    r = B.gptq_quantize_layer(st["W"], st["U"], b, g, sym, self.block, ws=ws, factor=st["factor"])
                     for k, src in (("qweight", r["qweight"]), ("scales", r["scales"]), ("zeros", r["zeros"]), ("loss", r["loss"]),
                                    ("info", r["dev_info"])):
                         o[k].copy_(src, non_blocking=True)
+
+                joins = []
+                for gi, (gs, gws) in enumerate(zip(st["grid_streams"], st["grid_ws"]), start=1):
+                    with torch.cuda.stream(gs):
+                        gs.wait_event(fac_done)
+                        grid(gi, gws)
+                        joins.append(torch.cuda.Event()); joins[-1].record(gs)
+                grid(0, st["ws"])
+                for j in joins:
+                    s.wait_event(j)
                 e = torch.cuda.Event(); e.record(s); ends.append(e)
         for e in ends:
             e.synchronize()
