@@ -420,6 +420,31 @@ def test_rtn_layer_bit_exact_and_equals_solver_on_diagonal_hessian(B, bits, grou
         assert torch.equal(q["qweight"], out["qweight"])
 
 
+@pytest.mark.parametrize("bits,group,C,sym,fp16", [
+    (2, 256, 2304, False, False), (3, 32, 2080, False, False), (3, 64, 2112, False, True), (4, 256, 2304, True, False),
+    (8, 256, 1024, False, False), (2, 0, 2080, False, False), (8, 0, 2048, False, False), (3, 96, 2016, False, False),
+    (4, 384, 2304, False, True), (2, 160, 2080, True, False), (3, 256, 2304, False, False), (O.BITS_TERNARY, 128, 2176, False, False),
+    (4, 16, 2080, False, False), (3, 4, 2080, False, False), (4, 2080, 2080, False, False), (3, 1024, 4096, False, False)])
+def test_rtn_layer_every_kind_of_group(B, bits, group, C, sym, fp16):
+    """gptq_rtn_layer over the group sizes its three kernels serve: runs of power-of-two groups (32 ... 256, with a last run
+    that is not full and a row that is not a multiple of 256 columns), one warp per group (multiples of 32 that are not a
+    power of two, groups of several hundred columns, per-row grids) and the small groups (4, 8, 16); symmetric grids and
+    fp16-rounded scales included.  Codes, scales and zero-points bit for bit against the oracle."""
+    R = 37
+    L = _layer(R, C, 64, cfg=14)
+    W16 = L.w()
+    out = B.gptq_rtn_layer(torch.from_numpy(W16).cuda(), bits, group, sym, scale_fp16=fp16)
+    torch.cuda.synchronize()
+    codes_ref, _ = O.rtn(W16, bits, group, sym, scale_fp16=fp16)
+    codes = O.unpack_codes(out["qweight"].cpu().numpy().view(np.uint32), bits, C)
+    assert np.array_equal(codes, codes_ref)
+    assert np.array_equal(O.pack_codes(codes, bits), out["qweight"].cpu().numpy().view(np.uint32))
+    g = group if group > 0 else C
+    grids = [O.find_params(W16[:, j:j + g].astype(np.float64), bits, sym, fp16) for j in range(0, C, g)]
+    assert np.array_equal(out["scales"].cpu().numpy().astype(np.float64), np.stack([a for a, _ in grids], 1))
+    assert np.array_equal(out["zeros"].cpu().numpy().astype(np.float64), np.stack([b for _, b in grids], 1))
+
+
 @pytest.mark.parametrize("bits,group,C", [(4, 0, 2048), (3, 128, 2048), (2, 32, 2048), (O.BITS_TERNARY, 8, 2048), (8, 0, 2048),
                                           (3, 0, 2048), (2, 128, 2048), (4, 128, 4096), (4, 1024, 2048), (O.BITS_TERNARY, 0, 2080),
                                           (8, 128, 1024), (3, 0, 2144), (4, 0, 96), (3, 384, 768)])
