@@ -730,7 +730,8 @@ def run_e2e(args, wl, state, device_value):
                 d2h_bytes_per_step=int(solver.d2h_bytes()), ms_per_step=dt * 1e3, steps=steps,
                 api="pipeline.HostLayerSolver.solve (pinned host buffers; one copy stream, the most expensive layer's activations "
                     "first, in token chunks of up to 4 GiB; Hessians accumulated chunk by chunk as the chunks land; every layer's stages "
-                    f"2-3 on its own stream, all {len(grids)} grid(s) from one Hessian and factor; results copied back to pinned memory)")
+                    f"2-3 on its own stream, replayed from a CUDA graph after the first solve, all {len(grids)} grid(s) from one Hessian "
+                    "and factor and side by side; results copied back to pinned memory)")
 
 
 def run_inference(args, wl):

@@ -150,12 +150,13 @@ class HostLayerSolver:
     (buffers are allocated once, for the shapes given, and reused by every solve()).
     """
 
-    def __init__(self, shapes: Sequence[tuple], grids: Sequence[tuple], block=128, damp=0.01, chunk_bytes=4 << 30, device=None,
+    def __init__(self, shapes: Sequence[tuple], grids: Sequence[tuple], block=128, damp=0.01, chunk_bytes=4 << 30, device=None, graphs=True,
                  factor=False):
         """shapes: (R, C, n_tokens) per layer; grids: (bits, group_size, sym) per grid."""
         dev = torch.device("cuda", torch.cuda.current_device()) if device is None else device
-        self.grids, self.block, self.damp = list(grids), block, damp
+        self.grids, self.block, self.damp, self.graphs = list(grids), block, damp, bool(graphs)
         # factor: stages 2 and 3 in the factor form (see BlockSolver) for the layers where it pays
+        # graphs: after the first solve(), every layer's stages 2-3 are replayed from a CUDA graph
         self.order = sorted(range(len(shapes)), key=lambda i: -(shapes[i][1] ** 2) * (shapes[i][2] + shapes[i][1]))
         self.copy_stream = torch.cuda.Stream(device=dev)
         self.main = torch.cuda.Stream(device=dev)
@@ -233,27 +234,10 @@ class HostLayerSolver:
             s = st["stream"]
             with torch.cuda.stream(s):
                 s.wait_event(h_done); s.wait_event(landed[(li, "W")])
-                B.gptq_prepare_hinv(st["H"], self.damp, U=st["U"], ws=st["ws"], dev_info=st["info_u"], factor=st["factor"])
-                st["info_host"][:-1].copy_(st["info_h"], non_blocking=True)
-                st["info_host"][-1].copy_(st["info_u"], non_blocking=True)
-                fac_done = torch.cuda.Event(); fac_done.record(s)
-
-                def grid(gi, ws):                 # stage 3 for one grid and its results' way back, on the current stream
-                    (b, g, sym), o = self.grids[gi], st["outs"][gi]
-                    r = B.gptq_quantize_layer(st["W"], st["U"], b, g, sym, self.block, ws=ws, factor=st["factor"])
-                    for k, src in (("qweight", r["qweight"]), ("scales", r["scales"]), ("zeros", r["zeros"]), ("loss", r["loss"]),
-                                   ("info", r["dev_info"])):
-                        o[k].copy_(src, non_blocking=True)
-
-                joins = []
-                for gi, (gs, gws) in enumerate(zip(st["grid_streams"], st["grid_ws"]), start=1):
-                    with torch.cuda.stream(gs):
-                        gs.wait_event(fac_done)
-                        grid(gi, gws)
-                        joins.append(torch.cuda.Event()); joins[-1].record(gs)
-                grid(0, st["ws"])
-                for j in joins:
-                    s.wait_event(j)
+                if st.get("graph") is not None:
+                    st["graph"].replay()
+                else:
+                    self._chain(st, s)
                 e = torch.cuda.Event(); e.record(s); ends.append(e)
         for e in ends:
             e.synchronize()
@@ -264,4 +248,42 @@ class HostLayerSolver:
             for o in st["outs"]:
                 if o["info"].tolist()[0] != 0:
                     raise B.GptqError(o["info"].tolist()[0], f"layer {li}: gptq_quantize_layer")
+        if self.graphs and any(st.get("graph") is None for st in self.state):
+            self._capture()
         return [st["outs"] for st in self.state]
+
+    def _chain(self, st, s):
+        """Stages 2 and 3 of one layer and their results' way back to the host, enqueued on s (the current stream)."""
+        B.gptq_prepare_hinv(st["H"], self.damp, U=st["U"], ws=st["ws"], dev_info=st["info_u"], factor=st["factor"])
+        st["info_host"][:-1].copy_(st["info_h"], non_blocking=True)
+        st["info_host"][-1].copy_(st["info_u"], non_blocking=True)
+        fac_done = torch.cuda.Event(); fac_done.record(s)
+
+        def grid(gi, ws):                         # stage 3 for one grid and its results' way back, on the current stream
+            (b, g, sym), o = self.grids[gi], st["outs"][gi]
+            r = B.gptq_quantize_layer(st["W"], st["U"], b, g, sym, self.block, ws=ws, factor=st["factor"])
+            for k, src in (("qweight", r["qweight"]), ("scales", r["scales"]), ("zeros", r["zeros"]), ("loss", r["loss"]),
+                           ("info", r["dev_info"])):
+                o[k].copy_(src, non_blocking=True)
+
+        joins = []
+        for gi, (gs, gws) in enumerate(zip(st["grid_streams"], st["grid_ws"]), start=1):
+            with torch.cuda.stream(gs):
+                gs.wait_event(fac_done)
+                grid(gi, gws)
+                joins.append(torch.cuda.Event()); joins[-1].record(gs)
+        grid(0, st["ws"])
+        for j in joins:
+            s.wait_event(j)
+
+    def _capture(self):
+        """After the first solve() (which ran eagerly and was checked): every layer's stages 2-3 become one CUDA graph,
+        the same kernels on the same buffers, so that later solves issue a few graph launches instead of thousands of
+        kernel launches from the host."""
+        torch.cuda.synchronize()
+        for st in self.state:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=st["stream"]):
+                self._chain(st, st["stream"])
+            st["graph"] = g
+        torch.cuda.synchronize()
