@@ -98,6 +98,17 @@ size_t gptq_hessian_workspace_bytes(int C, int64_t n_tokens);
 gptq_status_t gptq_hessian_accumulate(float* H, const void* X_bf16, int64_t n_tokens, int C,
                                       void* ws, size_t ws_bytes, int* dev_info, void* stream);
 
+/* The same sum for a caller that feeds one Hessian in several chunks (Section 5, Setup: Hessians are summed over
+ * calibration batches).  Only tiles on or above the diagonal are computed; gptq_hessian_accumulate ends with a pass
+ * that copies the upper triangle onto the lower one (2 C^2 floats of traffic), which only the last chunk needs.
+ *   gptq_hessian_accumulate_upper  adds to the upper triangle (diagonal included) and leaves the strictly lower
+ *                                  triangle as it is: it is stale until a later gptq_hessian_accumulate on the same H or
+ *                                  gptq_hessian_symmetrize has run.  Arguments and errors as for gptq_hessian_accumulate.
+ *   gptq_hessian_symmetrize        H[i][j] = H[j][i] for i > j (C % 32 == 0, H 16-byte aligned). */
+gptq_status_t gptq_hessian_accumulate_upper(float* H, const void* X_bf16, int64_t n_tokens, int C,
+                                            void* ws, size_t ws_bytes, int* dev_info, void* stream);
+gptq_status_t gptq_hessian_symmetrize(float* H, int C, void* stream);
+
 /* ------------------------------------------------------------------ stage 2
  * lambda = damp * mean(diag H);  H~ = H + lambda I          (Section 3, Step 3)
  * U = Cholesky(H~^-1)^T: upper triangular, positive diagonal, U^T U = H~^-1

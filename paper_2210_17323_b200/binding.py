@@ -44,6 +44,10 @@ def _load():
     lib.gptq_hessian_workspace_bytes.argtypes = [c.c_int, c.c_int64]
     lib.gptq_hessian_accumulate.restype = c.c_int
     lib.gptq_hessian_accumulate.argtypes = [c.c_void_p, c.c_void_p, c.c_int64, c.c_int, c.c_void_p, c.c_size_t, c.c_void_p, c.c_void_p]
+    lib.gptq_hessian_accumulate_upper.restype = c.c_int
+    lib.gptq_hessian_accumulate_upper.argtypes = lib.gptq_hessian_accumulate.argtypes
+    lib.gptq_hessian_symmetrize.restype = c.c_int
+    lib.gptq_hessian_symmetrize.argtypes = [c.c_void_p, c.c_int, c.c_void_p]
     lib.gptq_prepare_hinv_workspace_bytes.restype = c.c_size_t
     lib.gptq_prepare_hinv_workspace_bytes.argtypes = [c.c_int]
     lib.gptq_prepare_hinv.restype = c.c_int
@@ -145,19 +149,30 @@ def gptq_quantize_workspace_bytes(R, C, bits, group_size, block):
     return _lib.gptq_quantize_workspace_bytes(R, C, bits, group_size, block)
 
 
-def gptq_hessian_accumulate(H, X, n_tokens=None, ws=None, dev_info=None, stream=None):
-    """H += 2 X^T X for token-major bf16 X (n_tokens x C).  H: C x C fp32, zeroed by the caller first."""
+def gptq_hessian_accumulate(H, X, n_tokens=None, ws=None, dev_info=None, stream=None, upper_only=False):
+    """H += 2 X^T X for token-major bf16 X (n_tokens x C).  H: C x C fp32, zeroed by the caller first.
+    upper_only: gptq_hessian_accumulate_upper (a chunk that is not the last one: the lower triangle stays stale)."""
     with _alloc_on(stream):
         _check(H, torch.float32, "H")
         _check(X, torch.bfloat16, "X")
         C = H.shape[0]
         n = X.shape[0] if n_tokens is None else int(n_tokens)
         ws = _ws(_lib.gptq_hessian_workspace_bytes(C, n), H.device, ws)
-        st = _lib.gptq_hessian_accumulate(H.data_ptr(), X.data_ptr(), n, C, ws.data_ptr(), ws.numel(),
-                                          None if dev_info is None else dev_info.data_ptr(), _stream_ptr(stream))
+        fn = _lib.gptq_hessian_accumulate_upper if upper_only else _lib.gptq_hessian_accumulate
+        st = fn(H.data_ptr(), X.data_ptr(), n, C, ws.data_ptr(), ws.numel(),
+                None if dev_info is None else dev_info.data_ptr(), _stream_ptr(stream))
         if st != OK:
             raise GptqError(st, "gptq_hessian_accumulate")
         return H
+
+
+def gptq_hessian_symmetrize(H, stream=None):
+    """Copies the upper triangle of H onto the lower one (after chunks added with upper_only=True)."""
+    _check(H, torch.float32, "H")
+    st = _lib.gptq_hessian_symmetrize(H.data_ptr(), H.shape[0], _stream_ptr(stream))
+    if st != OK:
+        raise GptqError(st, "gptq_hessian_symmetrize")
+    return H
 
 
 def gptq_prepare_hinv(H, damp=0.01, U=None, ws=None, dev_info=None, stream=None, factor=False):

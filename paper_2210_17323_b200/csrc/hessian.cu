@@ -66,7 +66,7 @@ cudaError_t launch_mirror_upper_to_lower(float* H, int C, cudaStream_t stream) {
 }
 
 static gptq_status_t hessian_simt(float* H, const __nv_bfloat16* X, int64_t n_tokens, int C,
-                                  cudaStream_t stream) {
+                                  cudaStream_t stream, bool mirror) {
   const int64_t kMaxTokensPerLaunch = 1 << 30;  // K indices are 32-bit inside the tile kernel
   for (int64_t t0 = 0; t0 < n_tokens; t0 += kMaxTokensPerLaunch) {
     int64_t nt = n_tokens - t0 < kMaxTokensPerLaunch ? n_tokens - t0 : kMaxTokensPerLaunch;
@@ -78,7 +78,7 @@ static gptq_status_t hessian_simt(float* H, const __nv_bfloat16* X, int64_t n_to
     GPTQ_CUDA_TRY(launch_gemm_simt(C, C, nz, XtAsA{x, C}, XtAsB{x, C}, UpperTilesSplitK{nt},
                                    AddTwiceUpper{H, C}, stream));
   }
-  GPTQ_CUDA_TRY(launch_mirror_upper_to_lower(H, C, stream));
+  if (mirror) GPTQ_CUDA_TRY(launch_mirror_upper_to_lower(H, C, stream));
   return GPTQ_OK;
 }
 
@@ -89,16 +89,34 @@ extern "C" size_t gptq_hessian_workspace_bytes(int C, int64_t n_tokens) {
   return 0;
 }
 
-extern "C" gptq_status_t gptq_hessian_accumulate(float* H, const void* X_bf16, int64_t n_tokens, int C,
-                                                 void* ws, size_t ws_bytes, int* dev_info, void* stream) {
+static gptq_status_t hessian_accumulate_impl(float* H, const void* X_bf16, int64_t n_tokens, int C, int* dev_info,
+                                             void* stream, bool mirror) {
   using namespace gptq;
-  (void)ws; (void)ws_bytes;
   if (!H || C <= 0 || C % 32 != 0 || n_tokens < 0) return GPTQ_ERR_INVALID_ARG;
   if (n_tokens == 0) return GPTQ_OK;
   if (!X_bf16 || !aligned_to(X_bf16, 16) || !aligned_to(H, 16)) return GPTQ_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(X_bf16);
   if (dev_info) GPTQ_CUDA_TRY(cudaMemsetAsync(dev_info, 0, 2 * sizeof(int), s));
-  if (hessian_umma_supported(C, n_tokens)) return hessian_umma(H, X, n_tokens, C, dev_info, s);
-  return hessian_simt(H, X, n_tokens, C, s);
+  if (hessian_umma_supported(C, n_tokens)) return hessian_umma(H, X, n_tokens, C, dev_info, s, mirror);
+  return hessian_simt(H, X, n_tokens, C, s, mirror);
+}
+
+extern "C" gptq_status_t gptq_hessian_accumulate(float* H, const void* X_bf16, int64_t n_tokens, int C,
+                                                 void* ws, size_t ws_bytes, int* dev_info, void* stream) {
+  (void)ws; (void)ws_bytes;
+  return hessian_accumulate_impl(H, X_bf16, n_tokens, C, dev_info, stream, true);
+}
+
+extern "C" gptq_status_t gptq_hessian_accumulate_upper(float* H, const void* X_bf16, int64_t n_tokens, int C,
+                                                       void* ws, size_t ws_bytes, int* dev_info, void* stream) {
+  (void)ws; (void)ws_bytes;
+  return hessian_accumulate_impl(H, X_bf16, n_tokens, C, dev_info, stream, false);
+}
+
+extern "C" gptq_status_t gptq_hessian_symmetrize(float* H, int C, void* stream) {
+  using namespace gptq;
+  if (!H || C <= 0 || C % 32 != 0 || !aligned_to(H, 16)) return GPTQ_ERR_INVALID_ARG;
+  GPTQ_CUDA_TRY(launch_mirror_upper_to_lower(H, C, static_cast<cudaStream_t>(stream)));
+  return GPTQ_OK;
 }

@@ -257,7 +257,7 @@ bool hessian_umma_supported(int C, int64_t n_tokens) {
 }
 
 gptq_status_t hessian_umma(float* H, const __nv_bfloat16* X, int64_t n_tokens, int C, int* dev_info,
-                           cudaStream_t stream) {
+                           cudaStream_t stream, bool mirror) {
   CUtensorMap tmap;
   gptq_status_t st = make_tmap_2d(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)C, (uint64_t)n_tokens,
                                   (uint64_t)C * 2, 64, BK);
@@ -299,7 +299,7 @@ gptq_status_t hessian_umma(float* H, const __nv_bfloat16* X, int64_t n_tokens, i
                                        dev_info, stream);
   }
   if (st != GPTQ_OK) return st;
-  GPTQ_CUDA_TRY(launch_mirror_upper_to_lower(H, C, stream));
+  if (mirror) GPTQ_CUDA_TRY(launch_mirror_upper_to_lower(H, C, stream));
   return GPTQ_OK;
 }
 

@@ -175,7 +175,9 @@ gptq_status_t solve_layer_host_enqueue(const HostWs& w, StreamGuard& g, cudaStre
     }
     GPTQ_CUDA_TRY(cudaStreamWaitEvent(s, g.loaded[b], 0));
     // every chunk reports into the spare slot info[6..7]; the first non-OK report is kept in info[0..1]
-    st = gptq_hessian_accumulate(w.H, w.X[b], nt, C, w.stage_ws, w.stage_ws_bytes, w.info + 6, s);
+    // only the last chunk needs the pass that copies the upper triangle of H onto the lower one
+    st = (t0 + nt < n_tokens ? gptq_hessian_accumulate_upper : gptq_hessian_accumulate)(w.H, w.X[b], nt, C, w.stage_ws, w.stage_ws_bytes,
+                                                                                        w.info + 6, s);
     if (st != GPTQ_OK) return st;
     fold_info_kernel<<<1, 1, 0, s>>>(w.info, w.info + 6);
     GPTQ_LAUNCH_CHECK();

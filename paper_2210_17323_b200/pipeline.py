@@ -157,7 +157,10 @@ class HostLayerSolver:
         self.grids, self.block, self.damp, self.graphs = list(grids), block, damp, bool(graphs)
         # factor: stages 2 and 3 in the factor form (see BlockSolver) for the layers where it pays
         # graphs: after the first solve(), every layer's stages 2-3 are replayed from a CUDA graph
-        self.order = sorted(range(len(shapes)), key=lambda i: -(shapes[i][1] ** 2) * (shapes[i][2] + shapes[i][1]))
+        # most expensive layer first (Hessian C^2 n, factor ~ C^3, stage 3 ~ 3 R C^2 executed per grid): the layers whose
+        # activations cross last are then the cheapest ones, and the solve ends soon after the last copy
+        self.order = sorted(range(len(shapes)), key=lambda i: -(shapes[i][1] ** 2) * (shapes[i][2] + shapes[i][1] +
+                                                                                   3 * len(self.grids) * shapes[i][0]))
         self.copy_stream = torch.cuda.Stream(device=dev)
         self.main = torch.cuda.Stream(device=dev)
         self.state = []
@@ -229,7 +232,8 @@ class HostLayerSolver:
                 st["H"].zero_()
                 for ci, (t0, t1) in enumerate(st["chunks"]):
                     self.main.wait_event(landed[(li, ci)])
-                    B.gptq_hessian_accumulate(st["H"], st["X"][t0:t1], ws=st["ws"], dev_info=st["info_h"][ci])
+                    B.gptq_hessian_accumulate(st["H"], st["X"][t0:t1], ws=st["ws"], dev_info=st["info_h"][ci],
+                                              upper_only=ci + 1 < len(st["chunks"]))    # the last chunk mirrors H
                 h_done = torch.cuda.Event(); h_done.record(self.main)
             s = st["stream"]
             with torch.cuda.stream(s):

@@ -77,6 +77,30 @@ def test_hessian_integer_inputs_bit_exact_and_chunked(B):
     assert np.array_equal(H.cpu().numpy().astype(np.float64), exact)
 
 
+@pytest.mark.parametrize("C", [160, 1056])
+def test_hessian_chunks_into_the_upper_triangle_then_one_mirror(B, C):
+    """gptq_hessian_accumulate_upper adds to the upper triangle only and never writes strictly below the diagonal tiles'
+    rows; the last chunk (gptq_hessian_accumulate) or gptq_hessian_symmetrize completes H.  Integer-valued inputs: every
+    result is exact, so the chunked sum must equal the one-call sum bit for bit."""
+    r = np.random.default_rng(C)
+    m = 900
+    Xi = r.integers(-8, 9, size=(m, C)).astype(np.float32)
+    Xt = torch.from_numpy(Xi).cuda().to(torch.bfloat16)
+    exact = 2.0 * (Xi.astype(np.float64).T @ Xi.astype(np.float64))
+    H = torch.zeros((C, C), dtype=torch.float32, device="cuda")
+    B.gptq_hessian_accumulate(H, Xt[:100].contiguous(), upper_only=True)
+    B.gptq_hessian_accumulate(H, Xt[100:577].contiguous(), upper_only=True)
+    Hu = H.cpu().numpy().astype(np.float64)
+    part = 2.0 * (Xi[:577].astype(np.float64).T @ Xi[:577].astype(np.float64))
+    assert np.array_equal(np.triu(Hu), np.triu(part))                     # the upper triangle is complete after every call
+    B.gptq_hessian_accumulate(H, Xt[577:].contiguous())                     # the last chunk mirrors
+    assert np.array_equal(H.cpu().numpy().astype(np.float64), exact)
+    H2 = torch.zeros((C, C), dtype=torch.float32, device="cuda")
+    B.gptq_hessian_accumulate(H2, Xt, upper_only=True)
+    B.gptq_hessian_symmetrize(H2)
+    assert np.array_equal(H2.cpu().numpy().astype(np.float64), exact)
+
+
 # ------------------------------------------------------------------ stage 2
 @pytest.mark.parametrize("C", [32, 96, 160, 768, 1056, 2304])
 def test_prepare_hinv_matches_oracle(B, C):
