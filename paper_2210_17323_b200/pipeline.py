@@ -165,9 +165,16 @@ class HostLayerSolver:
         self.main = torch.cuda.Stream(device=dev)
         self.state = []
         for li, (R, C, n) in enumerate(shapes):
-            # token chunks of about chunk_bytes; the layer whose activations cross first starts with two short chunks
-            # (1/8 and 1/2 of a chunk) so that its Hessian is under way after a few tens of milliseconds
-            sizes = ([chunk_bytes // 8, chunk_bytes // 2] if li == self.order[0] else []) + [chunk_bytes]
+            # token chunks of about chunk_bytes.  The layer whose activations cross first starts with short chunks that grow
+            # by a quarter each: its Hessian is under way after a few milliseconds, and a chunk's copy never takes longer than
+            # the accumulation of the chunk before it as long as accumulating is at least 1.25 x slower than copying (true of
+            # the layers this order puts first), so the GPU does not wait for the next chunk
+            sizes = []
+            if li == self.order[0]:
+                b = chunk_bytes / 16
+                while b < chunk_bytes:
+                    sizes.append(int(b)); b *= 1.25
+            sizes.append(chunk_bytes)
             chunks, t0 = [], 0
             while t0 < n:
                 cb = sizes[min(len(chunks), len(sizes) - 1)]
