@@ -271,7 +271,8 @@ gptq_status_t gptq_matvec(const uint32_t* qweight, const float* scales, const fl
 
 /* ------------------------------------------------------------------ whole layer, host buffers
  * Stages 1-3 for one layer whose inputs and outputs live in HOST memory (Eq. 1's W and X in, the
- * packed W^ out): X is streamed to the device in token chunks of about 2 GiB, double-buffered on
+ * packed W^ out): X is streamed to the device in token chunks of up to about 2 GiB (the first ones short,
+ * growing by a quarter each, so that the accumulation starts after a few milliseconds), double-buffered on
  * an internal copy stream so that the transfer of a chunk overlaps the Hessian accumulation of the
  * previous one (Section 5, Setup: Hessians are accumulated over calibration batches); then
  * gptq_prepare_hinv and gptq_quantize_layer run and the results are copied back.

@@ -162,10 +162,19 @@ gptq_status_t solve_layer_host_enqueue(const HostWs& w, StreamGuard& g, cudaStre
   GPTQ_CUDA_TRY(cudaMemsetAsync(w.info, 0, 8 * sizeof(int), s));
   const __nv_bfloat16* Xh = static_cast<const __nv_bfloat16*>(X_bf16_host);
   gptq_status_t st;
+  // Chunks grow by a quarter each from 1/16 of the full chunk: the Hessian is under way after a few milliseconds, and a
+  // chunk's copy does not outlast the accumulation of the chunk before it wherever accumulating is at least 1.25 x slower
+  // than copying (wide layers); for narrow layers the copy is the bound either way.
   int k = 0;
-  for (int64_t t0 = 0; t0 < n_tokens; t0 += w.chunk_tokens, ++k) {
+  double grow = (double)w.chunk_tokens / 16.0;
+  int64_t nt = 0;
+  for (int64_t t0 = 0; t0 < n_tokens; t0 += nt, ++k) {
     const int b = k & 1;
-    const int64_t nt = n_tokens - t0 < w.chunk_tokens ? n_tokens - t0 : w.chunk_tokens;
+    int64_t want = grow >= (double)w.chunk_tokens ? w.chunk_tokens : (int64_t)grow / 64 * 64;
+    if (want < 64) want = 64;
+    if (want > w.chunk_tokens) want = w.chunk_tokens;
+    grow *= 1.25;
+    nt = n_tokens - t0 < want ? n_tokens - t0 : want;
     if (k >= 2) GPTQ_CUDA_TRY(cudaStreamWaitEvent(g.s, g.freed[b], 0));       // buffer b consumed by chunk k-2
     GPTQ_CUDA_TRY(cudaMemcpyAsync(w.X[b], Xh + t0 * C, (size_t)nt * C * 2, cudaMemcpyHostToDevice, g.s));
     GPTQ_CUDA_TRY(cudaEventRecord(g.loaded[b], g.s));

@@ -641,6 +641,28 @@ def test_solve_layer_from_host_buffers_several_grids(B):
     assert (a == b).mean() >= 0.999
 
 
+def test_solve_layer_host_streams_x_in_growing_chunks(B):
+    """gptq_solve_layer_host with more tokens than its first chunks hold (the chunks grow by a quarter each from 1/16 of
+    the full chunk; all but the last add to the upper triangle of H only).  Small-integer activations make every sum of the
+    Hessian exact, so the result must equal, bit for bit, that of the three device calls on the whole X at once."""
+    R, C, n = 48, 2048, 110000                      # full chunk = 2 GiB / (2 C) = 524288 tokens: chunks of 32768, 40960, 36272
+    r = np.random.default_rng(21)
+    Xi = r.integers(-3, 4, size=(n, C)).astype(np.float32)
+    Xi[:, ::7] *= 2.0                               # a spread of channel energies
+    Xh = torch.from_numpy(Xi).to(torch.bfloat16).contiguous().pin_memory()
+    Wh = torch.from_numpy(_layer(R, C, 64, cfg=15).w()).pin_memory()
+    host = B.gptq_solve_layer_host(Wh, Xh, 4, 128, False, 128, 0.01)
+    assert host["info"].tolist() == [0, 0]
+    H = torch.zeros((C, C), dtype=torch.float32, device="cuda")
+    B.gptq_hessian_accumulate(H, Xh.cuda())
+    F, info = B.gptq_prepare_hinv(H, 0.01, factor=True)      # the host call takes the factor form for C > 1024
+    dev = B.gptq_quantize_layer(Wh.cuda(), F, 4, 128, False, 128, factor=True)
+    torch.cuda.synchronize()
+    assert info.tolist() == [0, 0] and dev["dev_info"].tolist() == [0, 0]
+    assert torch.equal(host["qweight"], dev["qweight"].cpu())
+    assert torch.equal(host["scales"], dev["scales"].cpu()) and torch.equal(host["zeros"], dev["zeros"].cpu())
+
+
 def test_host_layer_solver_matches_the_oracle(B):
     """pipeline.HostLayerSolver: several layers from pinned host buffers in one overlapped schedule (one copy stream,
     Hessians chunk by chunk as the chunks land, every layer's stages 2-3 on its own stream, results back on the host).
